@@ -1,0 +1,249 @@
+"""CPU oracle for the TP a->b re-layout (test infrastructure, not part of the product).
+
+Thin numpy marshalling around ``amoeba_oracle.c`` (plain C element loops, compiled with gcc).  Only the tests,
+the smoke check and the benchmark's CPU-baseline leg import this package; the CUDA library and its Python
+binding never do, and nothing here imports them.
+
+Conventions (see the C file for the passages of the paper each function follows):
+  * elements are opaque 16-bit words, numpy ``uint16``;
+  * logical KV is ``KV[L][G][Hkv][2][D]`` with ``G`` the number of block-padded tokens of all sequences;
+  * a KV pool of one worker is ``pool[L][NB][Hkv/TP][2][T][D]``;
+  * one layer's logical weights are a dict ``{q,k,v,o,gate,up,down}`` of ``[out,in]`` arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "amoeba_oracle.c"
+_LIB = _HERE / "liboracle.so"
+
+OK, INVALID_ARG, NO_FREE_BLOCKS, BAD_BLOCK_ID = 0, 1, 4, 5
+
+
+def build(force: bool = False) -> Path:
+    """Compile the C oracle with gcc (no CUDA involved)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.run(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-o", str(tmp), str(_SRC)],
+                       check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Model(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("L", "hidden", "Hq", "Hkv", "D", "I")]
+
+
+class _Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q", "k", "v", "o", "gate", "up", "down")]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(str(build()))
+    return _lib
+
+
+def _model(m: dict) -> _Model:
+    return _Model(m["L"], m["hidden"], m["Hq"], m["Hkv"], m["D"], m["I"])
+
+
+def _i32(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def _ptr_array(arrs):
+    return (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+
+
+def set_threads(n: int) -> None:
+    """Number of OpenMP threads the layer loops may use (1 = serial)."""
+    os.environ["OMP_NUM_THREADS"] = str(n)
+    try:
+        omp = C.CDLL("libgomp.so.1")
+        omp.omp_set_num_threads(int(n))
+    except OSError:
+        pass
+
+
+def header_range(H: int, TP: int, i: int):
+    """1-indexed inclusive range of headers kept by worker W_i (Sec. 3.1)."""
+    f, l = C.c_int(), C.c_int()
+    lib().oracle_header_range(H, TP, i, C.byref(f), C.byref(l))
+    return f.value, l.value
+
+
+def worker_of_header(H: int, TP: int, header: int) -> int:
+    return lib().oracle_worker_of_header(H, TP, header)
+
+
+def padded_tokens(seq_lens, T: int) -> int:
+    sl, slp = _i32(seq_lens)
+    f = lib().oracle_padded_tokens
+    f.restype = C.c_int64
+    return f(len(sl), slp, T)
+
+
+def pool_elems_per_layer(m: dict, T: int, TP: int, NB: int) -> int:
+    return NB * (m["Hkv"] // TP) * 2 * T * m["D"]
+
+
+def kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=0xA5A5, layer_stride=None):
+    """Logical KV -> list of TP pools ``[L][NB][Hkv/TP][2][T][D]`` (uint16), untouched words = ``fill``."""
+    sl, slp = _i32(seq_lens)
+    bt, btp = _i32(bt)
+    per = pool_elems_per_layer(m, T, TP, NB)
+    stride = per if layer_stride is None else layer_stride
+    pools = [np.full(m["L"] * stride, fill, dtype=np.uint16) for _ in range(TP)]
+    KV = np.ascontiguousarray(KV, dtype=np.uint16)
+    mm = _model(m)
+    lib().oracle_kv_shard(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(stride), len(sl), slp, btp,
+                          bt.shape[1], _ptr_array(pools))
+    return pools
+
+
+def kv_shard_into(KV, m, T, TP, seq_lens, bt, pools, layer_stride):
+    """Same as kv_shard but writes over existing pools (their other words are preserved)."""
+    sl, slp = _i32(seq_lens)
+    bt, btp = _i32(bt)
+    KV = np.ascontiguousarray(KV, dtype=np.uint16)
+    mm = _model(m)
+    lib().oracle_kv_shard(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(layer_stride), len(sl), slp,
+                          btp, bt.shape[1], _ptr_array(pools))
+
+
+def kv_reconstruct(pools, m, T, TP, NB, seq_lens, bt, layer_stride=None):
+    sl, slp = _i32(seq_lens)
+    bt, btp = _i32(bt)
+    G = padded_tokens(sl, T)
+    KV = np.zeros((m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    stride = pool_elems_per_layer(m, T, TP, NB) if layer_stride is None else layer_stride
+    mm = _model(m)
+    lib().oracle_kv_reconstruct(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(stride), len(sl), slp,
+                                btp, bt.shape[1], _ptr_array(pools))
+    return KV
+
+
+def kv_transform(m, T, seq_lens, a, NB_src, src_bt, src_pools, b, NB_dst, dst_bt, dst_pools):
+    """TP a->b on the KV pools: writes the live blocks of ``dst_pools`` in place (reconstruct, then shard)."""
+    sl, slp = _i32(seq_lens)
+    sbt, sbtp = _i32(src_bt)
+    dbt, dbtp = _i32(dst_bt)
+    assert sbt.shape == dbt.shape
+    mm = _model(m)
+    rc = lib().oracle_kv_transform(C.byref(mm), T, len(sl), slp, sbt.shape[1], a,
+                                   C.c_int64(pool_elems_per_layer(m, T, a, NB_src)), sbtp, _ptr_array(src_pools), b,
+                                   C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)), dbtp, _ptr_array(dst_pools))
+    assert rc == 0
+
+
+def kv_copy_pairs(m, T, a, NB_src, src_pools, b, NB_dst, dst_pools, pairs, num_pairs, status=0):
+    pr, prp = _i32(pairs)
+    st = C.c_int32(status)
+    mm = _model(m)
+    lib().oracle_kv_copy_pairs(C.byref(mm), T, a, NB_src, C.c_int64(pool_elems_per_layer(m, T, a, NB_src)),
+                               _ptr_array(src_pools), b, NB_dst, C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)),
+                               _ptr_array(dst_pools), prp, int(num_pairs), C.byref(st))
+    return st.value
+
+
+WEIGHT_NAMES = ("q", "k", "v", "o", "gate", "up", "down")
+
+
+def shard_shapes(m: dict, TP: int, fused_qkv=True, fused_gate_up=True) -> dict:
+    """Shapes of one worker's weight buffers for one layer."""
+    hid, qr, kr, I = m["hidden"], m["Hq"] * m["D"] // TP, m["Hkv"] * m["D"] // TP, m["I"] // TP
+    sh = {"o": (hid, qr), "down": (hid, I)}
+    if fused_qkv:
+        sh["q"] = (qr + 2 * kr, hid)
+    else:
+        sh.update(q=(qr, hid), k=(kr, hid), v=(kr, hid))
+    if fused_gate_up:
+        sh["gate"] = (2 * I, hid)
+    else:
+        sh.update(gate=(I, hid), up=(I, hid))
+    return sh
+
+
+def _wstruct(d: dict) -> _Weights:
+    return _Weights(*[(d[n].ctypes.data if n in d else None) for n in WEIGHT_NAMES])
+
+
+def empty_shards(m, TP, fused_qkv=True, fused_gate_up=True, fill=0xA5A5):
+    return [{n: np.full(s, fill, dtype=np.uint16) for n, s in shard_shapes(m, TP, fused_qkv, fused_gate_up).items()}
+            for _ in range(TP)]
+
+
+def weights_shard(logical: dict, m, TP, fused_qkv=True, fused_gate_up=True):
+    """One layer's logical weights -> list of TP shard dicts (fused buffers live under 'q' and 'gate')."""
+    shards = empty_shards(m, TP, fused_qkv, fused_gate_up)
+    lg = _wstruct(logical)
+    mm = _model(m)
+    for r in range(TP):
+        sh = _wstruct(shards[r])
+        lib().oracle_weights_shard(C.byref(mm), TP, r, int(fused_qkv), int(fused_gate_up), C.byref(lg), C.byref(sh))
+    return shards
+
+
+def logical_shapes(m: dict) -> dict:
+    hid, qr, kr, I = m["hidden"], m["Hq"] * m["D"], m["Hkv"] * m["D"], m["I"]
+    return {"q": (qr, hid), "k": (kr, hid), "v": (kr, hid), "o": (hid, qr), "gate": (I, hid), "up": (I, hid),
+            "down": (hid, I)}
+
+
+def weights_reconstruct(shards, m, TP, fused_qkv=True, fused_gate_up=True):
+    logical = {n: np.zeros(s, dtype=np.uint16) for n, s in logical_shapes(m).items()}
+    lg = _wstruct(logical)
+    mm = _model(m)
+    for r in range(TP):
+        sh = _wstruct(shards[r])
+        lib().oracle_weights_reconstruct(C.byref(mm), TP, r, int(fused_qkv), int(fused_gate_up), C.byref(lg),
+                                         C.byref(sh))
+    return logical
+
+
+def weights_transform(src_shards, m, a, b, fused_qkv=True, fused_gate_up=True, dst_shards=None):
+    """TP a->b on one layer's weights (reconstruct, then shard); returns the b destination shard dicts."""
+    if dst_shards is None:
+        dst_shards = empty_shards(m, b, fused_qkv, fused_gate_up)
+    src = (_Weights * a)(*[_wstruct(s) for s in src_shards])
+    dst = (_Weights * b)(*[_wstruct(s) for s in dst_shards])
+    mm = _model(m)
+    rc = lib().oracle_weights_transform(C.byref(mm), int(fused_qkv), int(fused_gate_up), a, src, b, dst)
+    assert rc == 0
+    return dst_shards
+
+
+def assign_blocks(seq_lens, T, src_bt, NB_src, NB_dst, free_list=None, free_mask=None, pairs_cap=None, status=0):
+    """Destination block bookkeeping; returns (dst_bt, pairs[N,2], N, free_left, status)."""
+    sl, slp = _i32(seq_lens)
+    sbt, sbtp = _i32(src_bt)
+    S, maxb = sbt.shape
+    assert (free_list is None) != (free_mask is None)
+    if free_list is not None:
+        fl, flp = _i32(free_list)
+        n, fmp = len(fl), None
+    else:
+        fm = np.ascontiguousarray(free_mask, dtype=np.uint8)
+        n, flp, fmp = len(fm), None, fm.ctypes.data_as(C.POINTER(C.c_uint8))
+    if pairs_cap is None:
+        pairs_cap = S * maxb
+    dst_bt = np.empty((S, maxb), dtype=np.int32)
+    pairs = np.full((max(pairs_cap, 1), 2), -7, dtype=np.int32)
+    npairs, nfree, st = C.c_int32(0), C.c_int32(0), C.c_int32(status)
+    lib().oracle_assign_blocks(S, slp, T, sbtp, maxb, NB_src, flp, fmp, n, NB_dst,
+                               dst_bt.ctypes.data_as(C.POINTER(C.c_int32)),
+                               pairs.ctypes.data_as(C.POINTER(C.c_int32)), pairs_cap, C.byref(npairs),
+                               C.byref(nfree), C.byref(st))
+    return dst_bt, pairs[:npairs.value].copy(), npairs.value, nfree.value, st.value

@@ -1,0 +1,313 @@
+/*
+ * CPU oracle for the TP a->b re-layout of an LLM instance's state (Amoeba, runtime TP transformation).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the re-layout computes.
+ * It is used by the tests, by the smoke check and by the benchmark's CPU-baseline leg; the product
+ * library never links, loads or calls it, and it shares no header, helper or table with the CUDA path.
+ *
+ * Everything is an element-by-element loop over the *logical* (unsharded) tensors.  The result of a
+ * TP a->b transformation is a permutation of bytes, so the definition is exact: the expected TP=b state is
+ * "shard the logical state for TP=b", and the logical state is "un-shard the TP=a state".
+ *
+ * Definitions followed (paper section numbers):
+ *   - Head partition of the KV cache (Sec. 3.1, "Base solution"): worker W_i, i = 1..TP, keeps the headers
+ *     (H/TP)(i-1)+1 ... (H/TP)(i-1)+H/TP.  The functions below keep the paper's 1-indexed workers and headers.
+ *     With grouped-query attention (Sec. 2.1 footnote) H is the number of K/V heads.
+ *   - Header-centric KV layout (Sec. 3.1, "Improvement 1"): storage order [Block, Header, K/V, Token]; the
+ *     head dimension is innermost and every layer has its own array of blocks (the paper omits both).
+ *   - FFN partition (Sec. 3.2, Eq. 1): up_proj split column-wise, down_proj split row-wise in the paper's
+ *     [in,out] algebra FFN = f(I x U) x D.  Weights are stored [out,in] row-major here, so the paper's columns
+ *     of U are rows of up/gate (contiguous) and the paper's rows of D are columns of down (strided).
+ *     Attention projections follow the same rule by heads: q/k/v like U, o_proj like D.
+ *   - Destination block bookkeeping (Sec. 3.1: each worker "prepares reserved pages" for incoming KV): the
+ *     paper gives no order; the reading used here is sequences in index order, logical blocks in order, each
+ *     taking the next id of the ordered free list (list order, or ascending id when a mask is given).
+ *
+ * Elements are opaque 16-bit words (fp16 or bf16 makes no difference to movement).
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+    int32_t L;      /* layers */
+    int32_t hidden; /* model width */
+    int32_t Hq;     /* query heads */
+    int32_t Hkv;    /* key/value heads ("headers") */
+    int32_t D;      /* head dim */
+    int32_t I;      /* FFN intermediate width */
+} oracle_model;
+
+enum { ORACLE_OK = 0, ORACLE_INVALID_ARG = 1, ORACLE_NO_FREE_BLOCKS = 4, ORACLE_BAD_BLOCK_ID = 5 };
+
+/* ---- Sec. 3.1: which headers worker W_i keeps (1-indexed, inclusive range) ---- */
+void oracle_header_range(int H, int TP, int i, int* first, int* last) {
+    *first = (H / TP) * (i - 1) + 1;
+    *last = (H / TP) * (i - 1) + H / TP;
+}
+
+/* The worker that keeps a header: search the ranges, no closed form on purpose. */
+int oracle_worker_of_header(int H, int TP, int header) {
+    for (int i = 1; i <= TP; ++i) {
+        int first, last;
+        oracle_header_range(H, TP, i, &first, &last);
+        if (header >= first && header <= last) return i;
+    }
+    return 0;
+}
+
+static int64_t blocks_of(int32_t len, int T) { return ((int64_t)len + T - 1) / T; }
+
+/* Number of padded tokens (whole blocks) before sequence s in the logical KV array. */
+static int64_t token_base(const int32_t* seq_lens, int s, int T) {
+    int64_t g = 0;
+    for (int j = 0; j < s; ++j) g += blocks_of(seq_lens[j], T) * T;
+    return g;
+}
+
+int64_t oracle_padded_tokens(int S, const int32_t* seq_lens, int T) { return token_base(seq_lens, S, T); }
+
+/*
+ * Logical KV: KV[l][g][h][c][d]; g = padded global token (sequence s, token t -> token_base(s) + t, every
+ * sequence rounded up to whole blocks, slack tokens included), h = K/V head 0..Hkv-1, c = 0 (K) / 1 (V).
+ * Pool of worker r (0-indexed pointer array, worker r+1 in the paper's numbering):
+ *   pool[r][l*layer_stride + ((((blk*Hs + hl)*2 + c)*T + tok)*D + d)],  Hs = Hkv/TP headers per worker.
+ * dir = 0: logical -> pools (shard).  dir = 1: pools -> logical (reconstruct).
+ */
+static void kv_walk(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
+                    const int32_t* seq_lens, const int32_t* bt, int maxb, uint16_t* const* pools, int dir) {
+    const int Hs = m->Hkv / TP;
+    const int64_t G = token_base(seq_lens, S, T);
+#pragma omp parallel for schedule(static)
+    for (int l = 0; l < m->L; ++l) {
+        for (int s = 0; s < S; ++s) {
+            const int64_t g0 = token_base(seq_lens, s, T);
+            const int64_t ntok = blocks_of(seq_lens[s], T) * T;
+            for (int64_t t = 0; t < ntok; ++t) {
+                const int64_t blk = bt[(int64_t)s * maxb + t / T];
+                const int tok = (int)(t % T);
+                for (int header = 1; header <= m->Hkv; ++header) {
+                    const int w = oracle_worker_of_header(m->Hkv, TP, header); /* 1-indexed */
+                    int first, last;
+                    oracle_header_range(m->Hkv, TP, w, &first, &last);
+                    const int hl = header - first; /* position among the worker's own headers */
+                    uint16_t* pool = pools[w - 1] + (int64_t)l * layer_stride_elems;
+                    for (int c = 0; c < 2; ++c) {
+                        for (int d = 0; d < m->D; ++d) {
+                            const int64_t lo = ((((int64_t)l * G + g0 + t) * m->Hkv + (header - 1)) * 2 + c) * m->D + d;
+                            const int64_t po = ((((blk * Hs + hl) * 2 + c) * T + tok) * (int64_t)m->D) + d;
+                            if (dir == 0) pool[po] = KV[lo];
+                            else KV[lo] = pool[po];
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+void oracle_kv_shard(const uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
+                     const int32_t* seq_lens, const int32_t* bt, int maxb, uint16_t* const* pools) {
+    kv_walk((uint16_t*)KV, m, T, TP, layer_stride_elems, S, seq_lens, bt, maxb, pools, 0);
+}
+
+void oracle_kv_reconstruct(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
+                           const int32_t* seq_lens, const int32_t* bt, int maxb, const uint16_t* const* pools) {
+    kv_walk(KV, m, T, TP, layer_stride_elems, S, seq_lens, bt, maxb, (uint16_t* const*)pools, 1);
+}
+
+/* TP a -> b on the KV cache: un-shard the TP=a pools into the logical array, shard that for TP=b. */
+int oracle_kv_transform(const oracle_model* m, int T, int S, const int32_t* seq_lens, int maxb, int a,
+                        int64_t src_layer_stride, const int32_t* src_bt, const uint16_t* const* src_pools, int b,
+                        int64_t dst_layer_stride, const int32_t* dst_bt, uint16_t* const* dst_pools) {
+    const int64_t G = token_base(seq_lens, S, T);
+    const int64_t n = (int64_t)m->L * G * m->Hkv * 2 * m->D;
+    uint16_t* KV = (uint16_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(uint16_t));
+    if (!KV) return ORACLE_INVALID_ARG;
+    oracle_kv_reconstruct(KV, m, T, a, src_layer_stride, S, seq_lens, src_bt, maxb, src_pools);
+    oracle_kv_shard(KV, m, T, b, dst_layer_stride, S, seq_lens, dst_bt, maxb, dst_pools);
+    free(KV);
+    return ORACLE_OK;
+}
+
+/*
+ * One layer's logical weights, all [out,in] row-major:
+ *   q [Hq*D, hidden]  k,v [Hkv*D, hidden]  o [hidden, Hq*D]  gate,up [I, hidden]  down [hidden, I]
+ * Worker r (0-indexed here) of TP holds
+ *   q_r  = rows of its Hq/TP query heads        k_r, v_r = rows of its Hkv/TP K/V heads
+ *   gate_r, up_r = rows r*I/TP ...               (the paper's column-wise split of U, Eq. 1)
+ *   o_r  = columns of its query heads of o       down_r = columns r*I/TP ... of down   (row-wise split of D)
+ * each stored dense.  Fused buffers: qkv_r = [q_r; k_r; v_r], gate_up_r = [gate_r; up_r] (row concatenation).
+ * A shard set is 7 pointers {q,k,v,o,gate,up,down}; with fused_qkv the q pointer is the fused buffer and k,v are
+ * ignored, with fused_gate_up the gate pointer is the fused buffer and up is ignored.
+ * dir = 0: logical -> shard.  dir = 1: shard -> logical.
+ */
+typedef struct { uint16_t *q, *k, *v, *o, *gate, *up, *down; } oracle_weights;
+
+static void rows_walk(uint16_t* logical, int64_t rows_total, int64_t cols, int TP, int r, uint16_t* shard, int dir) {
+    const int64_t rows_r = rows_total / TP;
+    for (int64_t i = 0; i < rows_r; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            const int64_t lo = (r * rows_r + i) * cols + j;
+            if (dir == 0) shard[i * cols + j] = logical[lo];
+            else logical[lo] = shard[i * cols + j];
+        }
+}
+
+static void cols_walk(uint16_t* logical, int64_t rows, int64_t cols_total, int TP, int r, uint16_t* shard, int dir) {
+    const int64_t cols_r = cols_total / TP;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols_r; ++j) {
+            const int64_t lo = i * cols_total + r * cols_r + j;
+            if (dir == 0) shard[i * cols_r + j] = logical[lo];
+            else logical[lo] = shard[i * cols_r + j];
+        }
+}
+
+static void weights_walk(const oracle_model* m, int TP, int r, int fused_qkv, int fused_gate_up,
+                         const oracle_weights* lg, const oracle_weights* sh, int dir) {
+    const int64_t hid = m->hidden, qrows = (int64_t)m->Hq * m->D, kvrows = (int64_t)m->Hkv * m->D, I = m->I;
+    uint16_t* q_r = sh->q;
+    uint16_t* k_r = fused_qkv ? q_r + (qrows / TP) * hid : sh->k;
+    uint16_t* v_r = fused_qkv ? k_r + (kvrows / TP) * hid : sh->v;
+    uint16_t* gate_r = sh->gate;
+    uint16_t* up_r = fused_gate_up ? gate_r + (I / TP) * hid : sh->up;
+    rows_walk(lg->q, qrows, hid, TP, r, q_r, dir);
+    rows_walk(lg->k, kvrows, hid, TP, r, k_r, dir);
+    rows_walk(lg->v, kvrows, hid, TP, r, v_r, dir);
+    rows_walk(lg->gate, I, hid, TP, r, gate_r, dir);
+    rows_walk(lg->up, I, hid, TP, r, up_r, dir);
+    cols_walk(lg->o, hid, qrows, TP, r, sh->o, dir);
+    cols_walk(lg->down, hid, I, TP, r, sh->down, dir);
+}
+
+void oracle_weights_shard(const oracle_model* m, int TP, int r, int fused_qkv, int fused_gate_up,
+                          const oracle_weights* logical, const oracle_weights* shard) {
+    weights_walk(m, TP, r, fused_qkv, fused_gate_up, logical, shard, 0);
+}
+
+void oracle_weights_reconstruct(const oracle_model* m, int TP, int r, int fused_qkv, int fused_gate_up,
+                                const oracle_weights* logical, const oracle_weights* shard) {
+    weights_walk(m, TP, r, fused_qkv, fused_gate_up, logical, shard, 1);
+}
+
+/* TP a -> b on one layer's weights: un-shard the a shard sets into logical tensors, shard those b ways. */
+int oracle_weights_transform(const oracle_model* m, int fused_qkv, int fused_gate_up, int a,
+                             const oracle_weights* src /*[a]*/, int b, const oracle_weights* dst /*[b]*/) {
+    const int64_t hid = m->hidden, qrows = (int64_t)m->Hq * m->D, kvrows = (int64_t)m->Hkv * m->D, I = m->I;
+    oracle_weights lg;
+    lg.q = (uint16_t*)malloc((size_t)(qrows * hid) * 2);
+    lg.k = (uint16_t*)malloc((size_t)(kvrows * hid) * 2);
+    lg.v = (uint16_t*)malloc((size_t)(kvrows * hid) * 2);
+    lg.o = (uint16_t*)malloc((size_t)(qrows * hid) * 2);
+    lg.gate = (uint16_t*)malloc((size_t)(I * hid) * 2);
+    lg.up = (uint16_t*)malloc((size_t)(I * hid) * 2);
+    lg.down = (uint16_t*)malloc((size_t)(I * hid) * 2);
+    int rc = ORACLE_OK;
+    if (!lg.q || !lg.k || !lg.v || !lg.o || !lg.gate || !lg.up || !lg.down) rc = ORACLE_INVALID_ARG;
+    if (rc == ORACLE_OK) {
+        for (int r = 0; r < a; ++r) oracle_weights_reconstruct(m, a, r, fused_qkv, fused_gate_up, &lg, &src[r]);
+        for (int r = 0; r < b; ++r) oracle_weights_shard(m, b, r, fused_qkv, fused_gate_up, &lg, &dst[r]);
+    }
+    free(lg.q); free(lg.k); free(lg.v); free(lg.o); free(lg.gate); free(lg.up); free(lg.down);
+    return rc;
+}
+
+/*
+ * Destination block bookkeeping (Sec. 3.1, reserved pages for received KV; order = the reading stated above).
+ *
+ * in : seq_lens[S]; src_bt[S][maxb] (entries past a sequence's blocks are -1); either free_list[n] (ids in the
+ *      order they are to be handed out) or free_mask[n] (n = NB_dst; non-zero = free, handed out in ascending id).
+ * out: dst_bt[S][maxb] (-1 padded), pairs[N][2] = (src block, dst block) for the k-th block in (sequence, logical
+ *      block) order, *num_pairs = N, *free_count_out = free blocks left, *status.
+ *
+ * Whole-call errors (nothing is assigned: dst_bt all -1, N = 0, free count unchanged):
+ *   a negative length or a sequence longer than maxb blocks -> INVALID_ARG; more blocks than pairs_cap ->
+ *   INVALID_ARG; more blocks than free blocks -> NO_FREE_BLOCKS (checked in this order).
+ * Per-block errors -> BAD_BLOCK_ID: a free-list id outside [0, NB_dst) gives dst_bt entry -1 and pair (-1,-1);
+ *   a source id outside [0, NB_src) keeps the dst_bt entry but gives pair (-1,-1), so nothing is copied for it.
+ * status is sticky: it is only written while it still holds 0.
+ */
+void oracle_assign_blocks(int S, const int32_t* seq_lens, int T, const int32_t* src_bt, int maxb, int NB_src,
+                          const int32_t* free_list, const uint8_t* free_mask, int n, int NB_dst, int32_t* dst_bt,
+                          int32_t* pairs, int pairs_cap, int32_t* num_pairs, int32_t* free_count_out,
+                          int32_t* status) {
+    int32_t* ordered = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    int64_t n_free = 0;
+    if (free_list) {
+        for (int i = 0; i < n; ++i) ordered[n_free++] = free_list[i];
+    } else {
+        for (int id = 0; id < n; ++id)
+            if (free_mask[id]) ordered[n_free++] = id;
+    }
+    for (int64_t i = 0; i < (int64_t)S * maxb; ++i) dst_bt[i] = -1;
+    *num_pairs = 0;
+    *free_count_out = (int32_t)n_free;
+
+    int err = ORACLE_OK;
+    int64_t total = 0;
+    for (int s = 0; s < S; ++s) {
+        if (seq_lens[s] < 0 || blocks_of(seq_lens[s], T) > maxb) err = ORACLE_INVALID_ARG;
+        else total += blocks_of(seq_lens[s], T);
+    }
+    if (err == ORACLE_OK && total > pairs_cap) err = ORACLE_INVALID_ARG;
+    if (err == ORACLE_OK && total > n_free) err = ORACLE_NO_FREE_BLOCKS;
+    if (err != ORACLE_OK) {
+        if (*status == 0) *status = err;
+        free(ordered);
+        return;
+    }
+
+    int64_t k = 0;
+    for (int s = 0; s < S; ++s) {
+        for (int64_t i = 0; i < blocks_of(seq_lens[s], T); ++i) {
+            const int32_t src = src_bt[(int64_t)s * maxb + i];
+            const int32_t dst = ordered[k];
+            const int dst_ok = dst >= 0 && dst < NB_dst;
+            const int src_ok = src >= 0 && src < NB_src;
+            dst_bt[(int64_t)s * maxb + i] = dst_ok ? dst : -1;
+            pairs[2 * k + 0] = (dst_ok && src_ok) ? src : -1;
+            pairs[2 * k + 1] = (dst_ok && src_ok) ? dst : -1;
+            if (!(dst_ok && src_ok) && *status == 0) *status = ORACLE_BAD_BLOCK_ID;
+            ++k;
+        }
+    }
+    *num_pairs = (int32_t)k;
+    *free_count_out = (int32_t)(n_free - k);
+    free(ordered);
+}
+
+/*
+ * Copy the blocks named in a pair list, for every layer and every header: the same expected result as
+ * oracle_kv_transform when the pair list comes from oracle_assign_blocks, but usable when a pair is (-1,-1)
+ * (skipped) or a block id is out of range (skipped, BAD_BLOCK_ID).  Element loops through the logical
+ * coordinates (header -> source worker / destination worker), no run copies.
+ */
+void oracle_kv_copy_pairs(const oracle_model* m, int T, int a, int NB_src, int64_t src_layer_stride,
+                          const uint16_t* const* src_pools, int b, int NB_dst, int64_t dst_layer_stride,
+                          uint16_t* const* dst_pools, const int32_t* pairs, int num_pairs, int32_t* status) {
+    const int Ha = m->Hkv / a, Hb = m->Hkv / b;
+    for (int k = 0; k < num_pairs; ++k) {
+        const int64_t p = pairs[2 * k], q = pairs[2 * k + 1];
+        if (p < 0 || q < 0) continue;
+        if (p >= NB_src || q >= NB_dst) {
+            if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+            continue;
+        }
+        for (int l = 0; l < m->L; ++l)
+            for (int header = 1; header <= m->Hkv; ++header) {
+                const int wa = oracle_worker_of_header(m->Hkv, a, header);
+                const int wb = oracle_worker_of_header(m->Hkv, b, header);
+                int fa, fb, last;
+                oracle_header_range(m->Hkv, a, wa, &fa, &last);
+                oracle_header_range(m->Hkv, b, wb, &fb, &last);
+                const uint16_t* sp = src_pools[wa - 1] + (int64_t)l * src_layer_stride;
+                uint16_t* dp = dst_pools[wb - 1] + (int64_t)l * dst_layer_stride;
+                for (int c = 0; c < 2; ++c)
+                    for (int tok = 0; tok < T; ++tok)
+                        for (int d = 0; d < m->D; ++d)
+                            dp[((((q * Hb + (header - fb)) * 2 + c) * T + tok) * (int64_t)m->D) + d] =
+                                sp[((((p * Ha + (header - fa)) * 2 + c) * T + tok) * (int64_t)m->D) + d];
+            }
+    }
+}
