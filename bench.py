@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the TP a->b re-layout hot path on B200.
+
+One step = one whole transformation of one instance: block-table rewrite, KV-cache migration and weight
+re-partition (three C-ABI calls, all kernels of the library).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+N > 1 (under torchrun) runs one independent instance per GPU (the path has no exchange step on one node: every
+worker's shard lives on the same GPU), so scaling is weak and the value is the sum over ranks / max time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "reshard GB/s (read+write)"
+DEFAULT_CONFIG = "llama3_8b_1to4"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM bytes (read + written) per algorithmic byte of kv_reshard, from the ncu capture summarised in
+# profiles/ (None until a capture exists for the default copy path).
+NCU_KV_TRAFFIC_RATIO = None
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.t.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if n_gpus > 0 else "gloo")
+    return rank, world, local
+
+
+def aggregate(world: int, seconds: float, bytes_per_rank: float, device=None):
+    """Whole-job time (max over ranks) and bytes (sum over ranks); identity for one process."""
+    if world == 1:
+        return seconds, bytes_per_rank
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    b = torch.tensor([bytes_per_rank], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(b.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=48, w_layers=2, threads=1):
+    """A bounded sample of the workload for the CPU oracle: the first n_seqs sequences over kv_layers layers of
+    KV, and w_layers layers of weights.  Returns a closure that runs one oracle a->b pass and the bytes it moves."""
+    import oracle
+
+    oracle.build()
+    oracle.set_threads(threads)
+    cfg = wl.CONFIGS[cfg_name]
+    m, a, b, T = dict(cfg["model"]), cfg["a"], cfg["b"], wl.BLOCK_TOKENS
+    lens = wl.draw_seq_lens(cfg, name=cfg_name)[:n_seqs]
+    m_kv = dict(m, L=kv_layers)
+    st = wl.draw_kv_state(cfg, name=cfg_name, seq_lens=lens)
+    G = int(st["blocks_per_seq"].sum()) * T
+    KV = wl.draw_kv_logical(dict(cfg, model=m_kv), G, range(kv_layers))
+    src = oracle.kv_shard(KV, m_kv, T, a, st["NB_src"], lens, st["src_bt"])
+    del KV
+    free = dict(free_list=st.get("dst_free_list"), free_mask=st.get("dst_free_mask"))
+    dst = [np.full(kv_layers * oracle.pool_elems_per_layer(m_kv, T, b, st["NB_dst"]), 0xA5A5, np.uint16)
+           for _ in range(b)]
+    W = [oracle.weights_shard(wl.draw_weights_logical(cfg, l), m, a) for l in range(w_layers)]
+    Wd = [oracle.empty_shards(m, b) for _ in range(w_layers)]
+    e = 2
+    kv_bytes = 2 * st["n_live"] * kv_layers * m["Hkv"] * 2 * T * m["D"] * e
+    w_bytes = 2 * w_layers * e * (2 * m["Hq"] * m["D"] * m["hidden"] + 2 * m["Hkv"] * m["D"] * m["hidden"]
+                                  + 3 * m["hidden"] * m["I"])
+
+    def run():
+        dst_bt, pairs, n, left, status = oracle.assign_blocks(lens, T, st["src_bt"], st["NB_src"], st["NB_dst"], **free)
+        assert status == 0
+        oracle.kv_transform(m_kv, T, lens, a, st["NB_src"], st["src_bt"], src, b, st["NB_dst"], dst_bt, dst)
+        for l in range(w_layers):
+            oracle.weights_transform(W[l], m, a, b, dst_shards=Wd[l])
+
+    desc = (f"{cfg_name}: first {len(lens)} of {cfg['S']} sequences ({st['n_live']} blocks) x {kv_layers} of "
+            f"{m['L']} KV layers + {w_layers} of {m['L']} weight layers")
+    return run, kv_bytes + w_bytes, desc
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle as it stands, timed on the host cores on a bounded sample per step."""
+    if rank != 0:
+        return
+    run, nbytes, desc = oracle_sample(args.config)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = nbytes / dt / 1e9
+    cfg = wl.CONFIGS[args.config]
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']}", "sample": desc},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------ GPU leg
+def build_session(cfg_name: str, device, layers=None, kv=True, weights=True, seed=wl.DEFAULT_SEED, fill=True):
+    import torch
+
+    from paper_2509_19729_b200.session import Session
+
+    cfg = wl.CONFIGS[cfg_name]
+    m = dict(cfg["model"])
+    kv_layers = cfg.get("kv_layers")
+    if layers is not None:  # a slice of the model's layers (all tensors of those layers)
+        m["L"] = layers
+        kv_layers = None if kv_layers is None else min(kv_layers, layers)
+    st = wl.draw_kv_state(cfg, seed=seed, name=cfg_name)
+    s = Session(m, cfg["a"], cfg["b"], st["NB_src"], st["NB_dst"], cfg["S"], st["maxb"], st["n_live"],
+                kv_layers=kv_layers, kv=kv, weights=weights, device=device, dst_fill=None)
+    s.set_tables(st["seq_lens"], st["src_bt"], st.get("dst_free_list"), st.get("dst_free_mask"))
+    if fill:
+        for i, p in enumerate(s.src_pools):
+            wl.hash_fill_(p, seed, 100 + i)
+        for i, p in enumerate(s._wbufs[:cfg["a"]]):
+            n = p.numel() // 8 * 8
+            wl.hash_fill_(p[:n], seed, 200 + i)
+        for p in s.dst_pools + s._wbufs[cfg["a"]:]:
+            p.fill_(0xA5)
+    torch.cuda.synchronize()
+    return s, st
+
+
+def host_free_bytes() -> int:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def run_e2e(args, device, world):
+    """The same metric through the public calls with the state in pinned HOST memory: every step copies the
+    sources host->device, runs the three calls, and copies the destinations device->host."""
+    import torch
+
+    cfg = wl.CONFIGS[args.config]
+    L_full = cfg["model"]["L"]
+    # size the slice so that pinned host buffers stay modest
+    budget = min(int(args.e2e_gib * 2**30), host_free_bytes() // 4)
+    # bytes per layer (sources + destinations) from a one-layer session
+    s1, st = build_session(args.config, device, layers=1, fill=False)
+    per_layer = sum(p.numel() for p in s1.src_pools + s1.dst_pools + s1._wbufs)
+    del s1
+    torch.cuda.empty_cache()
+    layers = int(max(1, min(L_full, budget // max(per_layer, 1))))
+    s, st = build_session(args.config, device, layers=layers)
+    src_dev = s.src_pools + s._wbufs[:cfg["a"]]
+    dst_dev = s.dst_pools + s._wbufs[cfg["a"]:]
+    src_host = [torch.empty(t.numel(), dtype=torch.uint8).pin_memory() for t in src_dev]
+    dst_host = [torch.empty(t.numel(), dtype=torch.uint8).pin_memory() for t in dst_dev]
+    for h, d in zip(src_host, src_dev):
+        h.copy_(d)
+    tabs_host = [torch.from_numpy(st["seq_lens"]).pin_memory(), torch.from_numpy(st["src_bt"]).pin_memory()]
+    dst_bt_host = torch.empty(s.dst_bt.shape, dtype=torch.int32).pin_memory()
+    h2d = sum(t.numel() for t in src_host) + sum(t.numel() * 4 for t in tabs_host)
+    d2h = sum(t.numel() for t in dst_host) + dst_bt_host.numel() * 4
+    stream = torch.cuda.current_stream()
+
+    def step():
+        s.seq_lens.copy_(tabs_host[0], non_blocking=True)
+        s.src_bt.copy_(tabs_host[1], non_blocking=True)
+        for h, d in zip(src_host, src_dev):
+            d.copy_(h, non_blocking=True)
+        s.status.zero_()
+        s.step()
+        for h, d in zip(dst_host, dst_dev):
+            h.copy_(d, non_blocking=True)
+        dst_bt_host.copy_(s.dst_bt, non_blocking=True)
+
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k = max(2, min(args.steps, 5))
+    e0.record(stream)
+    for _ in range(k):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    sec = e0.elapsed_time(e1) / 1e3 / k
+    kvb, wb = s.bytes_rw(st["n_live"])
+    sec, tot = aggregate(world, sec, kvb + wb, device)
+    return {"value": tot / sec / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": sec * 1e3,
+            "sample": f"first {layers} of {L_full} layers (all sequences), state in pinned host memory, "
+                      f"copies and kernels on one stream"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=list(wl.CONFIGS))
+    ap.add_argument("--copy-path", type=int, default=0, help="0 default, 1 vector ld/st, 2 bulk-copy ring")
+    ap.add_argument("--chunk", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-gib", type=float, default=24.0, help="cap on pinned host memory for the e2e leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.layers is None else args.warmup
+
+    rank, world, local = dist_setup(args.gpus if args.impl == "ours" else 0)
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    cfg = wl.CONFIGS[args.config]
+    s, st = build_session(args.config, device, layers=args.layers)
+    for opt, val in ((A.OPT_COPY_PATH, args.copy_path), (A.OPT_CHUNK_BYTES, args.chunk), (A.OPT_STAGES, args.stages),
+                     (A.OPT_CTAS_PER_SM, args.ctas_per_sm)):
+        if val:
+            s.set_option(opt, val)
+    kv_bytes, w_bytes = s.bytes_rw(st["n_live"])
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    for _ in range(args.warmup):
+        s.status.zero_()
+        s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0, f"device status {int(s.status.item())}"
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    marks = []
+    launches0 = A.amoeba_launch_count()
+    t_begin, t_end = ev(), ev()
+    torch.cuda.synchronize()
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        m = [ev() for _ in range(4)]
+        m[0].record(stream)
+        s.rewrite_block_tables()
+        m[1].record(stream)
+        s.reshard_kv()
+        m[2].record(stream)
+        s.reshard_weights()
+        m[3].record(stream)
+        marks.append(m)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    barrier(world)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0, f"device status {int(s.status.item())}"
+    sec = t_begin.elapsed_time(t_end) / 1e3 / args.steps
+    phase = [[m[i].elapsed_time(m[i + 1]) for m in marks] for i in range(3)]
+    bt_ms, kv_ms, w_ms = (statistics.mean(p) for p in phase)
+    sec_all, bytes_all = aggregate(world, sec, kv_bytes + w_bytes, device)
+    n_seq_layers = (s.L, s.kv_layers, int(s.info.chunk_bytes))
+    del s
+    torch.cuda.empty_cache()
+    e2e = None if args.no_e2e else run_e2e(args, device, world)
+    if rank != 0:
+        return
+
+    peak, peak_kind = peaks()
+    kv_gbs = kv_bytes / (kv_ms / 1e3) / 1e9
+    w_gbs = w_bytes / (w_ms / 1e3) / 1e9 if w_bytes else None
+    out = {
+        "metric": METRIC, "value": bytes_all / sec_all / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']}", "layers": n_seq_layers[0], "kv_layers": n_seq_layers[1],
+                   "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
+                   "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2",
+                   "copy_path": {0: "default", 1: "ldst", 2: "bulk"}[args.copy_path],
+                   "chunk_bytes": n_seq_layers[2]},
+        "phases_ms": {"rewrite_block_tables": bt_ms, "reshard_kv": kv_ms, "reshard_weights": w_ms,
+                      "reshard_kv_min": min(phase[1]), "reshard_weights_min": min(phase[2])},
+        "phases_gbs": {"reshard_kv": kv_gbs, "reshard_weights": w_gbs},
+        "pct_of_nominal_8TBs": {"reshard_kv": 100 * kv_gbs / NOMINAL_HBM_GBS,
+                                "reshard_weights": 100 * w_gbs / NOMINAL_HBM_GBS if w_gbs else None},
+        "roofline": {"kernel": "kv_reshard", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": None if NCU_KV_TRAFFIC_RATIO is None else NCU_KV_TRAFFIC_RATIO * kv_bytes},
+        "roofline_weights": None if not w_gbs else {"kernel": "w_reshard", "bound": "hbm", "achieved": w_gbs,
+                                                    "peak": peak, "unit": "GB/s", "frac": w_gbs / peak},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if e2e is not None:
+        out["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        run, nbytes, desc = oracle_sample(args.config)
+        t0 = time.perf_counter()
+        run()
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                               "sample": desc, "seconds": dt}
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,201 @@
+/*
+ * amoeba.h - C ABI of the on-GPU TP a->b re-layout library (sm_100a).
+ *
+ * The library re-lays-out the state of one running LLM instance from a tensor-parallel partition of degree a to
+ * one of degree b without recomputing anything (the transformation the Amoeba paper introduces in its Sec. 1 and
+ * designs in Sec. 3.1 - 3.2).  The state is
+ *   - the paged, head-sharded KV cache in the header-centric layout of Sec. 3.1 ("Improvement 1"):
+ *       pool of worker r:  [layer][block][header of r][K/V][token][head_dim]
+ *     where worker r (0-indexed here; W_{r+1} in the paper) owns the K/V headers r*Hkv/tp ... (r+1)*Hkv/tp - 1
+ *     (Sec. 3.1 "Base solution", 1-indexed there), and
+ *   - the projection weights, stored [out,in] row-major and partitioned as in Sec. 3.2, Eq. 1:
+ *     q/k/v/gate/up by output rows (the paper's column-wise split of U), o_proj/down_proj by input columns (the
+ *     paper's row-wise split of D).
+ * All shards of all workers live on the one GPU; nothing crosses GPUs.
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless its name starts with h_ or the comment says "host array".
+ *     The caller owns every buffer and the stream; the library owns only the plan object.
+ *   - Data calls are asynchronous on the given stream (a cudaStream_t passed as void*; NULL = default stream),
+ *     never synchronise, never allocate, and are out of place: destination buffers must not overlap sources.
+ *   - Errors the host can see return a code and launch nothing.  Errors only the device can see (bad block ids,
+ *     not enough free blocks) are written to *d_status: an int32 the caller zeroes beforehand; the first non-zero
+ *     code sticks, offending items are skipped, the kernel never traps.
+ *   - Only destination blocks named in the pair list, and destination weight bytes covered by the layout, are
+ *     written.  Every other destination byte keeps its value.
+ *   - Block ids are int32; byte offsets are 64-bit.  Pointers, run lengths and pitches must be multiples of 16 B
+ *     (checked: AMOEBA_ERR_ALIGNMENT).
+ *   - Thread-compatible: no global mutable state besides an atomic launch counter; a plan may be used from several threads if its options are not
+ *     changed concurrently.  No C++ exception crosses this boundary.
+ */
+#ifndef AMOEBA_H_
+#define AMOEBA_H_
+
+#include <stdint.h>
+
+#define AMOEBA_API __attribute__((visibility("default")))
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AMOEBA_OK = 0,
+    AMOEBA_ERR_INVALID_ARG = 1,    /* null pointer, negative size, inconsistent layouts, bad sequence length */
+    AMOEBA_ERR_UNSUPPORTED = 2,    /* e.g. head count not divisible by tp, unknown kv_order */
+    AMOEBA_ERR_ALIGNMENT = 3,      /* a pointer, run or pitch is not a multiple of 16 bytes */
+    AMOEBA_ERR_NO_FREE_BLOCKS = 4, /* destination has fewer free blocks than the sequences need */
+    AMOEBA_ERR_BAD_BLOCK_ID = 5,   /* a block id outside its pool (or -1 inside a sequence) */
+    AMOEBA_ERR_CUDA = 6,           /* a CUDA runtime call failed (launch error, no device) */
+    AMOEBA_ERR_TIMEOUT = 7         /* a bounded on-device wait on the kernel's own bulk copy ran out */
+} amoeba_status;
+
+enum { AMOEBA_KV_HEAD_MAJOR = 0 /* [block][header][K/V][token][dim], Sec. 3.1 Improvement 1 */ };
+enum { AMOEBA_MAX_TP = 32 }; /* and at most 22 intersecting (source worker, destination worker) pairs */
+
+/* Transformer shape.  elem_bytes is the size of one weight / KV element (2: fp16 or bf16). */
+typedef struct {
+    int32_t num_layers, hidden, num_q_heads, num_kv_heads, head_dim, intermediate, elem_bytes;
+} amoeba_model;
+
+/* How one instance's state is laid out at one TP degree. */
+typedef struct {
+    amoeba_model model;
+    int32_t tp;            /* number of workers; must divide num_q_heads, num_kv_heads and intermediate */
+    int32_t block_tokens;  /* tokens per KV block */
+    int32_t num_blocks;    /* capacity of every worker's pool, in blocks, per layer */
+    int32_t kv_order;      /* AMOEBA_KV_HEAD_MAJOR */
+    int32_t fused_qkv;     /* 1: worker buffer [q_r; k_r; v_r] (pointer in .q, .k/.v unused); 0: three buffers */
+    int32_t fused_gate_up; /* 1: worker buffer [gate_r; up_r] (pointer in .gate, .up unused); 0: two buffers */
+    int64_t kv_layer_stride_bytes; /* distance between layers inside a worker's pool; 0 = dense */
+} amoeba_layout;
+
+/* One worker's weight buffers for one layer (device pointers; unused slots NULL). */
+typedef struct {
+    void *q, *k, *v, *o, *gate, *up, *down;
+} amoeba_layer_weights;
+
+/* Buffer sizes implied by a layout: one worker's KV pool over all layers, and one worker's buffer of one layer for
+ * `tensor` (0..6 = q,k,v,o,gate,up,down; a fused buffer is asked for by its first member, its other members give 0).
+ * Errors: INVALID_ARG, UNSUPPORTED (same checks as amoeba_plan_create). */
+AMOEBA_API amoeba_status amoeba_layout_kv_pool_bytes(const amoeba_layout* layout, int64_t* bytes);
+AMOEBA_API amoeba_status amoeba_layout_weight_bytes(const amoeba_layout* layout, int32_t tensor, int64_t* bytes);
+
+typedef struct amoeba_plan amoeba_plan; /* opaque, host memory only */
+
+/*
+ * amoeba_plan_create  (the planning step, "amoeba_plan(src_layout, dst_layout)")
+ * Validates the two layouts (same model, same block_tokens; tp divides the head counts and the FFN width) and
+ * derives, from the partition rules of Sec. 3.1 / Eq. 1, which byte ranges of which source worker go to which
+ * destination worker: the K/V header run shared by one source and one destination worker, and one copy descriptor
+ * per intersecting (source worker, destination worker, tensor).  Needs no GPU.  *out is owned by the caller until
+ * amoeba_plan_destroy.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT.
+ */
+AMOEBA_API amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* dst, amoeba_plan** out);
+AMOEBA_API void amoeba_plan_destroy(amoeba_plan* plan);
+
+/* Algorithmic bytes (read + written) of re-laying-out n_blocks live KV blocks over all layers, and of all layers'
+ * weights: what the roofline figures are computed from.  Either output may be NULL. */
+AMOEBA_API amoeba_status amoeba_plan_bytes(const amoeba_plan* plan, int64_t n_blocks, int64_t* kv_bytes_rw, int64_t* w_bytes_rw);
+
+/* What the planner derived, for inspection and host-side tests. */
+typedef struct {
+    int32_t heads_per_run;   /* consecutive K/V headers that share one source and one destination worker */
+    int32_t runs_per_block;  /* num_kv_heads / heads_per_run */
+    int64_t run_bytes;       /* heads_per_run * 2 * block_tokens * head_dim * elem_bytes */
+    int64_t chunk_bytes;     /* size of one copy work item (divides run_bytes) */
+    int64_t src_block_bytes, dst_block_bytes;   /* one block in a source / destination worker's pool */
+    int64_t src_layer_stride, dst_layer_stride; /* bytes between layers in a pool */
+} amoeba_kv_info;
+AMOEBA_API amoeba_status amoeba_plan_kv_info(const amoeba_plan* plan, amoeba_kv_info* out);
+
+/* One weight copy descriptor, relative to the buffers of one layer: n_rows runs of row_bytes each, run i read at
+ * src_off + i*src_pitch of source worker src_rank's buffer `src_tensor` (0..6 = q,k,v,o,gate,up,down; a fused
+ * buffer is named by its first member) and written at dst_off + i*dst_pitch of the destination's. */
+typedef struct {
+    int32_t src_rank, src_tensor, dst_rank, dst_tensor;
+    int64_t src_off, dst_off, row_bytes, src_pitch, dst_pitch;
+    int32_t n_rows, reserved;
+} amoeba_weight_desc;
+AMOEBA_API int32_t amoeba_plan_num_weight_descs(const amoeba_plan* plan);
+AMOEBA_API amoeba_status amoeba_plan_weight_desc(const amoeba_plan* plan, int32_t index, amoeba_weight_desc* out);
+
+/* Tuning knobs (defaults are chosen from measurements; the tests and the benchmark sweep them). */
+enum {
+    AMOEBA_OPT_COPY_PATH = 0,   /* 0 = default, 1 = 16-byte vector loads/stores, 2 = bulk-copy (TMA) ring */
+    AMOEBA_OPT_CTAS_PER_SM = 1, /* persistent grid = this * SM count (0 = default) */
+    AMOEBA_OPT_CHUNK_BYTES = 2, /* upper bound of one copy work item (0 = default) */
+    AMOEBA_OPT_STAGES = 3       /* bulk-copy ring depth per warp (0 = default) */
+};
+AMOEBA_API amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t value);
+
+/*
+ * amoeba_rewrite_block_tables  (destination block bookkeeping: Sec. 3.1, the reserved pages each worker prepares
+ * for the KV it receives; the paper gives no order, the one used is stated below)
+ *
+ * Sequence s needs nblk[s] = ceil(seq_lens[s] / block_tokens) blocks.  Walking sequences in index order and their
+ * blocks in logical order, the k-th block overall gets the k-th id of the ordered destination free list - the list
+ * d_dst_free_list[n_free_or_nb] as given, or, if that is NULL, the ascending ids whose byte in
+ * d_dst_free_mask[n_free_or_nb] is non-zero (the mask covers the whole destination pool).  Exactly one of the two
+ * is non-NULL.
+ *
+ * in  d_src_bt   int32 [num_seqs][max_blocks_per_seq], entries past a sequence's blocks are -1
+ *     d_seq_lens int32 [num_seqs]
+ * out d_dst_bt   int32 [num_seqs][max_blocks_per_seq], fully written, -1 past each sequence's blocks
+ *     d_pairs    int32 [pairs_cap][2]: entry k = (source block, destination block) of the k-th block
+ *     d_num_pairs, d_dst_free_count_out  int32 scalars: number of pairs, free blocks left
+ *     d_status   int32 scalar, sticky (see conventions)
+ * d_workspace: scratch of at least amoeba_rewrite_workspace_bytes(...) bytes, 16-byte aligned, contents irrelevant
+ *     before and after; calls that overlap on the GPU need separate workspaces.
+ *
+ * Device-detected errors.  Whole call (d_dst_bt all -1, 0 pairs, free count unchanged): a negative length or a
+ * sequence needing more than max_blocks_per_seq blocks, or more blocks than pairs_cap -> INVALID_ARG; more blocks
+ * than free blocks -> NO_FREE_BLOCKS.  Per block -> BAD_BLOCK_ID: a free id outside [0, dst num_blocks) gives table
+ * entry -1 and pair (-1,-1); a source id outside [0, src num_blocks) keeps the table entry, pair (-1,-1).
+ * Host-detected: INVALID_ARG (null pointers, negative sizes, both or neither free form), ALIGNMENT, CUDA.
+ */
+AMOEBA_API amoeba_status amoeba_rewrite_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs, int32_t n_free_or_nb,
+                                             int64_t* bytes);
+AMOEBA_API amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt, const int32_t* d_seq_lens,
+                                          int32_t num_seqs, int32_t max_blocks_per_seq,
+                                          const int32_t* d_dst_free_list, const uint8_t* d_dst_free_mask,
+                                          int32_t n_free_or_nb, int32_t* d_dst_bt, int32_t* d_pairs,
+                                          int32_t pairs_cap, int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
+                                          int32_t* d_status, void* d_workspace, int64_t workspace_bytes,
+                                          void* cuda_stream);
+
+/*
+ * amoeba_reshard_kv  (KV cache migration in the head dimension, Sec. 3.1: every header of every live block moves
+ * from the source worker that holds it to the destination worker that keeps it; here as an on-GPU gather/scatter)
+ *
+ * For every pair k < min(*d_num_pairs, pairs_cap) with both ids >= 0, every layer in [layer_begin, layer_end) and
+ * every K/V header h: the 2*block_tokens*head_dim elements of (block, header) are copied from
+ * src_pools[h / (Hkv/a)] to dst_pools[h / (Hkv/b)] at the pool addresses of the header-centric layout.
+ * src_pools / dst_pools are HOST arrays of a / b device pointers (read during the call only).
+ * A pair with an id outside its pool is skipped and sets BAD_BLOCK_ID in *d_status.
+ */
+AMOEBA_API amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools, void* const* dst_pools,
+                                const int32_t* d_pairs, const int32_t* d_num_pairs, int32_t pairs_cap,
+                                int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
+
+/*
+ * amoeba_reshard_weights  (model weight transformation, Sec. 3.2: the copy that re-partitions the weights; Eq. 1
+ * fixes which rows / columns each worker holds)
+ *
+ * src is a HOST array [a][num_layers] (worker-major) of device pointers, dst likewise [b][num_layers]; only layers
+ * in [layer_begin, layer_end) are read.  A caller transforming a few layers per inference step (Sec. 3.3's
+ * layer-by-layer order) passes successive ranges.
+ */
+AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const amoeba_layer_weights* src,
+                                     const amoeba_layer_weights* dst, int32_t layer_begin, int32_t layer_end,
+                                     int32_t* d_status, void* cuda_stream);
+
+/* Number of kernels the library has launched in this process (for launch accounting in benchmarks). */
+AMOEBA_API int64_t amoeba_launch_count(void);
+
+AMOEBA_API const char* amoeba_status_string(amoeba_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMOEBA_H_ */

@@ -1,0 +1,257 @@
+"""ctypes binding of ``libamoeba.so``: argument marshalling only, every step runs in the CUDA kernels.
+
+Device buffers are ``torch`` CUDA tensors (or raw integer device addresses); the stream defaults to torch's
+current stream.  Every function raises :class:`AmoebaError` when the C call returns a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Optional, Sequence
+
+from . import build as _build
+
+__all__ = [
+    "AmoebaError", "Model", "Layout", "LayerWeights", "KvInfo", "WeightDesc", "Plan", "STATUS_NAMES", "TENSOR_NAMES",
+    "OPT_COPY_PATH", "OPT_CTAS_PER_SM", "OPT_CHUNK_BYTES", "OPT_STAGES", "COPY_PATH_LDST", "COPY_PATH_BULK",
+    "amoeba_plan_create", "amoeba_plan_destroy", "amoeba_layout_kv_pool_bytes", "amoeba_layout_weight_bytes", "amoeba_plan_bytes", "amoeba_plan_kv_info",
+    "amoeba_plan_num_weight_descs", "amoeba_plan_weight_desc", "amoeba_plan_set_option",
+    "amoeba_rewrite_workspace_bytes", "amoeba_rewrite_block_tables", "amoeba_reshard_kv", "amoeba_reshard_weights",
+    "amoeba_launch_count", "amoeba_status_string", "library_path", "make_layout",
+]
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NO_FREE_BLOCKS, ERR_BAD_BLOCK_ID, ERR_CUDA, ERR_TIMEOUT = range(8)
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS", "BAD_BLOCK_ID", "CUDA", "TIMEOUT"]
+__all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
+            "ERR_CUDA", "ERR_TIMEOUT"]
+OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES = range(4)
+COPY_PATH_LDST, COPY_PATH_BULK = 1, 2
+TENSOR_NAMES = ("q", "k", "v", "o", "gate", "up", "down")
+
+
+class AmoebaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {amoeba_status_string(status)} (status {status})")
+
+
+class Model(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("num_layers", "hidden", "num_q_heads", "num_kv_heads", "head_dim", "intermediate", "elem_bytes")]
+
+
+class Layout(C.Structure):
+    _fields_ = [("model", Model), ("tp", C.c_int32), ("block_tokens", C.c_int32), ("num_blocks", C.c_int32),
+                ("kv_order", C.c_int32), ("fused_qkv", C.c_int32), ("fused_gate_up", C.c_int32),
+                ("kv_layer_stride_bytes", C.c_int64)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in TENSOR_NAMES]
+
+
+class KvInfo(C.Structure):
+    _fields_ = [("heads_per_run", C.c_int32), ("runs_per_block", C.c_int32), ("run_bytes", C.c_int64),
+                ("chunk_bytes", C.c_int64), ("src_block_bytes", C.c_int64), ("dst_block_bytes", C.c_int64),
+                ("src_layer_stride", C.c_int64), ("dst_layer_stride", C.c_int64)]
+
+
+class WeightDesc(C.Structure):
+    _fields_ = [("src_rank", C.c_int32), ("src_tensor", C.c_int32), ("dst_rank", C.c_int32), ("dst_tensor", C.c_int32),
+                ("src_off", C.c_int64), ("dst_off", C.c_int64), ("row_bytes", C.c_int64), ("src_pitch", C.c_int64),
+                ("dst_pitch", C.c_int64), ("n_rows", C.c_int32), ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def library_path():
+    return _build.LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if _build.needs_build():
+        try:
+            _build.build()
+        except Exception as e:  # no silent fallback: the product is the CUDA library
+            raise ImportError(f"libamoeba.so is missing or stale and could not be built: {e}") from e
+    lib = C.CDLL(str(_build.LIB))
+    P, I32, I64, VP = C.POINTER, C.c_int32, C.c_int64, C.c_void_p
+    sig = {
+        "amoeba_plan_create": (I32, [P(Layout), P(Layout), P(VP)]),
+        "amoeba_plan_destroy": (None, [VP]),
+        "amoeba_layout_kv_pool_bytes": (I32, [P(Layout), P(I64)]),
+        "amoeba_layout_weight_bytes": (I32, [P(Layout), I32, P(I64)]),
+        "amoeba_plan_bytes": (I32, [VP, I64, P(I64), P(I64)]),
+        "amoeba_plan_kv_info": (I32, [VP, P(KvInfo)]),
+        "amoeba_plan_num_weight_descs": (I32, [VP]),
+        "amoeba_plan_weight_desc": (I32, [VP, I32, P(WeightDesc)]),
+        "amoeba_plan_set_option": (I32, [VP, I32, I64]),
+        "amoeba_rewrite_workspace_bytes": (I32, [VP, I32, I32, P(I64)]),
+        "amoeba_rewrite_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP, I64, VP]),
+        "amoeba_reshard_kv": (I32, [VP, P(VP), P(VP), VP, VP, I32, I32, I32, VP, VP]),
+        "amoeba_reshard_weights": (I32, [VP, P(LayerWeights), P(LayerWeights), I32, I32, VP, VP]),
+        "amoeba_launch_count": (I64, []),
+        "amoeba_status_string": (C.c_char_p, [I32]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(lib, name)
+        f.restype, f.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def _ptr(x) -> Optional[int]:
+    """Device address of a torch tensor, an int address, or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise AmoebaError(status, where)
+
+
+class Plan:
+    """Owner of an ``amoeba_plan*``."""
+
+    def __init__(self, handle: int, src: Layout, dst: Layout):
+        self.handle, self.src, self.dst = handle, src, dst
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _load().amoeba_plan_destroy(self.handle)
+            self.handle = None
+
+
+def make_layout(model: dict, tp: int, num_blocks: int, block_tokens: int = 16, fused_qkv: bool = True,
+                fused_gate_up: bool = True, elem_bytes: int = 2, kv_layer_stride_bytes: int = 0) -> Layout:
+    """Layout from a shape dict with keys L, hidden, Hq, Hkv, D, I."""
+    m = Model(model["L"], model["hidden"], model["Hq"], model["Hkv"], model["D"], model["I"], elem_bytes)
+    return Layout(m, tp, block_tokens, num_blocks, 0, int(fused_qkv), int(fused_gate_up), kv_layer_stride_bytes)
+
+
+def amoeba_status_string(status: int) -> str:
+    return _load().amoeba_status_string(int(status)).decode()
+
+
+def amoeba_plan_create(src: Layout, dst: Layout) -> Plan:
+    h = C.c_void_p()
+    _check(_load().amoeba_plan_create(C.byref(src), C.byref(dst), C.byref(h)), "amoeba_plan_create")
+    return Plan(h.value, src, dst)
+
+
+def amoeba_layout_kv_pool_bytes(layout: Layout) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_layout_kv_pool_bytes(C.byref(layout), C.byref(out)), "amoeba_layout_kv_pool_bytes")
+    return out.value
+
+
+def amoeba_layout_weight_bytes(layout: Layout, tensor: int) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_layout_weight_bytes(C.byref(layout), tensor, C.byref(out)), "amoeba_layout_weight_bytes")
+    return out.value
+
+
+def amoeba_plan_destroy(plan: Plan) -> None:
+    plan.__del__()
+
+
+def amoeba_plan_bytes(plan: Plan, n_blocks: int):
+    kv, w = C.c_int64(), C.c_int64()
+    _check(_load().amoeba_plan_bytes(plan.handle, n_blocks, C.byref(kv), C.byref(w)), "amoeba_plan_bytes")
+    return kv.value, w.value
+
+
+def amoeba_plan_kv_info(plan: Plan) -> KvInfo:
+    out = KvInfo()
+    _check(_load().amoeba_plan_kv_info(plan.handle, C.byref(out)), "amoeba_plan_kv_info")
+    return out
+
+
+def amoeba_plan_num_weight_descs(plan: Plan) -> int:
+    return _load().amoeba_plan_num_weight_descs(plan.handle)
+
+
+def amoeba_plan_weight_desc(plan: Plan, index: int) -> WeightDesc:
+    out = WeightDesc()
+    _check(_load().amoeba_plan_weight_desc(plan.handle, index, C.byref(out)), "amoeba_plan_weight_desc")
+    return out
+
+
+def amoeba_plan_set_option(plan: Plan, option: int, value: int) -> None:
+    _check(_load().amoeba_plan_set_option(plan.handle, option, value), "amoeba_plan_set_option")
+
+
+def amoeba_rewrite_workspace_bytes(plan: Plan, num_seqs: int, n_free_or_nb: int) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_rewrite_workspace_bytes(plan.handle, num_seqs, n_free_or_nb, C.byref(out)),
+           "amoeba_rewrite_workspace_bytes")
+    return out.value
+
+
+def amoeba_rewrite_block_tables(plan: Plan, src_bt, seq_lens, num_seqs: int, max_blocks_per_seq: int, dst_free_list,
+                                dst_free_mask, n_free_or_nb: int, dst_bt, pairs, pairs_cap: int, num_pairs,
+                                dst_free_count_out, status, workspace, workspace_bytes: int, stream=None) -> None:
+    _check(_load().amoeba_rewrite_block_tables(
+        plan.handle, _ptr(src_bt), _ptr(seq_lens), num_seqs, max_blocks_per_seq, _ptr(dst_free_list),
+        _ptr(dst_free_mask), n_free_or_nb, _ptr(dst_bt), _ptr(pairs), pairs_cap, _ptr(num_pairs),
+        _ptr(dst_free_count_out), _ptr(status), _ptr(workspace), workspace_bytes, _stream(stream)),
+        "amoeba_rewrite_block_tables")
+
+
+def amoeba_reshard_kv(plan: Plan, src_pools: Sequence, dst_pools: Sequence, pairs, num_pairs, pairs_cap: int,
+                      layer_begin: int, layer_end: int, status, stream=None) -> None:
+    sp = (C.c_void_p * len(src_pools))(*[_ptr(x) for x in src_pools])
+    dp = (C.c_void_p * len(dst_pools))(*[_ptr(x) for x in dst_pools])
+    if len(src_pools) != plan.src.tp or len(dst_pools) != plan.dst.tp:
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_reshard_kv (pool count != tp)")
+    _check(_load().amoeba_reshard_kv(plan.handle, sp, dp, _ptr(pairs), _ptr(num_pairs), pairs_cap, layer_begin,
+                                     layer_end, _ptr(status), _stream(stream)), "amoeba_reshard_kv")
+
+
+def pack_weights(shards: Sequence[Sequence[dict]]):
+    """[rank][layer] dicts {tensor name: tensor or address} -> C array of LayerWeights, rank-major."""
+    n_rank, n_layer = len(shards), len(shards[0])
+    arr = (LayerWeights * (n_rank * n_layer))()
+    for r in range(n_rank):
+        for l in range(n_layer):
+            for name in TENSOR_NAMES:
+                setattr(arr[r * n_layer + l], name, _ptr(shards[r][l].get(name)))
+    return arr
+
+
+__all__.append("pack_weights")
+
+
+def amoeba_reshard_weights(plan: Plan, src, dst, layer_begin: int, layer_end: int, status, stream=None) -> None:
+    """``src`` / ``dst``: ``pack_weights`` arrays or [rank][layer] lists of dicts."""
+    if not isinstance(src, C.Array):
+        src = pack_weights(src)
+    if not isinstance(dst, C.Array):
+        dst = pack_weights(dst)
+    L = plan.src.model.num_layers
+    if len(src) != plan.src.tp * L or len(dst) != plan.dst.tp * L:
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_reshard_weights (need [tp][num_layers] entries)")
+    _check(_load().amoeba_reshard_weights(plan.handle, src, dst, layer_begin, layer_end, _ptr(status),
+                                          _stream(stream)), "amoeba_reshard_weights")
+
+
+def amoeba_launch_count() -> int:
+    return _load().amoeba_launch_count()
+
+
+_load()

@@ -1,0 +1,211 @@
+// Destination block bookkeeping for the KV migration (Sec. 3.1: each worker prepares reserved pages for the KV it
+// receives).  Two launches, no CTA ever waits on another:
+//   bt_scan   (1 CTA)   blocks per sequence, exclusive prefix sum over the sequences, and - when the free blocks
+//                       come as a byte mask - their compaction into an ascending id list (ballot + popc prefix
+//                       sums, one warp-wide ballot per 32 mask bytes); decides the whole-call errors.
+//   bt_assign (grid)    one warp per 128-entry segment of a block-table row: k-th block overall takes the k-th free
+//                       id; writes the destination table (with -1 padding) and the (source, destination) pair list.
+#include <cuda_runtime.h>
+
+#include "launch.hpp"
+#include "plan.hpp"
+
+namespace amoeba {
+
+struct BtHeader {  // first 64 bytes of the workspace
+    int32_t total;   // blocks assigned by this call (0 on a whole-call error)
+    int32_t n_free;  // free destination blocks before the call
+    int32_t err;     // whole-call error code or 0
+    int32_t pad[13];
+};
+
+constexpr int kScanThreads = 1024;
+
+// Exclusive scan of one value per thread across the CTA; returns the thread's offset, *total = CTA sum.
+__device__ __forceinline__ int32_t cta_exclusive_scan(int32_t v, int32_t* warp_sums, int32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int32_t incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int32_t t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int32_t w = warp_sums[lane];  // kScanThreads / 32 == 32 warps
+        int32_t wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t t = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += t;
+        }
+        warp_sums[lane] = wi - w;                // exclusive warp offsets
+        if (lane == 31) warp_sums[32] = wi;      // CTA total
+    }
+    __syncthreads();
+    const int32_t off = warp_sums[warp] + incl - v;
+    *total = warp_sums[32];
+    __syncthreads();  // warp_sums may be reused by the caller's next round
+    return off;
+}
+
+__global__ void __launch_bounds__(kScanThreads) bt_scan(const int32_t* __restrict__ seq_lens, int32_t num_seqs,
+                                                        int32_t block_tokens, int32_t max_blocks_per_seq,
+                                                        const uint8_t* __restrict__ free_mask, int32_t n_free_or_nb,
+                                                        int32_t pairs_cap, BtHeader* hdr, int32_t* __restrict__ seq_off,
+                                                        int32_t* __restrict__ free_ids, int32_t* num_pairs,
+                                                        int32_t* free_count_out, int32_t* status) {
+    __shared__ int32_t warp_sums[33];
+    __shared__ int32_t bad_len;
+    if (threadIdx.x == 0) bad_len = 0;
+    __syncthreads();
+
+    // ---- blocks per sequence and their exclusive prefix sum
+    int64_t carry = 0;
+    for (int32_t base = 0; base < num_seqs; base += kScanThreads) {
+        const int32_t s = base + threadIdx.x;
+        int32_t nb = 0;
+        if (s < num_seqs) {
+            const int32_t len = seq_lens[s];
+            const int64_t need = ((int64_t)len + block_tokens - 1) / block_tokens;
+            if (len < 0 || need > max_blocks_per_seq) bad_len = 1;
+            else nb = (int32_t)need;
+        }
+        int32_t tile_total;
+        const int32_t off = cta_exclusive_scan(nb, warp_sums, &tile_total);
+        if (s < num_seqs) seq_off[s] = (int32_t)min(carry + off, (int64_t)INT32_MAX);
+        carry += tile_total;
+    }
+    const int64_t total = carry;
+
+    // ---- ordered free list from the mask: ascending ids of the non-zero bytes
+    int64_t n_free = n_free_or_nb;
+    if (free_mask) {
+        const int lane = threadIdx.x & 31;
+        int32_t found = 0;
+        for (int32_t base = 0; base < n_free_or_nb; base += kScanThreads) {
+            const int32_t id = base + threadIdx.x;
+            const bool is_free = id < n_free_or_nb && free_mask[id] != 0;
+            const uint32_t ballot = __ballot_sync(0xffffffffu, is_free);
+            int32_t tile_total;
+            const int32_t warp_off = cta_exclusive_scan(lane == 0 ? __popc(ballot) : 0, warp_sums, &tile_total);
+            const int32_t my_warp_off = __shfl_sync(0xffffffffu, warp_off, 0);
+            if (is_free) free_ids[found + my_warp_off + __popc(ballot & ((1u << lane) - 1u))] = id;
+            found += tile_total;
+        }
+        n_free = found;
+    }
+
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int32_t err = 0;
+        if (bad_len) err = AMOEBA_ERR_INVALID_ARG;
+        else if (total > pairs_cap) err = AMOEBA_ERR_INVALID_ARG;
+        else if (total > n_free) err = AMOEBA_ERR_NO_FREE_BLOCKS;
+        const int32_t assigned = err ? 0 : (int32_t)total;
+        hdr->total = assigned;
+        hdr->n_free = (int32_t)n_free;
+        hdr->err = err;
+        *num_pairs = assigned;
+        *free_count_out = (int32_t)n_free - assigned;
+        if (err) atomicCAS(status, 0, err);
+    }
+}
+
+constexpr int kSegment = 128;  // table entries one warp handles per step
+
+__global__ void __launch_bounds__(256) bt_assign(const int32_t* __restrict__ src_bt,
+                                                 const int32_t* __restrict__ seq_lens, int32_t num_seqs,
+                                                 int32_t block_tokens, int32_t max_blocks_per_seq,
+                                                 const int32_t* __restrict__ free_ids, const BtHeader* hdr,
+                                                 const int32_t* __restrict__ seq_off, int32_t nb_src, int32_t nb_dst,
+                                                 int32_t* __restrict__ dst_bt, int2* __restrict__ pairs,
+                                                 int32_t* status) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int32_t segs_per_row = (max_blocks_per_seq + kSegment - 1) / kSegment;
+    const bool call_failed = hdr->err != 0;
+    bool bad = false;
+    for (int64_t unit = warp; unit < (int64_t)num_seqs * segs_per_row; unit += n_warps) {
+        const int32_t s = (int32_t)(unit / segs_per_row);
+        const int32_t col0 = (int32_t)(unit - (int64_t)s * segs_per_row) * kSegment;
+        const int32_t nb = call_failed ? 0 : (int32_t)(((int64_t)seq_lens[s] + block_tokens - 1) / block_tokens);
+        const int32_t off = seq_off[s];
+        for (int32_t i = col0 + lane; i < min(col0 + kSegment, max_blocks_per_seq); i += 32) {
+            int32_t out = -1;
+            if (i < nb) {
+                const int32_t k = off + i;
+                const int32_t dst = free_ids[k];
+                const int32_t src = src_bt[(int64_t)s * max_blocks_per_seq + i];
+                const bool dst_ok = dst >= 0 && dst < nb_dst, src_ok = src >= 0 && src < nb_src;
+                out = dst_ok ? dst : -1;
+                pairs[k] = (dst_ok && src_ok) ? make_int2(src, dst) : make_int2(-1, -1);
+                bad |= !(dst_ok && src_ok);
+            }
+            dst_bt[(int64_t)s * max_blocks_per_seq + i] = out;
+        }
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+}
+
+static int64_t align16(int64_t x) { return (x + 15) & ~int64_t(15); }
+
+}  // namespace amoeba
+
+using namespace amoeba;
+
+extern "C" amoeba_status amoeba_rewrite_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs,
+                                                        int32_t n_free_or_nb, int64_t* bytes) {
+    if (!plan || !bytes || num_seqs < 0 || n_free_or_nb < 0) return AMOEBA_ERR_INVALID_ARG;
+    *bytes = (int64_t)sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)) + align16(4 * (int64_t)n_free_or_nb);
+    return AMOEBA_OK;
+}
+
+extern "C" amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
+                                                     const int32_t* d_seq_lens, int32_t num_seqs,
+                                                     int32_t max_blocks_per_seq, const int32_t* d_dst_free_list,
+                                                     const uint8_t* d_dst_free_mask, int32_t n_free_or_nb,
+                                                     int32_t* d_dst_bt, int32_t* d_pairs, int32_t pairs_cap,
+                                                     int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
+                                                     int32_t* d_status, void* d_workspace, int64_t workspace_bytes,
+                                                     void* cuda_stream) {
+    if (!plan || num_seqs < 0 || max_blocks_per_seq <= 0 || n_free_or_nb < 0 || pairs_cap < 0)
+        return AMOEBA_ERR_INVALID_ARG;
+    if ((d_dst_free_list != nullptr) == (d_dst_free_mask != nullptr)) return AMOEBA_ERR_INVALID_ARG;
+    if (!d_num_pairs || !d_dst_free_count_out || !d_status || !d_workspace) return AMOEBA_ERR_INVALID_ARG;
+    if (num_seqs > 0 && (!d_src_bt || !d_seq_lens || !d_dst_bt)) return AMOEBA_ERR_INVALID_ARG;
+    if (pairs_cap > 0 && !d_pairs) return AMOEBA_ERR_INVALID_ARG;
+    if (d_dst_free_mask && n_free_or_nb != plan->dst.num_blocks) return AMOEBA_ERR_INVALID_ARG;
+    int64_t need = 0;
+    amoeba_rewrite_workspace_bytes(plan, num_seqs, n_free_or_nb, &need);
+    if (workspace_bytes < need) return AMOEBA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_workspace) % 16 || reinterpret_cast<uintptr_t>(d_pairs) % 8)
+        return AMOEBA_ERR_ALIGNMENT;
+
+    char* ws = static_cast<char*>(d_workspace);
+    BtHeader* hdr = reinterpret_cast<BtHeader*>(ws);
+    int32_t* seq_off = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader));
+    int32_t* compact = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)));
+    const int32_t* free_ids = d_dst_free_mask ? compact : d_dst_free_list;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    bt_scan<<<1, kScanThreads, 0, stream>>>(d_seq_lens, num_seqs, plan->src.block_tokens, max_blocks_per_seq,
+                                            d_dst_free_mask, n_free_or_nb, pairs_cap, hdr, seq_off, compact,
+                                            d_num_pairs, d_dst_free_count_out, d_status);
+    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    if (num_seqs == 0) return AMOEBA_OK;
+
+    DeviceInfo dev;
+    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    const int64_t units = (int64_t)num_seqs * ((max_blocks_per_seq + kSegment - 1) / kSegment);
+    const int grid = (int)std::min<int64_t>((units + 7) / 8, (int64_t)dev.sms * 8);
+    bt_assign<<<grid, 256, 0, stream>>>(d_src_bt, d_seq_lens, num_seqs, plan->src.block_tokens, max_blocks_per_seq,
+                                        free_ids, hdr, seq_off, plan->src.num_blocks, plan->dst.num_blocks, d_dst_bt,
+                                        reinterpret_cast<int2*>(d_pairs), d_status);
+    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    return AMOEBA_OK;
+}

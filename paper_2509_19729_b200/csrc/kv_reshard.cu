@@ -1,0 +1,176 @@
+// KV cache migration in the head dimension (Sec. 3.1) as an on-GPU gather/scatter between the pools of the
+// source workers (TP = a) and of the destination workers (TP = b), header-centric layout
+// [layer][block][header][K/V][token][dim] on both sides.
+//
+// Work decomposition: (layer, pair, run, chunk).  A run is heads_per_run = gcd(Hkv/a, Hkv/b) consecutive headers
+// of one block: contiguous in exactly one source pool and one destination pool.  Runs are cut into equal chunks
+// (the copy work items), dealt round-robin to a persistent grid; layer is the slowest index so that concurrently
+// running CTAs touch neighbouring DRAM pages.
+#include <cuda_runtime.h>
+
+#include "copy_engine.cuh"
+#include "launch.hpp"
+#include "plan.hpp"
+
+namespace amoeba {
+
+struct KvParams {
+    const char* src[AMOEBA_MAX_TP];
+    char* dst[AMOEBA_MAX_TP];
+    const int32_t* pairs;      // [cap][2]
+    const int32_t* num_pairs;  // device scalar
+    int32_t* status;
+    int64_t unit_bytes, chunk_bytes, src_layer_stride, dst_layer_stride;
+    int32_t pairs_cap, layer_begin, n_layers;
+    int32_t nb_src, nb_dst;
+    int32_t heads_src, heads_dst, heads_per_run, runs_per_block, chunks_per_run;
+};
+
+struct KvItems {
+    const KvParams& p;
+    int32_t n_pairs;
+    __device__ __forceinline__ int64_t count() const {
+        return (int64_t)n_pairs * p.n_layers * p.runs_per_block * p.chunks_per_run;
+    }
+    // n_rows == 0 marks a skipped pair.
+    __device__ __forceinline__ Item operator()(int64_t w) const {
+        const int32_t chunk = (int32_t)(w % p.chunks_per_run);
+        int64_t t = w / p.chunks_per_run;
+        const int32_t run = (int32_t)(t % p.runs_per_block);
+        t /= p.runs_per_block;
+        const int32_t pair = (int32_t)(t % n_pairs);
+        const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
+        const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
+        Item it;
+        it.n_rows = 1;
+        it.row_bytes = (int32_t)p.chunk_bytes;
+        it.src_pitch = it.dst_pitch = 0;
+        if (ids.x < 0 || ids.y < 0) {  // the table rewrite already reported this one
+            it.n_rows = 0;
+            it.src = nullptr;
+            it.dst = nullptr;
+            return it;
+        }
+        if (ids.x >= p.nb_src || ids.y >= p.nb_dst) {
+            if (run == 0 && chunk == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+            it.n_rows = 0;
+            it.src = nullptr;
+            it.dst = nullptr;
+            return it;
+        }
+        const int32_t h0 = run * p.heads_per_run;  // first header of the run
+        const int32_t ra = h0 / p.heads_src, ha = h0 - ra * p.heads_src;
+        const int32_t rb = h0 / p.heads_dst, hb = h0 - rb * p.heads_dst;
+        const int64_t in_run = (int64_t)chunk * p.chunk_bytes;
+        it.src = p.src[ra] + layer * p.src_layer_stride + ((int64_t)ids.x * p.heads_src + ha) * p.unit_bytes + in_run;
+        it.dst = p.dst[rb] + layer * p.dst_layer_stride + ((int64_t)ids.y * p.heads_dst + hb) * p.unit_bytes + in_run;
+        return it;
+    }
+};
+
+__device__ __forceinline__ int32_t clamp_pairs(const KvParams& p) {
+    const int32_t n = *p.num_pairs;
+    return n < 0 ? 0 : (n > p.pairs_cap ? p.pairs_cap : n);
+}
+
+template <int UNROLL>
+__global__ void __launch_bounds__(256) kv_reshard_ldst(const __grid_constant__ KvParams p) {
+    const KvItems items{p, clamp_pairs(p)};
+    const int64_t n = items.count();
+    for (int64_t w = blockIdx.x; w < n; w += gridDim.x) {
+        const Item it = items(w);
+        if (it.n_rows) cta_copy_item<UNROLL>(it);
+    }
+}
+
+template <int NS, int LAG>
+__global__ void __launch_bounds__(1024) kv_reshard_bulk(const __grid_constant__ KvParams p, int stage_bytes) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * NS;
+    char* stages = smem + 1024 + (int64_t)warp * NS * stage_bytes;
+    const KvItems items{p, clamp_pairs(p)};
+    const bool ok = warp_bulk_ring<NS, LAG>(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
+                                            (int64_t)gridDim.x * nwarps, stages, stage_bytes, bars);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
+}
+
+template <int NS, int LAG>
+static cudaError_t launch_bulk(const KvParams& p, int grid, int warps, int stage_bytes, cudaStream_t stream) {
+    const size_t smem = 1024 + (size_t)warps * NS * stage_bytes;
+    cudaError_t e = cudaFuncSetAttribute(kv_reshard_bulk<NS, LAG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    kv_reshard_bulk<NS, LAG><<<grid, warps * 32, smem, stream>>>(p, stage_bytes);
+    return cudaGetLastError();
+}
+
+}  // namespace amoeba
+
+using namespace amoeba;
+
+extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools,
+                                           void* const* dst_pools, const int32_t* d_pairs, const int32_t* d_num_pairs,
+                                           int32_t pairs_cap, int32_t layer_begin, int32_t layer_end, int32_t* d_status,
+                                           void* cuda_stream) {
+    if (!plan || !src_pools || !dst_pools || !d_pairs || !d_num_pairs || !d_status || pairs_cap < 0)
+        return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_model& m = plan->src.model;
+    if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_pairs) % 8) return AMOEBA_ERR_ALIGNMENT;
+    KvParams p{};
+    for (int r = 0; r < plan->src.tp; ++r) {
+        if (!src_pools[r]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(src_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        p.src[r] = static_cast<const char*>(src_pools[r]);
+    }
+    for (int r = 0; r < plan->dst.tp; ++r) {
+        if (!dst_pools[r]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(dst_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        p.dst[r] = static_cast<char*>(dst_pools[r]);
+    }
+    if (pairs_cap == 0 || layer_begin == layer_end) return AMOEBA_OK;
+    p.pairs = d_pairs;
+    p.num_pairs = d_num_pairs;
+    p.status = d_status;
+    p.unit_bytes = plan->unit_bytes;
+    p.chunk_bytes = plan->chunk_bytes;
+    p.src_layer_stride = plan->src_layer_stride;
+    p.dst_layer_stride = plan->dst_layer_stride;
+    p.pairs_cap = pairs_cap;
+    p.layer_begin = layer_begin;
+    p.n_layers = layer_end - layer_begin;
+    p.nb_src = plan->src.num_blocks;
+    p.nb_dst = plan->dst.num_blocks;
+    p.heads_src = plan->heads_src;
+    p.heads_dst = plan->heads_dst;
+    p.heads_per_run = plan->heads_per_run;
+    p.runs_per_block = plan->runs_per_block;
+    p.chunks_per_run = (int32_t)(plan->run_bytes / plan->chunk_bytes);
+
+    DeviceInfo dev;
+    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * p.runs_per_block * p.chunks_per_run;
+    cudaError_t e;
+    const int path = plan->opt.copy_path ? plan->opt.copy_path : kDefaultCopyPath;
+    if (path == 1) {
+        const int per_sm = plan->opt.ctas_per_sm ? plan->opt.ctas_per_sm : 8;
+        const int grid = (int)std::min<int64_t>(max_items, (int64_t)dev.sms * per_sm);
+        kv_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
+        e = cudaGetLastError();
+    } else {
+        const BulkShape bs = bulk_shape(dev, plan->opt, (int)plan->chunk_bytes);
+        const int grid = (int)std::min<int64_t>((max_items + bs.warps - 1) / bs.warps, (int64_t)dev.sms * bs.ctas_per_sm);
+        switch (bs.stages) {
+            case 2: e = launch_bulk<2, 1>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+            case 3: e = launch_bulk<3, 2>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+            case 4: e = launch_bulk<4, 2>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+            case 6: e = launch_bulk<6, 3>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+            default: e = launch_bulk<8, 4>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+        }
+    }
+    if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    return AMOEBA_OK;
+}

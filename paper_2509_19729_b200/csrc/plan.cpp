@@ -1,0 +1,332 @@
+// Host planner of the TP a->b re-layout: validates the two layouts and derives, from the partition rules
+// (K/V headers per worker: Sec. 3.1 "Base solution"; weight rows / columns per worker: Sec. 3.2, Eq. 1),
+// which byte ranges go from which source worker to which destination worker.  No CUDA in this file.
+#include <algorithm>
+#include <atomic>
+#include <cstdlib>
+#include <new>
+#include <numeric>
+
+#include "plan.hpp"
+
+namespace amoeba {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static bool same_model(const amoeba_model& x, const amoeba_model& y) {
+    return x.num_layers == y.num_layers && x.hidden == y.hidden && x.num_q_heads == y.num_q_heads &&
+           x.num_kv_heads == y.num_kv_heads && x.head_dim == y.head_dim && x.intermediate == y.intermediate &&
+           x.elem_bytes == y.elem_bytes;
+}
+
+static amoeba_status check_layout(const amoeba_layout& l) {
+    const amoeba_model& m = l.model;
+    if (m.num_layers <= 0 || m.hidden <= 0 || m.num_q_heads <= 0 || m.num_kv_heads <= 0 || m.head_dim <= 0 ||
+        m.intermediate <= 0 || l.tp <= 0 || l.block_tokens <= 0 || l.num_blocks <= 0 || l.kv_layer_stride_bytes < 0)
+        return AMOEBA_ERR_INVALID_ARG;
+    if (m.elem_bytes != 2) return AMOEBA_ERR_UNSUPPORTED;
+    if (l.kv_order != AMOEBA_KV_HEAD_MAJOR) return AMOEBA_ERR_UNSUPPORTED;
+    if (l.tp > AMOEBA_MAX_TP) return AMOEBA_ERR_UNSUPPORTED;
+    // Even partition of the headers and of the FFN width over the workers; K/V header replication for
+    // tp > num_kv_heads is not a re-layout of existing state and is not handled.
+    if (m.num_q_heads % l.tp || m.num_kv_heads % l.tp || m.intermediate % l.tp) return AMOEBA_ERR_UNSUPPORTED;
+    if (m.num_q_heads % m.num_kv_heads) return AMOEBA_ERR_UNSUPPORTED;
+    return AMOEBA_OK;
+}
+
+// Largest divisor d of `total` with d <= cap and d % 16 == 0 (total % 16 == 0 is a precondition).
+static int64_t chunk_of(int64_t total, int64_t cap) {
+    for (int64_t n = std::max<int64_t>(1, (total + cap - 1) / cap); n <= total / 16; ++n)
+        if (total % n == 0 && (total / n) % 16 == 0) return total / n;
+    return 16;
+}
+
+amoeba_status finalize_chunks(amoeba_plan* p) {
+    const int64_t cap = p->opt.chunk_bytes > 0 ? p->opt.chunk_bytes : 16384;
+    if (cap < 16 || cap % 16) return AMOEBA_ERR_INVALID_ARG;
+    p->chunk_bytes = chunk_of(p->run_bytes, cap);
+    p->wdev.clear();
+    int64_t item = 0;
+    for (const amoeba_weight_desc& d : p->wdescs) {
+        WDescDev w{};
+        w.src_off = d.src_off;
+        w.dst_off = d.dst_off;
+        w.src_pitch = d.src_pitch;
+        w.dst_pitch = d.dst_pitch;
+        w.row_bytes = d.row_bytes;
+        w.n_rows = d.n_rows;
+        w.src_slot = d.src_rank * kNumTensors + d.src_tensor;
+        w.dst_slot = d.dst_rank * kNumTensors + d.dst_tensor;
+        if (d.row_bytes > cap) {
+            w.rows_per_item = 1;
+            w.col_chunks = (int32_t)((d.row_bytes + cap - 1) / cap);
+            w.chunk_bytes = (int32_t)cap;
+        } else {
+            w.rows_per_item = (int32_t)std::min<int64_t>(std::max<int64_t>(1, cap / d.row_bytes), d.n_rows);
+            w.col_chunks = 1;
+            w.chunk_bytes = (int32_t)d.row_bytes;
+        }
+        w.item_begin = (int32_t)item;
+        item += (int64_t)((d.n_rows + w.rows_per_item - 1) / w.rows_per_item) * w.col_chunks;
+        if (item > INT32_MAX) return AMOEBA_ERR_UNSUPPORTED;
+        p->wdev.push_back(w);
+    }
+    p->items_per_layer = (int32_t)item;
+    return AMOEBA_OK;
+}
+
+struct Range {
+    int64_t lo, hi;
+};
+static Range part(int64_t total, int tp, int r) { return {total / tp * r, total / tp * (r + 1)}; }
+
+// Tensors partitioned by output rows: shard r holds rows part(rows, tp, r) of the logical [rows, cols] tensor.
+// `sec_src` / `sec_dst` are the byte offsets of this tensor's section inside a fused worker buffer.
+static void add_row_split(std::vector<amoeba_weight_desc>& out, int a, int b, int64_t rows, int64_t row_bytes,
+                          int src_tensor, int64_t sec_src, int dst_tensor, int64_t sec_dst) {
+    for (int i = 0; i < a; ++i)
+        for (int j = 0; j < b; ++j) {
+            const Range s = part(rows, a, i), d = part(rows, b, j);
+            const int64_t lo = std::max(s.lo, d.lo), hi = std::min(s.hi, d.hi);
+            if (lo >= hi) continue;
+            amoeba_weight_desc w{};
+            w.src_rank = i;
+            w.dst_rank = j;
+            w.src_tensor = src_tensor;
+            w.dst_tensor = dst_tensor;
+            w.src_off = sec_src + (lo - s.lo) * row_bytes;
+            w.dst_off = sec_dst + (lo - d.lo) * row_bytes;
+            w.row_bytes = (hi - lo) * row_bytes;  // consecutive rows are one contiguous run
+            w.n_rows = 1;
+            w.src_pitch = w.dst_pitch = w.row_bytes;
+            out.push_back(w);
+        }
+}
+
+// Tensors partitioned by input columns: shard r holds columns part(cols, tp, r) of the logical [rows, cols]
+// tensor as a dense [rows, cols/tp] buffer.
+static void add_col_split(std::vector<amoeba_weight_desc>& out, int a, int b, int64_t rows, int64_t cols, int64_t e,
+                          int tensor) {
+    for (int i = 0; i < a; ++i)
+        for (int j = 0; j < b; ++j) {
+            const Range s = part(cols, a, i), d = part(cols, b, j);
+            const int64_t lo = std::max(s.lo, d.lo), hi = std::min(s.hi, d.hi);
+            if (lo >= hi) continue;
+            amoeba_weight_desc w{};
+            w.src_rank = i;
+            w.dst_rank = j;
+            w.src_tensor = w.dst_tensor = tensor;
+            w.src_off = (lo - s.lo) * e;
+            w.dst_off = (lo - d.lo) * e;
+            w.row_bytes = (hi - lo) * e;
+            w.n_rows = (int32_t)rows;
+            w.src_pitch = (s.hi - s.lo) * e;
+            w.dst_pitch = (d.hi - d.lo) * e;
+            if (w.src_pitch == w.row_bytes && w.dst_pitch == w.row_bytes) {  // both dense: one run
+                w.row_bytes *= rows;
+                w.n_rows = 1;
+                w.src_pitch = w.dst_pitch = w.row_bytes;
+            }
+            out.push_back(w);
+        }
+}
+
+}  // namespace amoeba
+
+using namespace amoeba;
+
+extern "C" {
+
+amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* dst, amoeba_plan** out) {
+    if (!src || !dst || !out) return AMOEBA_ERR_INVALID_ARG;
+    *out = nullptr;
+    amoeba_status st = check_layout(*src);
+    if (st != AMOEBA_OK) return st;
+    st = check_layout(*dst);
+    if (st != AMOEBA_OK) return st;
+    if (!same_model(src->model, dst->model) || src->block_tokens != dst->block_tokens) return AMOEBA_ERR_INVALID_ARG;
+
+    amoeba_plan* p = new (std::nothrow) amoeba_plan();
+    if (!p) return AMOEBA_ERR_INVALID_ARG;
+    p->src = *src;
+    p->dst = *dst;
+    const amoeba_model& m = src->model;
+    const int a = src->tp, b = dst->tp;
+    const int64_t e = m.elem_bytes;
+
+    // ---- KV: headers h .. h+g-1 with g = gcd(Hkv/a, Hkv/b) never straddle a worker boundary on either side,
+    // so each such group is one contiguous run in the source block and in the destination block.
+    p->heads_src = m.num_kv_heads / a;
+    p->heads_dst = m.num_kv_heads / b;
+    p->heads_per_run = std::gcd(p->heads_src, p->heads_dst);
+    p->runs_per_block = m.num_kv_heads / p->heads_per_run;
+    p->unit_bytes = 2 * (int64_t)src->block_tokens * m.head_dim * e;
+    p->run_bytes = p->heads_per_run * p->unit_bytes;
+    p->src_block_bytes = p->heads_src * p->unit_bytes;
+    p->dst_block_bytes = p->heads_dst * p->unit_bytes;
+    const int64_t src_dense = p->src_block_bytes * src->num_blocks, dst_dense = p->dst_block_bytes * dst->num_blocks;
+    p->src_layer_stride = src->kv_layer_stride_bytes ? src->kv_layer_stride_bytes : src_dense;
+    p->dst_layer_stride = dst->kv_layer_stride_bytes ? dst->kv_layer_stride_bytes : dst_dense;
+    if (p->src_layer_stride < src_dense || p->dst_layer_stride < dst_dense) {
+        delete p;
+        return AMOEBA_ERR_INVALID_ARG;
+    }
+    if (p->unit_bytes % 16 || p->src_layer_stride % 16 || p->dst_layer_stride % 16) {
+        delete p;
+        return AMOEBA_ERR_ALIGNMENT;
+    }
+
+    // ---- weights
+    const int64_t hid = m.hidden, qrows = (int64_t)m.num_q_heads * m.head_dim,
+                  kvrows = (int64_t)m.num_kv_heads * m.head_dim, I = m.intermediate;
+    const int64_t rb = hid * e;  // bytes of one [*, hidden] row
+    enum { Q, K, V, O, GATE, UP, DOWN };
+    auto& w = p->wdescs;
+    // fused buffers: [q_r; k_r; v_r] and [gate_r; up_r], named by their first member
+    const int64_t k_sec_s = src->fused_qkv ? qrows / a * rb : 0, v_sec_s = src->fused_qkv ? (qrows + kvrows) / a * rb : 0;
+    const int64_t k_sec_d = dst->fused_qkv ? qrows / b * rb : 0, v_sec_d = dst->fused_qkv ? (qrows + kvrows) / b * rb : 0;
+    add_row_split(w, a, b, qrows, rb, Q, 0, Q, 0);
+    add_row_split(w, a, b, kvrows, rb, src->fused_qkv ? Q : K, k_sec_s, dst->fused_qkv ? Q : K, k_sec_d);
+    add_row_split(w, a, b, kvrows, rb, src->fused_qkv ? Q : V, v_sec_s, dst->fused_qkv ? Q : V, v_sec_d);
+    add_col_split(w, a, b, hid, qrows, e, O);
+    add_row_split(w, a, b, I, rb, GATE, 0, GATE, 0);
+    add_row_split(w, a, b, I, rb, src->fused_gate_up ? GATE : UP, src->fused_gate_up ? I / a * rb : 0,
+                  dst->fused_gate_up ? GATE : UP, dst->fused_gate_up ? I / b * rb : 0);
+    add_col_split(w, a, b, hid, I, e, DOWN);
+    if ((int)w.size() > kMaxWeightDescs) {
+        delete p;
+        return AMOEBA_ERR_UNSUPPORTED;
+    }
+    p->weight_bytes_per_layer = 0;
+    for (const auto& d : w) {
+        if (d.row_bytes % 16 || d.src_off % 16 || d.dst_off % 16 || d.src_pitch % 16 || d.dst_pitch % 16) {
+            delete p;
+            return AMOEBA_ERR_ALIGNMENT;
+        }
+        p->weight_bytes_per_layer += d.row_bytes * d.n_rows;
+    }
+
+    if (const char* env = std::getenv("AMOEBA_COPY_PATH")) {
+        if (env[0] == 'l') p->opt.copy_path = 1;
+        if (env[0] == 't') p->opt.copy_path = 2;
+    }
+    st = finalize_chunks(p);
+    if (st != AMOEBA_OK) {
+        delete p;
+        return st;
+    }
+    *out = p;
+    return AMOEBA_OK;
+}
+
+void amoeba_plan_destroy(amoeba_plan* plan) { delete plan; }
+
+amoeba_status amoeba_layout_kv_pool_bytes(const amoeba_layout* l, int64_t* bytes) {
+    if (!l || !bytes) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_status st = check_layout(*l);
+    if (st != AMOEBA_OK) return st;
+    const amoeba_model& m = l->model;
+    const int64_t dense = (int64_t)l->num_blocks * (m.num_kv_heads / l->tp) * 2 * l->block_tokens * m.head_dim * m.elem_bytes;
+    if (l->kv_layer_stride_bytes && l->kv_layer_stride_bytes < dense) return AMOEBA_ERR_INVALID_ARG;
+    *bytes = (l->kv_layer_stride_bytes ? l->kv_layer_stride_bytes : dense) * m.num_layers;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_layout_weight_bytes(const amoeba_layout* l, int32_t tensor, int64_t* bytes) {
+    if (!l || !bytes || tensor < 0 || tensor >= kNumTensors) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_status st = check_layout(*l);
+    if (st != AMOEBA_OK) return st;
+    const amoeba_model& m = l->model;
+    const int64_t e = m.elem_bytes, hid = m.hidden, q = (int64_t)m.num_q_heads * m.head_dim / l->tp,
+                  kv = (int64_t)m.num_kv_heads * m.head_dim / l->tp, I = m.intermediate / l->tp;
+    int64_t rows = 0;  // rows of `hidden` elements each ([rows, hidden] or [hidden, rows]: same byte count)
+    switch (tensor) {
+        case 0: rows = l->fused_qkv ? q + 2 * kv : q; break;
+        case 1: case 2: rows = l->fused_qkv ? 0 : kv; break;
+        case 3: rows = q; break;
+        case 4: rows = l->fused_gate_up ? 2 * I : I; break;
+        case 5: rows = l->fused_gate_up ? 0 : I; break;
+        case 6: rows = I; break;
+    }
+    *bytes = rows * hid * e;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_plan_bytes(const amoeba_plan* plan, int64_t n_blocks, int64_t* kv_bytes_rw, int64_t* w_bytes_rw) {
+    if (!plan || n_blocks < 0) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_model& m = plan->src.model;
+    if (kv_bytes_rw) *kv_bytes_rw = 2 * n_blocks * m.num_layers * m.num_kv_heads * plan->unit_bytes;
+    if (w_bytes_rw) *w_bytes_rw = 2 * plan->weight_bytes_per_layer * m.num_layers;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_plan_kv_info(const amoeba_plan* plan, amoeba_kv_info* out) {
+    if (!plan || !out) return AMOEBA_ERR_INVALID_ARG;
+    out->heads_per_run = plan->heads_per_run;
+    out->runs_per_block = plan->runs_per_block;
+    out->run_bytes = plan->run_bytes;
+    out->chunk_bytes = plan->chunk_bytes;
+    out->src_block_bytes = plan->src_block_bytes;
+    out->dst_block_bytes = plan->dst_block_bytes;
+    out->src_layer_stride = plan->src_layer_stride;
+    out->dst_layer_stride = plan->dst_layer_stride;
+    return AMOEBA_OK;
+}
+
+int32_t amoeba_plan_num_weight_descs(const amoeba_plan* plan) { return plan ? (int32_t)plan->wdescs.size() : 0; }
+
+amoeba_status amoeba_plan_weight_desc(const amoeba_plan* plan, int32_t index, amoeba_weight_desc* out) {
+    if (!plan || !out || index < 0 || index >= (int32_t)plan->wdescs.size()) return AMOEBA_ERR_INVALID_ARG;
+    *out = plan->wdescs[index];
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t value) {
+    if (!plan || value < 0) return AMOEBA_ERR_INVALID_ARG;
+    Options old = plan->opt;
+    switch (option) {
+        case AMOEBA_OPT_COPY_PATH:
+            if (value > 2) return AMOEBA_ERR_INVALID_ARG;
+            plan->opt.copy_path = (int)value;
+            break;
+        case AMOEBA_OPT_CTAS_PER_SM:
+            if (value > 32) return AMOEBA_ERR_INVALID_ARG;
+            plan->opt.ctas_per_sm = (int)value;
+            break;
+        case AMOEBA_OPT_CHUNK_BYTES:
+            if (value > 65536) return AMOEBA_ERR_INVALID_ARG;
+            plan->opt.chunk_bytes = value;
+            break;
+        case AMOEBA_OPT_STAGES:
+            if (value > 16) return AMOEBA_ERR_INVALID_ARG;
+            plan->opt.stages = (int)value;
+            break;
+        default:
+            return AMOEBA_ERR_INVALID_ARG;
+    }
+    amoeba_status st = finalize_chunks(plan);
+    if (st != AMOEBA_OK) {
+        plan->opt = old;
+        finalize_chunks(plan);
+    }
+    return st;
+}
+
+int64_t amoeba_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* amoeba_status_string(amoeba_status s) {
+    switch (s) {
+        case AMOEBA_OK: return "ok";
+        case AMOEBA_ERR_INVALID_ARG: return "invalid argument";
+        case AMOEBA_ERR_UNSUPPORTED: return "unsupported layout";
+        case AMOEBA_ERR_ALIGNMENT: return "pointer, run or pitch not a multiple of 16 bytes";
+        case AMOEBA_ERR_NO_FREE_BLOCKS: return "not enough free destination blocks";
+        case AMOEBA_ERR_BAD_BLOCK_ID: return "block id out of range";
+        case AMOEBA_ERR_CUDA: return "CUDA runtime error";
+        case AMOEBA_ERR_TIMEOUT: return "on-device wait for a bulk copy ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,57 @@
+// Internal definitions shared by the host planner and the kernel launchers of the re-layout library.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "amoeba.h"
+
+namespace amoeba {
+
+constexpr int kNumTensors = 7;  // q,k,v,o,gate,up,down
+constexpr int kMaxWeightDescs = 160;
+constexpr int kMaxWeightPtrs = 2048;  // per launch: layers * (a + b) * kNumTensors pointers
+
+// One weight copy descriptor as the kernels see it (per layer, relative to that layer's buffers).
+struct WDescDev {
+    int64_t src_off, dst_off;      // bytes into the source / destination buffer
+    int64_t src_pitch, dst_pitch;  // bytes between consecutive rows
+    int64_t row_bytes;             // bytes per row
+    int32_t n_rows;
+    int32_t src_slot, dst_slot;    // rank * kNumTensors + tensor
+    int32_t rows_per_item;         // rows one work item covers (1 when a row is split into column chunks)
+    int32_t col_chunks;            // work items per row group along the row
+    int32_t chunk_bytes;           // bytes per column chunk (last one may be shorter)
+    int32_t item_begin;            // first work item of this descriptor within a layer
+    int32_t pad;
+};
+
+struct Options {
+    int copy_path = 0;    // 0 default, 1 vector ld/st, 2 bulk-copy ring
+    int ctas_per_sm = 0;  // 0 default
+    int64_t chunk_bytes = 0;
+    int stages = 0;
+};
+
+}  // namespace amoeba
+
+struct amoeba_plan {
+    amoeba_layout src, dst;
+    // KV
+    int32_t heads_src, heads_dst;  // K/V headers per source / destination worker
+    int32_t heads_per_run, runs_per_block;
+    int64_t unit_bytes;  // one (block, header): 2 * T * D * e
+    int64_t run_bytes, chunk_bytes;
+    int64_t src_block_bytes, dst_block_bytes, src_layer_stride, dst_layer_stride;
+    // weights
+    std::vector<amoeba_weight_desc> wdescs;  // public form
+    std::vector<amoeba::WDescDev> wdev;      // kernel form (chunked with the current options)
+    int32_t items_per_layer;
+    int64_t weight_bytes_per_layer;  // one copy (read side)
+    amoeba::Options opt;
+};
+
+namespace amoeba {
+// Re-derives chunk sizes and the per-descriptor work-item split from plan->opt.
+amoeba_status finalize_chunks(amoeba_plan* p);
+void count_launch(int n = 1);
+}  // namespace amoeba

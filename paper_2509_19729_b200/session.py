@@ -1,0 +1,135 @@
+"""Device-side state of one TP a->b transformation and the calls that run it.
+
+Plumbing only: allocates the source and destination buffers with torch (sizes come from the C library), uploads
+tables, and issues the three C-ABI calls of one transformation in order.  No re-layout arithmetic lives here.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as A
+
+
+def _carve(buf: torch.Tensor, sizes, align: int = 256):
+    """Views of `sizes` bytes each into one uint8 buffer, each starting on an `align` boundary."""
+    out, off = [], 0
+    for n in sizes:
+        out.append(buf[off:off + n])
+        off += (n + align - 1) // align * align
+    return out
+
+
+def _carved_bytes(sizes, align: int = 256) -> int:
+    return sum((n + align - 1) // align * align for n in sizes)
+
+
+class Session:
+    """All buffers of one transformation on one GPU.
+
+    model: shape dict (L, hidden, Hq, Hkv, D, I); a, b: source / destination TP; NB_src / NB_dst: pool capacities;
+    kv_layers: number of layers the KV pools hold (the first kv_layers layers; None = all); weights: allocate the
+    weight shards too.  Buffers are uint8 tensors; KV pools are one tensor per worker.
+    """
+
+    def __init__(self, model: dict, a: int, b: int, NB_src: int, NB_dst: int, num_seqs: int, max_blocks_per_seq: int,
+                 pairs_cap: int, kv_layers: Optional[int] = None, kv: bool = True, weights: bool = True,
+                 fused_qkv: bool = True, fused_gate_up: bool = True, block_tokens: int = 16, device="cuda:0",
+                 dst_fill: Optional[int] = 0xA5):
+        self.model, self.a, self.b = model, a, b
+        self.device = torch.device(device)
+        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up)
+        self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up)
+        self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
+        self.info = A.amoeba_plan_kv_info(self.plan)
+        self.L = model["L"]
+        self.kv_layers = self.L if kv_layers is None else kv_layers
+        self.num_seqs, self.maxb, self.pairs_cap = num_seqs, max_blocks_per_seq, pairs_cap
+        dev = self.device
+        i32 = dict(dtype=torch.int32, device=dev)
+        # tables
+        self.src_bt = torch.full((num_seqs, max_blocks_per_seq), -1, **i32)
+        self.dst_bt = torch.full((num_seqs, max_blocks_per_seq), -2, **i32)
+        self.seq_lens = torch.zeros(num_seqs, **i32)
+        self.pairs = torch.full((max(pairs_cap, 1), 2), -3, **i32)
+        self.num_pairs = torch.zeros(1, **i32)
+        self.free_count = torch.zeros(1, **i32)
+        self.status = torch.zeros(1, **i32)
+        self.free_list = None
+        self.free_mask = None
+        self.workspace = None
+        # KV pools: only the first kv_layers layers are held
+        self.src_pools, self.dst_pools = [], []
+        if kv:
+            for lay, tp, pools in ((self.src_layout, a, self.src_pools), (self.dst_layout, b, self.dst_pools)):
+                per_layer = A.amoeba_layout_kv_pool_bytes(lay) // self.L
+                for _ in range(tp):
+                    pools.append(torch.empty(per_layer * self.kv_layers, dtype=torch.uint8, device=dev))
+            if dst_fill is not None:
+                for p in self.dst_pools:
+                    p.fill_(dst_fill)
+        # weights: one buffer per worker, carved into [layer][tensor] views
+        self.src_w, self.dst_w, self._wbufs = [], [], []
+        if weights:
+            for lay, tp, out in ((self.src_layout, a, self.src_w), (self.dst_layout, b, self.dst_w)):
+                sizes = [A.amoeba_layout_weight_bytes(lay, t) for t in range(len(A.TENSOR_NAMES))]
+                used = [(n, s) for n, s in zip(A.TENSOR_NAMES, sizes) if s]
+                for _ in range(tp):
+                    buf = torch.empty(_carved_bytes([s for _, s in used]) * self.L, dtype=torch.uint8, device=dev)
+                    views = _carve(buf, [s for _, s in used] * self.L)
+                    self._wbufs.append(buf)
+                    out.append([{n: views[l * len(used) + i] for i, (n, _) in enumerate(used)} for l in range(self.L)])
+            if dst_fill is not None:
+                for buf in self._wbufs[a:]:
+                    buf.fill_(dst_fill)
+            self._src_w_packed = A.pack_weights(self.src_w)
+            self._dst_w_packed = A.pack_weights(self.dst_w)
+
+    # ---- inputs
+    def set_tables(self, seq_lens, src_bt, free_list=None, free_mask=None) -> None:
+        """Upload sequence lengths, the source block table and the destination free blocks (numpy or torch, host)."""
+        self.seq_lens.copy_(torch.as_tensor(seq_lens, dtype=torch.int32))
+        self.src_bt.copy_(torch.as_tensor(src_bt, dtype=torch.int32))
+        assert (free_list is None) != (free_mask is None)
+        if free_list is not None:
+            self.free_list = torch.as_tensor(free_list, dtype=torch.int32).to(self.device)
+            self.free_mask, n = None, self.free_list.numel()
+        else:
+            self.free_mask = torch.as_tensor(free_mask, dtype=torch.uint8).to(self.device)
+            self.free_list, n = None, self.free_mask.numel()
+        self.n_free_or_nb = n
+        self.workspace_bytes = A.amoeba_rewrite_workspace_bytes(self.plan, self.num_seqs, n)
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+
+    # ---- the three calls of one transformation
+    def rewrite_block_tables(self, stream=None) -> None:
+        A.amoeba_rewrite_block_tables(self.plan, self.src_bt, self.seq_lens, self.num_seqs, self.maxb, self.free_list,
+                                      self.free_mask, self.n_free_or_nb, self.dst_bt, self.pairs, self.pairs_cap,
+                                      self.num_pairs, self.free_count, self.status, self.workspace,
+                                      self.workspace_bytes, stream)
+
+    def reshard_kv(self, stream=None, layer_begin: int = 0, layer_end: Optional[int] = None) -> None:
+        A.amoeba_reshard_kv(self.plan, self.src_pools, self.dst_pools, self.pairs, self.num_pairs, self.pairs_cap,
+                            layer_begin, self.kv_layers if layer_end is None else layer_end, self.status, stream)
+
+    def reshard_weights(self, stream=None, layer_begin: int = 0, layer_end: Optional[int] = None) -> None:
+        A.amoeba_reshard_weights(self.plan, self._src_w_packed, self._dst_w_packed, layer_begin,
+                                 self.L if layer_end is None else layer_end, self.status, stream)
+
+    def step(self, stream=None) -> None:
+        """One whole transformation: table rewrite, KV migration, weight re-partition (asynchronous)."""
+        self.rewrite_block_tables(stream)
+        if self.src_pools:
+            self.reshard_kv(stream)
+        if self.src_w:
+            self.reshard_weights(stream)
+
+    def set_option(self, option: int, value: int) -> None:
+        A.amoeba_plan_set_option(self.plan, option, value)
+        self.info = A.amoeba_plan_kv_info(self.plan)
+
+    def bytes_rw(self, n_blocks: int):
+        """(KV bytes, weight bytes) read+written by one step with n_blocks live blocks over the held KV layers."""
+        kv, w = A.amoeba_plan_bytes(self.plan, n_blocks)
+        return kv * self.kv_layers // self.L if self.src_pools else 0, w if self.src_w else 0

@@ -1,0 +1,185 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: bit-exact on every output byte."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from harness import check_case, make_case, run_case
+
+pytestmark = pytest.mark.gpu
+
+LDST, BULK = 1, 2
+SMALL40 = dict(L=2, hidden=320, Hq=40, Hkv=40, D=16, I=640)  # 40-head shape: divisors 1,2,4,5,8,10,20,40
+GQA = dict(L=3, hidden=512, Hq=16, Hkv=8, D=128, I=1792)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    import torch
+
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_2509_19729_b200 as A
+
+    assert A.library_path().exists()
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+def test_tiny_config_end_to_end(path):
+    cfg = wl.CONFIGS["tiny_2to1"]
+    lens = wl.draw_seq_lens(cfg, name="tiny_2to1")
+    c = make_case(cfg["model"], cfg["a"], cfg["b"], lens, src_free=0.25, dst_slack=0.25, dtype="fp16", seed=1)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("a,b", [(1, 2), (2, 1), (1, 4), (4, 1), (2, 8), (8, 2), (4, 4), (1, 1), (8, 1), (1, 8)])
+def test_gqa_shapes_all_directions(path, a, b):
+    lens = [1, 16, 17, 300, 0, 77, 1024, 5]
+    c = make_case(GQA, a, b, lens, seed=a * 16 + b)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("a,b", [(4, 5), (5, 8), (8, 5), (10, 4), (10, 20), (20, 1), (5, 5)])
+def test_non_nested_partitions(path, a, b):
+    lens = [33, 7, 0, 64, 129]
+    c = make_case(SMALL40, a, b, lens, T=8, seed=a * 64 + b)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("fq,fg", [(False, False), (True, False), (False, True)])
+def test_unfused_weight_buffers(path, fq, fg):
+    c = make_case(GQA, 2, 4, [40], fused_qkv=fq, fused_gate_up=fg, kv=True, seed=5)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+def test_free_mask_compaction_and_foreign_blocks(path):
+    lens = list(np.random.default_rng(3).integers(1, 600, size=200))
+    c = make_case(dict(GQA, L=1), 4, 1, lens, dst_form="mask", dst_occupied=0.3, src_free=0.3, weights=False, seed=9)
+    s = run_case(c, path)
+    check_case(c, s)  # foreign (occupied) blocks keep the fill: whole-pool comparison
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("chunk", [1024, 4096, 8192, 32768])
+def test_chunk_sizes_and_ragged_tails(path, chunk):
+    import paper_2509_19729_b200 as A
+
+    lens = [16 * 37 + 3, 1, 16 * 64]
+    c = make_case(dict(L=2, hidden=1024 + 64, Hq=8, Hkv=8, D=128, I=2816 + 256), 2, 4, lens, seed=chunk)
+    check_case(c, run_case(c, path, options=[(A.OPT_CHUNK_BYTES, chunk)]))
+
+
+@pytest.mark.parametrize("stages", [2, 3, 4, 6, 8])
+def test_bulk_ring_depths(stages):
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 1, 4, [500, 20, 1000], seed=stages)
+    check_case(c, run_case(c, BULK, options=[(A.OPT_STAGES, stages)]))
+    check_case(c, run_case(c, BULK, options=[(A.OPT_STAGES, stages), (A.OPT_CHUNK_BYTES, 4096), (A.OPT_CTAS_PER_SM, 2)]))
+
+
+def test_long_single_row_and_many_sequences():
+    # one very long row (many 128-entry segments) next to many short ones; > 1024 sequences (several scan tiles)
+    lens = [16 * 3000] + list(np.random.default_rng(4).integers(0, 40, size=2500))
+    c = make_case(dict(L=1, hidden=128, Hq=2, Hkv=2, D=64, I=256), 1, 2, lens, weights=False, seed=11)
+    check_case(c, run_case(c, BULK))
+
+
+def test_empty_inputs():
+    c = make_case(GQA, 2, 1, [0, 0, 0], weights=False, seed=2)
+    check_case(c, run_case(c, BULK))
+
+
+def test_repeated_steps_are_idempotent():
+    c = make_case(GQA, 2, 4, [100, 200, 300], seed=21)
+    check_case(c, run_case(c, BULK, steps=3))
+
+
+# ---------------- device-detected errors (values, never traps) ----------------
+def test_not_enough_free_blocks():
+    lens = [160, 160]
+    free = (np.arange(19, dtype=np.int32), None)  # need 20
+    c = make_case(GQA, 2, 1, lens, free_override=free, weights=False, seed=3)
+    assert c.exp_status == 4
+    check_case(c, run_case(c, BULK))
+
+
+def test_invalid_lengths_and_pairs_cap():
+    c = make_case(GQA, 2, 1, [160, -5, 16], weights=False, seed=3)
+    assert c.exp_status == 1
+    check_case(c, run_case(c, LDST))
+    c = make_case(GQA, 2, 1, [160, 160], weights=False, seed=3, pairs_cap=19)
+    assert c.exp_status == 1
+    check_case(c, run_case(c, LDST))
+
+
+@pytest.mark.parametrize("path", [LDST, BULK])
+def test_bad_block_ids_are_skipped(path):
+    lens = [160, 48]
+    base = make_case(GQA, 2, 1, lens, weights=False, seed=4)
+    bt = base.src_bt.copy()
+    bt[0, 3] = base.NB_src + 7  # out of range source id
+    bt[1, 1] = -1               # hole inside a sequence
+    free = base.free_list.copy()
+    free[5] = base.NB_dst       # out of range destination id
+    c = make_case(GQA, 2, 1, lens, weights=False, seed=4, src_bt_override=bt, free_override=(free, None))
+    assert c.exp_status == 5
+    check_case(c, run_case(c, path))
+
+
+def test_host_detected_errors():
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    m = GQA
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_plan_create(A.make_layout(m, 3, 8), A.make_layout(m, 1, 8))
+    assert e.value.status == A.ERR_UNSUPPORTED
+    c = make_case(m, 2, 1, [40], weights=False, seed=1)
+    s = run_case(c, BULK)
+    with pytest.raises(A.AmoebaError) as e:  # misaligned pool pointer
+        A.amoeba_reshard_kv(s.plan, [s.src_pools[0].data_ptr() + 4, s.src_pools[1]], s.dst_pools, s.pairs,
+                            s.num_pairs, s.pairs_cap, 0, 1, s.status)
+    assert e.value.status == A.ERR_ALIGNMENT
+    with pytest.raises(A.AmoebaError) as e:  # layer range outside the model
+        A.amoeba_reshard_kv(s.plan, s.src_pools, s.dst_pools, s.pairs, s.num_pairs, s.pairs_cap, 0, m["L"] + 1,
+                            s.status)
+    assert e.value.status == A.ERR_INVALID_ARG
+    with pytest.raises(A.AmoebaError) as e:  # workspace too small
+        A.amoeba_rewrite_block_tables(s.plan, s.src_bt, s.seq_lens, s.num_seqs, s.maxb, s.free_list, None,
+                                      s.n_free_or_nb, s.dst_bt, s.pairs, s.pairs_cap, s.num_pairs, s.free_count,
+                                      s.status, s.workspace, 8)
+    assert e.value.status == A.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    check_case(c, s)  # the failed calls launched nothing
+
+
+def test_layer_ranges_compose():
+    """Transforming layer ranges one after the other (a few layers per inference step) equals one full call."""
+    import torch
+
+    c = make_case(GQA, 1, 2, [100, 37], seed=8)
+    s = run_case(c, BULK, steps=0)
+    s.status.zero_()
+    s.rewrite_block_tables()
+    for l in range(c.model["L"]):
+        s.reshard_kv(layer_begin=l, layer_end=l + 1)
+        s.reshard_weights(layer_begin=l, layer_end=l + 1)
+    torch.cuda.synchronize()
+    check_case(c, s)
+
+
+def test_side_stream():
+    import torch
+
+    c = make_case(GQA, 4, 2, [100, 37, 900], seed=12)
+    s = run_case(c, BULK, steps=0)
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        s.step(st)
+    st.synchronize()
+    check_case(c, s)

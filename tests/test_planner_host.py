@@ -1,0 +1,124 @@
+"""Host-side checks that need no GPU: the shared library loads and exports every declared symbol; the planner's
+descriptors, applied with plain numpy byte copies, reproduce the oracle's result; layout validation."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2509_19729_b200 as A
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SMALL40 = dict(L=1, hidden=40, Hq=40, Hkv=40, D=8, I=320)
+GQA = dict(L=1, hidden=64, Hq=16, Hkv=8, D=16, I=192)
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "amoeba.h")).read()
+    names = re.findall(r"AMOEBA_API\s+[\w\s\*]+?\b(amoeba_\w+)\s*\(", header)
+    assert len(names) >= 15 and len(set(names)) == len(names)
+    lib = C.CDLL(str(A.library_path()))
+    for n in names:
+        assert hasattr(lib, n), n
+    assert A.amoeba_status_string(0) == "ok" and "block" in A.amoeba_status_string(A.ERR_BAD_BLOCK_ID)
+
+
+def _apply_descs(plan, src_bufs, dst_bufs):
+    """src_bufs / dst_bufs: [rank][tensor index] -> uint8 arrays.  Returns per-destination write counts."""
+    counts = [[np.zeros(len(b), np.int32) if b is not None else None for b in r] for r in dst_bufs]
+    for i in range(A.amoeba_plan_num_weight_descs(plan)):
+        d = A.amoeba_plan_weight_desc(plan, i)
+        s, t = src_bufs[d.src_rank][d.src_tensor], dst_bufs[d.dst_rank][d.dst_tensor]
+        for r in range(d.n_rows):
+            so, to = d.src_off + r * d.src_pitch, d.dst_off + r * d.dst_pitch
+            t[to:to + d.row_bytes] = s[so:so + d.row_bytes]
+            counts[d.dst_rank][d.dst_tensor][to:to + d.row_bytes] += 1
+    return counts
+
+
+@pytest.mark.parametrize("fq,fg", [(True, True), (False, False)])
+@pytest.mark.parametrize("model,a,b", [(GQA, 1, 2), (GQA, 2, 1), (GQA, 1, 4), (GQA, 2, 8), (GQA, 8, 2), (GQA, 4, 4),
+                                       (SMALL40, 4, 5), (SMALL40, 5, 8), (SMALL40, 8, 5), (SMALL40, 10, 20),
+                                       (SMALL40, 20, 1)])
+def test_weight_descriptors_reproduce_oracle(oracle, model, a, b, fq, fg):
+    g = np.random.default_rng(a * 100 + b)
+    W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in oracle.logical_shapes(model).items()}
+    src = oracle.weights_shard(W, model, a, fq, fg)
+    exp = oracle.weights_transform(src, model, a, b, fq, fg)
+    plan = A.amoeba_plan_create(A.make_layout(model, a, 4, fused_qkv=fq, fused_gate_up=fg),
+                                A.make_layout(model, b, 4, fused_qkv=fq, fused_gate_up=fg))
+    as_bytes = lambda sh: [[sh_r[n].reshape(-1).view(np.uint8) if n in sh_r else None for n in A.TENSOR_NAMES]
+                           for sh_r in sh]
+    dst = [[np.full(e.size, 0xA5, np.uint8) if e is not None else None for e in r] for r in as_bytes(exp)]
+    counts = _apply_descs(plan, as_bytes(src), dst)
+    for r in range(b):
+        for t, n in enumerate(A.TENSOR_NAMES):
+            if n in exp[r]:
+                assert np.array_equal(dst[r][t], exp[r][n].reshape(-1).view(np.uint8)), (r, n)
+                assert np.all(counts[r][t] == 1)  # every destination byte written exactly once
+                lay = A.make_layout(model, b, 4, fused_qkv=fq, fused_gate_up=fg)
+                assert A.amoeba_layout_weight_bytes(lay, t) == exp[r][n].size * 2
+    kv, w = A.amoeba_plan_bytes(plan, 3)
+    assert w == 2 * sum(x.size * 2 for x in W.values())
+    assert kv == 2 * 3 * model["L"] * model["Hkv"] * 2 * 16 * model["D"] * 2
+
+
+@pytest.mark.parametrize("Hkv,a,b", [(8, 1, 4), (8, 2, 8), (8, 8, 2), (40, 4, 5), (40, 5, 8), (40, 10, 20), (32, 1, 2)])
+def test_kv_runs_never_straddle_a_worker(oracle, Hkv, a, b):
+    m = dict(L=2, hidden=Hkv * 8, Hq=Hkv, Hkv=Hkv, D=8, I=Hkv * 8)
+    plan = A.amoeba_plan_create(A.make_layout(m, a, 10), A.make_layout(m, b, 12))
+    info = A.amoeba_plan_kv_info(plan)
+    g = info.heads_per_run
+    assert g * info.runs_per_block == Hkv
+    unit = 2 * 16 * m["D"] * 2
+    assert info.run_bytes == g * unit and info.run_bytes % info.chunk_bytes == 0 and info.chunk_bytes % 16 == 0
+    assert info.src_block_bytes == Hkv // a * unit and info.dst_block_bytes == Hkv // b * unit
+    assert info.src_layer_stride == 10 * info.src_block_bytes and info.dst_layer_stride == 12 * info.dst_block_bytes
+    for run in range(info.runs_per_block):
+        heads = range(run * g + 1, (run + 1) * g + 1)  # 1-indexed headers of this run
+        assert len({oracle.worker_of_header(Hkv, a, h) for h in heads}) == 1
+        assert len({oracle.worker_of_header(Hkv, b, h) for h in heads}) == 1
+    # and no larger uniform run would do
+    if g < Hkv:
+        bigger = [k for k in range(g + 1, Hkv + 1) if Hkv % k == 0 and (Hkv // a) % k == 0 and (Hkv // b) % k == 0]
+        assert not bigger
+
+
+def test_layout_validation():
+    m = GQA
+    ok = A.make_layout(m, 2, 8)
+    for bad, code in [
+        (A.make_layout(m, 3, 8), A.ERR_UNSUPPORTED),                     # 3 does not divide the head counts
+        (A.make_layout(m, 16, 8), A.ERR_UNSUPPORTED),                    # more workers than K/V heads
+        (A.make_layout(m, 2, 0), A.ERR_INVALID_ARG),                     # empty pool
+        (A.make_layout(dict(m, D=12), 2, 8), A.ERR_INVALID_ARG),         # different model on the two sides
+        (A.make_layout(m, 2, 8, block_tokens=8), A.ERR_INVALID_ARG),     # different block size
+        (A.make_layout(m, 2, 8, elem_bytes=3), A.ERR_UNSUPPORTED),
+        (A.make_layout(m, 2, 8, kv_layer_stride_bytes=1024), A.ERR_INVALID_ARG),  # stride smaller than a layer
+    ]:
+        with pytest.raises(A.AmoebaError) as e:
+            A.amoeba_plan_create(ok, bad)
+        assert e.value.status == code, (e.value.status, code)
+    tiny_rows = dict(L=1, hidden=4, Hq=2, Hkv=2, D=2, I=4)  # 8-byte rows: not copyable in 16-byte units
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_plan_create(A.make_layout(tiny_rows, 1, 8), A.make_layout(tiny_rows, 2, 8))
+    assert e.value.status == A.ERR_ALIGNMENT
+    plan = A.amoeba_plan_create(ok, A.make_layout(m, 4, 8))
+    with pytest.raises(A.AmoebaError):
+        A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, 24)  # not a multiple of 16
+    A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, 1024)
+    assert A.amoeba_plan_kv_info(plan).chunk_bytes == 1024
+    assert A.amoeba_rewrite_workspace_bytes(plan, 10, 100) >= 64 + 44 + 400
+
+
+def test_no_device_means_cuda_error_not_a_fallback():
+    import torch
+
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    m = GQA
+    plan = A.amoeba_plan_create(A.make_layout(m, 2, 8), A.make_layout(m, 1, 8))
+    with pytest.raises(A.AmoebaError) as e:  # non-null fake addresses, aligned: passes validation, then no device
+        A.amoeba_reshard_kv(plan, [4096, 8192], [12288], 4096, 4096, 4, 0, 1, 4096, stream=0)
+    assert e.value.status == A.ERR_CUDA
