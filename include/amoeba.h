@@ -47,7 +47,8 @@ typedef enum {
     AMOEBA_ERR_NO_FREE_BLOCKS = 4, /* destination has fewer free blocks than the sequences need */
     AMOEBA_ERR_BAD_BLOCK_ID = 5,   /* a block id outside its pool (or -1 inside a sequence) */
     AMOEBA_ERR_CUDA = 6,           /* a CUDA runtime call failed (launch error, no device) */
-    AMOEBA_ERR_TIMEOUT = 7         /* a bounded on-device wait on the kernel's own bulk copy ran out */
+    AMOEBA_ERR_TIMEOUT = 7,        /* a bounded on-device wait on the kernel's own bulk copy ran out */
+    AMOEBA_ERR_TOO_LARGE = 8       /* the problem needs more scratch than the library's built-in scratch array holds */
 } amoeba_status;
 
 enum { AMOEBA_KV_HEAD_MAJOR = 0 /* [block][header][K/V][token][dim], Sec. 3.1 Improvement 1 */ };
@@ -163,6 +164,39 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
                                           int32_t pairs_cap, int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
                                           int32_t* d_status, void* d_workspace, int64_t workspace_bytes,
                                           void* cuda_stream);
+
+/*
+ * amoeba_rewrite_block_tables_builtin_scratch  (no counterpart in the paper: a packaging variant of the call above)
+ *
+ * Same computation, same arguments and same outputs as amoeba_rewrite_block_tables, minus the workspace: the scratch
+ * the two kernels need lives in an array that is part of the library's device image instead of being supplied by the
+ * caller.  It exists for callers that must not, or cannot, allocate device memory at the point where a
+ * transformation is triggered: a serving process whose memory pool has already claimed the whole GPU for weights and
+ * KV blocks (so a cudaMalloc would fail or fragment the pool), code running inside a region where allocation is
+ * forbidden by the host framework, or a plug-in that is handed buffers and a stream but no allocator.  This call
+ * performs no cudaMalloc / cudaFree and calls no allocating routine of any library.
+ *
+ * Limit: the scratch array is AMOEBA_BUILTIN_SCRATCH_BYTES (1 MiB) per GPU, held by every GPU that loads the library
+ * until the process exits.  It must cover amoeba_rewrite_workspace_bytes(num_seqs, n_free_or_nb), i.e. roughly
+ * num_seqs + n_free_or_nb <= 262 000 table entries; larger problems are refused with AMOEBA_ERR_TOO_LARGE and
+ * nothing is launched - use amoeba_rewrite_block_tables with your own workspace for those.
+ *
+ * First use on a device: the first call made while a given device is current looks up that device's address of the
+ * array (one cudaGetSymbolAddress, checked; AMOEBA_ERR_CUDA if it fails) and remembers it.  Make that first call
+ * during start-up, outside any stream capture; later calls on the device only launch the two kernels.
+ *
+ * Sharing: all calls on one GPU use the same array, and it keeps whatever the previous call left in it.  Nothing in
+ * it has to start at zero (the kernels write every word before reading it), so no clearing is needed; but two calls
+ * whose kernels can overlap on the GPU (different streams without an ordering between them, or different threads or
+ * processes' worth of streams on one context) race on it and produce garbage.  Order such calls on one stream, or
+ * with events, or give the concurrent ones their own workspace through amoeba_rewrite_block_tables.
+ */
+enum { AMOEBA_BUILTIN_SCRATCH_BYTES = 1 << 20 };
+AMOEBA_API amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
+    const amoeba_plan* plan, const int32_t* d_src_bt, const int32_t* d_seq_lens, int32_t num_seqs,
+    int32_t max_blocks_per_seq, const int32_t* d_dst_free_list, const uint8_t* d_dst_free_mask, int32_t n_free_or_nb,
+    int32_t* d_dst_bt, int32_t* d_pairs, int32_t pairs_cap, int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
+    int32_t* d_status, void* cuda_stream);
 
 /*
  * amoeba_reshard_kv  (KV cache migration in the head dimension, Sec. 3.1: every header of every live block moves

@@ -19,10 +19,14 @@ __all__ = [
     "amoeba_launch_count", "amoeba_status_string", "library_path", "make_layout",
 ]
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NO_FREE_BLOCKS, ERR_BAD_BLOCK_ID, ERR_CUDA, ERR_TIMEOUT = range(8)
-STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS", "BAD_BLOCK_ID", "CUDA", "TIMEOUT"]
+(OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NO_FREE_BLOCKS, ERR_BAD_BLOCK_ID, ERR_CUDA, ERR_TIMEOUT,
+ ERR_TOO_LARGE) = range(9)
+STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS", "BAD_BLOCK_ID", "CUDA", "TIMEOUT",
+                "TOO_LARGE"]
+BUILTIN_SCRATCH_BYTES = 1 << 20
 __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
-            "ERR_CUDA", "ERR_TIMEOUT"]
+            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "BUILTIN_SCRATCH_BYTES",
+            "amoeba_rewrite_block_tables_builtin_scratch"]
 OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES = range(4)
 COPY_PATH_LDST, COPY_PATH_BULK = 1, 2
 TENSOR_NAMES = ("q", "k", "v", "o", "gate", "up", "down")
@@ -91,6 +95,7 @@ def _load():
         "amoeba_plan_set_option": (I32, [VP, I32, I64]),
         "amoeba_rewrite_workspace_bytes": (I32, [VP, I32, I32, P(I64)]),
         "amoeba_rewrite_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP, I64, VP]),
+        "amoeba_rewrite_block_tables_builtin_scratch": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP]),
         "amoeba_reshard_kv": (I32, [VP, P(VP), P(VP), VP, VP, I32, I32, I32, VP, VP]),
         "amoeba_reshard_weights": (I32, [VP, P(LayerWeights), P(LayerWeights), I32, I32, VP, VP]),
         "amoeba_launch_count": (I64, []),
@@ -211,6 +216,22 @@ def amoeba_rewrite_block_tables(plan: Plan, src_bt, seq_lens, num_seqs: int, max
         _ptr(dst_free_mask), n_free_or_nb, _ptr(dst_bt), _ptr(pairs), pairs_cap, _ptr(num_pairs),
         _ptr(dst_free_count_out), _ptr(status), _ptr(workspace), workspace_bytes, _stream(stream)),
         "amoeba_rewrite_block_tables")
+
+
+def amoeba_rewrite_block_tables_builtin_scratch(plan: Plan, src_bt, seq_lens, num_seqs: int, max_blocks_per_seq: int,
+                                                dst_free_list, dst_free_mask, n_free_or_nb: int, dst_bt, pairs,
+                                                pairs_cap: int, num_pairs, dst_free_count_out, status,
+                                                stream=None) -> None:
+    """``amoeba_rewrite_block_tables`` for callers that cannot allocate device memory (a serving process whose pool
+    owns the whole GPU, code inside a no-allocation region, a plug-in without an allocator): the scratch is a 1 MiB
+    array built into the library, so no workspace is passed.  Problems whose workspace would exceed
+    ``BUILTIN_SCRATCH_BYTES`` raise ``AmoebaError`` with ``ERR_TOO_LARGE``.  The first call on a device resolves the
+    array's address (do it at start-up, outside stream capture); calls that may overlap on the GPU share the array
+    and must be ordered by the caller."""
+    _check(_load().amoeba_rewrite_block_tables_builtin_scratch(
+        plan.handle, _ptr(src_bt), _ptr(seq_lens), num_seqs, max_blocks_per_seq, _ptr(dst_free_list),
+        _ptr(dst_free_mask), n_free_or_nb, _ptr(dst_bt), _ptr(pairs), pairs_cap, _ptr(num_pairs),
+        _ptr(dst_free_count_out), _ptr(status), _stream(stream)), "amoeba_rewrite_block_tables_builtin_scratch")
 
 
 def amoeba_reshard_kv(plan: Plan, src_pools: Sequence, dst_pools: Sequence, pairs, num_pairs, pairs_cap: int,

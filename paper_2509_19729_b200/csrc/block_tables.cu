@@ -7,6 +7,8 @@
 //                       id; writes the destination table (with -1 padding) and the (source, destination) pair list.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "launch.hpp"
 #include "plan.hpp"
 
@@ -208,4 +210,47 @@ extern "C" amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
     if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();
     return AMOEBA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate device memory: the scratch is an array in the library's device image.
+namespace amoeba {
+
+// One copy per GPU that loads this library, alive until the process exits.
+static __device__ __align__(256) unsigned char g_builtin_scratch[AMOEBA_BUILTIN_SCRATCH_BYTES];
+
+// In host code `g_builtin_scratch` is only a handle for the runtime, not an address a kernel could use; the
+// device-side address is asked for once per device and remembered here (index = device ordinal).
+constexpr int kMaxDevices = 64;
+static void* g_builtin_scratch_addr[kMaxDevices];
+static std::mutex g_builtin_scratch_mutex;
+
+}  // namespace amoeba
+
+extern "C" amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
+    const amoeba_plan* plan, const int32_t* d_src_bt, const int32_t* d_seq_lens, int32_t num_seqs,
+    int32_t max_blocks_per_seq, const int32_t* d_dst_free_list, const uint8_t* d_dst_free_mask, int32_t n_free_or_nb,
+    int32_t* d_dst_bt, int32_t* d_pairs, int32_t pairs_cap, int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
+    int32_t* d_status, void* cuda_stream) {
+    int64_t need = 0;
+    const amoeba_status st = amoeba_rewrite_workspace_bytes(plan, num_seqs, n_free_or_nb, &need);
+    if (st != AMOEBA_OK) return st;
+    if (need > (int64_t)AMOEBA_BUILTIN_SCRATCH_BYTES) return AMOEBA_ERR_TOO_LARGE;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AMOEBA_ERR_CUDA;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_builtin_scratch_mutex);
+        if (!g_builtin_scratch_addr[dev]) {  // first use with this device current
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) return AMOEBA_ERR_CUDA;
+            g_builtin_scratch_addr[dev] = p;
+        }
+        scratch = g_builtin_scratch_addr[dev];
+    }
+    return amoeba_rewrite_block_tables(plan, d_src_bt, d_seq_lens, num_seqs, max_blocks_per_seq, d_dst_free_list,
+                                       d_dst_free_mask, n_free_or_nb, d_dst_bt, d_pairs, pairs_cap, d_num_pairs,
+                                       d_dst_free_count_out, d_status, scratch, AMOEBA_BUILTIN_SCRATCH_BYTES,
+                                       cuda_stream);
 }

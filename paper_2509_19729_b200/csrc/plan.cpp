@@ -325,6 +325,7 @@ const char* amoeba_status_string(amoeba_status s) {
         case AMOEBA_ERR_BAD_BLOCK_ID: return "block id out of range";
         case AMOEBA_ERR_CUDA: return "CUDA runtime error";
         case AMOEBA_ERR_TIMEOUT: return "on-device wait for a bulk copy ran out";
+        case AMOEBA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch array";
     }
     return "unknown status";
 }
