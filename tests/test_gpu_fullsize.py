@@ -1,0 +1,97 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times.
+
+The source buffers are filled on the device with a counter hash; the tables are compared whole with the oracle's;
+the KV result is compared on sampled (layer, sequence, block) units - for each, the source worker slices are fetched,
+the oracle re-lays-out that one block on the CPU, and the destination worker slices must equal it; the weights of
+sampled layers are compared whole.  Size-independent properties: word sums are conserved, untouched destination
+blocks keep their fill."""
+import numpy as np
+import pytest
+
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FULL = ["llama3_8b_1to4", "llama3_8b_2to8", "llama2_7b_1to2", "llama2_13b_4to1", "llama3_70b_slice_8to2"]
+
+
+def _block_view(pool, n_layers, NB):
+    return pool.view(n_layers, NB, -1)  # [layer][block][bytes of one block in this worker's pool]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_config(name, oracle):
+    import torch
+
+    import bench
+
+    assert torch.cuda.is_available()
+    cfg = wl.CONFIGS[name]
+    m, a, b, T = cfg["model"], cfg["a"], cfg["b"], wl.BLOCK_TOKENS
+    device = torch.device("cuda:0")
+    s, st = bench.build_session(name, device)
+    try:
+        s.status.zero_()
+        s.step()
+        torch.cuda.synchronize()
+
+        # ---- tables: whole comparison
+        exp_bt, exp_pairs, exp_n, exp_left, exp_status = oracle.assign_blocks(
+            st["seq_lens"], T, st["src_bt"], st["NB_src"], st["NB_dst"], free_list=st.get("dst_free_list"),
+            free_mask=st.get("dst_free_mask"), pairs_cap=st["n_live"])
+        assert exp_status == 0 and int(s.status.item()) == 0
+        assert int(s.num_pairs.item()) == exp_n == st["n_live"] and int(s.free_count.item()) == exp_left
+        dst_bt = s.dst_bt.cpu().numpy()
+        assert np.array_equal(dst_bt, exp_bt)
+        assert np.array_equal(s.pairs.cpu().numpy()[:exp_n], exp_pairs)
+
+        # ---- KV: sampled blocks, each re-laid-out by the oracle on its own
+        Lkv = s.kv_layers
+        src_v = [_block_view(p, Lkv, st["NB_src"]) for p in s.src_pools]
+        dst_v = [_block_view(p, Lkv, st["NB_dst"]) for p in s.dst_pools]
+        g = np.random.default_rng(7)
+        one = dict(m, L=1)
+        seqs = np.flatnonzero(st["blocks_per_seq"] > 0)
+        for _ in range(96):
+            l = int(g.integers(Lkv))
+            q = int(g.choice(seqs))
+            i = int(g.integers(st["blocks_per_seq"][q]))
+            sid, did = int(st["src_bt"][q, i]), int(dst_bt[q, i])
+            src1 = [v[l, sid].cpu().numpy().view(np.uint16).copy() for v in src_v]  # NB = 1 pools
+            exp1 = [np.zeros(d[l, did].numel() // 2, np.uint16) for d in dst_v]
+            oracle.kv_transform(one, T, [T], a, 1, [[0]], src1, b, 1, [[0]], exp1)
+            for r in range(b):
+                got = dst_v[r][l, did].cpu().numpy().view(np.uint16)
+                assert np.array_equal(got, exp1[r]), (name, l, q, i, r)
+
+        # ---- untouched destination blocks keep the fill (sampled)
+        used = np.zeros(st["NB_dst"], bool)
+        used[exp_pairs[:, 1]] = True
+        idle = np.flatnonzero(~used)
+        if idle.size:
+            for did in g.choice(idle, size=min(16, idle.size), replace=False):
+                for v in dst_v:
+                    assert bool((v[int(g.integers(Lkv)), int(did)] == 0xA5).all())
+
+        # ---- word sums are conserved over the live blocks of every layer (any size, any permutation)
+        live_src = torch.as_tensor(exp_pairs[:, 0].astype(np.int64), device=device)
+        live_dst = torch.as_tensor(exp_pairs[:, 1].astype(np.int64), device=device)
+        for l in sorted(set(int(x) for x in g.integers(Lkv, size=3))):
+            ssum = sum(int(v[l].view(torch.int64).view(st["NB_src"], -1).index_select(0, live_src).sum().item())
+                       for v in src_v)
+            dsum = sum(int(v[l].view(torch.int64).view(st["NB_dst"], -1).index_select(0, live_dst).sum().item())
+                       for v in dst_v)
+            assert (ssum - dsum) % (1 << 64) == 0
+
+        # ---- weights: whole comparison of sampled layers
+        for l in sorted(set([0, m["L"] - 1, int(g.integers(m["L"]))])):
+            src_sh = [{n: t.cpu().numpy().view(np.uint16).reshape(oracle.shard_shapes(m, a)[n])
+                       for n, t in s.src_w[r][l].items()} for r in range(a)]
+            exp = oracle.weights_transform(src_sh, m, a, b)
+            for r in range(b):
+                for n, e in exp[r].items():
+                    got = s.dst_w[r][l][n].cpu().numpy().view(np.uint16)
+                    assert np.array_equal(got, e.reshape(-1)), (name, "weights", l, r, n)
+    finally:
+        del s
+        torch.cuda.empty_cache()

@@ -39,7 +39,7 @@ CONFIGS = {
                            kv_layers=None),
     "llama2_13b_4to1": dict(model=_model(40, 5120, 40, 40, 128, 13824), dtype="bf16", a=4, b=1, S=256,
                             lens=("lognormal", 1024, 1.0, 32768), src_free=0.30, dst_form="mask",
-                            dst_occupied=0.30, dst_slack=0.0, kv_layers=6),
+                            dst_occupied=0.30, dst_slack=0.0, kv_layers=4),
     "llama3_8b_1to4": dict(model=_model(32, 4096, 32, 8, 128, 14336), dtype="bf16", a=1, b=4, S=128,
                            lens=("uniform", 512, 8192), src_free=0.0, dst_form="list", dst_slack=1 / 64,
                            kv_layers=None),
