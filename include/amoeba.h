@@ -121,12 +121,20 @@ typedef struct {
 AMOEBA_API int32_t amoeba_plan_num_weight_descs(const amoeba_plan* plan);
 AMOEBA_API amoeba_status amoeba_plan_weight_desc(const amoeba_plan* plan, int32_t index, amoeba_weight_desc* out);
 
-/* Tuning knobs (defaults are chosen from measurements; the tests and the benchmark sweep them). */
+/* Tuning knobs (defaults are chosen from measurements; the tests and the benchmark sweep them).  An option id
+ * sets both copy kernels; id + AMOEBA_OPT_WEIGHTS_ONLY sets the weight kernel only, id + AMOEBA_OPT_KV_ONLY the KV
+ * kernel only.  Value 0 = the kernel's default. */
 enum {
-    AMOEBA_OPT_COPY_PATH = 0,   /* 0 = default, 1 = 16-byte vector loads/stores, 2 = bulk-copy (TMA) ring */
-    AMOEBA_OPT_CTAS_PER_SM = 1, /* persistent grid = this * SM count (0 = default) */
-    AMOEBA_OPT_CHUNK_BYTES = 2, /* upper bound of one copy work item (0 = default) */
-    AMOEBA_OPT_STAGES = 3       /* bulk-copy ring depth per warp (0 = default) */
+    AMOEBA_OPT_COPY_PATH = 0,   /* 1 = 16-byte vector loads/stores, 2 = bulk-copy (TMA) ring per warp,
+                                   3 = bulk-copy ring shared by a producer warp and a consumer warp */
+    AMOEBA_OPT_CTAS_PER_SM = 1, /* persistent grid = this * SM count */
+    AMOEBA_OPT_CHUNK_BYTES = 2, /* upper bound of one copy work item, multiple of 16, <= 65536 */
+    AMOEBA_OPT_STAGES = 3,      /* bulk-copy ring depth (2..16) */
+    AMOEBA_OPT_LAG = 4,         /* path 2: loads issued ahead of stores; path 3: stores kept in flight (< stages) */
+    AMOEBA_OPT_WARPS = 5,       /* bulk-copy rings per CTA */
+    AMOEBA_OPT_L2_HINT = 6,     /* 1 = none, 2 = loads evict-first, 3 = stores evict-first, 4 = both */
+    AMOEBA_OPT_WEIGHTS_ONLY = 16,
+    AMOEBA_OPT_KV_ONLY = 32
 };
 AMOEBA_API amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t value);
 

@@ -7,7 +7,8 @@ binding never do, and nothing here imports them.
 Conventions (see the C file for the passages of the paper each function follows):
   * elements are opaque 16-bit words, numpy ``uint16``;
   * logical KV is ``KV[L][G][Hkv][2][D]`` with ``G`` the number of block-padded tokens of all sequences;
-  * a KV pool of one worker is ``pool[L][NB][Hkv/TP][2][T][D]``;
+  * a KV pool of one worker is ``pool[L][NB][Hkv/TP][2][T][D]`` (header-centric) or
+    ``pool[L][2][NB][T][Hkv/TP][D]`` (token-first);
   * one layer's logical weights are a dict ``{q,k,v,o,gate,up,down}`` of ``[out,in]`` arrays.
 """
 from __future__ import annotations
@@ -24,6 +25,7 @@ _SRC = _HERE / "amoeba_oracle.c"
 _LIB = _HERE / "liboracle.so"
 
 OK, INVALID_ARG, NO_FREE_BLOCKS, BAD_BLOCK_ID = 0, 1, 4, 5
+HEADER_CENTRIC, TOKEN_FIRST = 0, 1  # KV storage orders (Sec. 3.1)
 
 
 def build(force: bool = False) -> Path:
@@ -99,8 +101,8 @@ def pool_elems_per_layer(m: dict, T: int, TP: int, NB: int) -> int:
     return NB * (m["Hkv"] // TP) * 2 * T * m["D"]
 
 
-def kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=0xA5A5, layer_stride=None):
-    """Logical KV -> list of TP pools ``[L][NB][Hkv/TP][2][T][D]`` (uint16), untouched words = ``fill``."""
+def kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=0xA5A5, layer_stride=None, order=HEADER_CENTRIC):
+    """Logical KV -> list of TP pools (uint16, ``order`` storage order), untouched words = ``fill``."""
     sl, slp = _i32(seq_lens)
     bt, btp = _i32(bt)
     per = pool_elems_per_layer(m, T, TP, NB)
@@ -108,53 +110,47 @@ def kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=0xA5A5, layer_stride=None):
     pools = [np.full(m["L"] * stride, fill, dtype=np.uint16) for _ in range(TP)]
     KV = np.ascontiguousarray(KV, dtype=np.uint16)
     mm = _model(m)
-    lib().oracle_kv_shard(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(stride), len(sl), slp, btp,
-                          bt.shape[1], _ptr_array(pools))
+    lib().oracle_kv_shard(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, NB, order, C.c_int64(stride), len(sl),
+                          slp, btp, bt.shape[1], _ptr_array(pools))
     return pools
 
 
-def kv_shard_into(KV, m, T, TP, seq_lens, bt, pools, layer_stride):
-    """Same as kv_shard but writes over existing pools (their other words are preserved)."""
-    sl, slp = _i32(seq_lens)
-    bt, btp = _i32(bt)
-    KV = np.ascontiguousarray(KV, dtype=np.uint16)
-    mm = _model(m)
-    lib().oracle_kv_shard(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(layer_stride), len(sl), slp,
-                          btp, bt.shape[1], _ptr_array(pools))
-
-
-def kv_reconstruct(pools, m, T, TP, NB, seq_lens, bt, layer_stride=None):
+def kv_reconstruct(pools, m, T, TP, NB, seq_lens, bt, layer_stride=None, order=HEADER_CENTRIC):
     sl, slp = _i32(seq_lens)
     bt, btp = _i32(bt)
     G = padded_tokens(sl, T)
     KV = np.zeros((m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
     stride = pool_elems_per_layer(m, T, TP, NB) if layer_stride is None else layer_stride
     mm = _model(m)
-    lib().oracle_kv_reconstruct(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, C.c_int64(stride), len(sl), slp,
-                                btp, bt.shape[1], _ptr_array(pools))
+    lib().oracle_kv_reconstruct(KV.ctypes.data_as(C.c_void_p), C.byref(mm), T, TP, NB, order, C.c_int64(stride),
+                                len(sl), slp, btp, bt.shape[1], _ptr_array(pools))
     return KV
 
 
-def kv_transform(m, T, seq_lens, a, NB_src, src_bt, src_pools, b, NB_dst, dst_bt, dst_pools):
+def kv_transform(m, T, seq_lens, a, NB_src, src_bt, src_pools, b, NB_dst, dst_bt, dst_pools,
+                 src_order=HEADER_CENTRIC, dst_order=HEADER_CENTRIC):
     """TP a->b on the KV pools: writes the live blocks of ``dst_pools`` in place (reconstruct, then shard)."""
     sl, slp = _i32(seq_lens)
     sbt, sbtp = _i32(src_bt)
     dbt, dbtp = _i32(dst_bt)
     assert sbt.shape == dbt.shape
     mm = _model(m)
-    rc = lib().oracle_kv_transform(C.byref(mm), T, len(sl), slp, sbt.shape[1], a,
+    rc = lib().oracle_kv_transform(C.byref(mm), T, len(sl), slp, sbt.shape[1], a, NB_src, src_order,
                                    C.c_int64(pool_elems_per_layer(m, T, a, NB_src)), sbtp, _ptr_array(src_pools), b,
-                                   C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)), dbtp, _ptr_array(dst_pools))
+                                   NB_dst, dst_order, C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)), dbtp,
+                                   _ptr_array(dst_pools))
     assert rc == 0
 
 
-def kv_copy_pairs(m, T, a, NB_src, src_pools, b, NB_dst, dst_pools, pairs, num_pairs, status=0):
+def kv_copy_pairs(m, T, a, NB_src, src_pools, b, NB_dst, dst_pools, pairs, num_pairs, status=0,
+                  src_order=HEADER_CENTRIC, dst_order=HEADER_CENTRIC):
     pr, prp = _i32(pairs)
     st = C.c_int32(status)
     mm = _model(m)
-    lib().oracle_kv_copy_pairs(C.byref(mm), T, a, NB_src, C.c_int64(pool_elems_per_layer(m, T, a, NB_src)),
-                               _ptr_array(src_pools), b, NB_dst, C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)),
-                               _ptr_array(dst_pools), prp, int(num_pairs), C.byref(st))
+    lib().oracle_kv_copy_pairs(C.byref(mm), T, a, NB_src, src_order,
+                               C.c_int64(pool_elems_per_layer(m, T, a, NB_src)), _ptr_array(src_pools), b, NB_dst,
+                               dst_order, C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)), _ptr_array(dst_pools),
+                               prp, int(num_pairs), C.byref(st))
     return st.value
 
 

@@ -15,6 +15,9 @@
  *     With grouped-query attention (Sec. 2.1 footnote) H is the number of K/V heads.
  *   - Header-centric KV layout (Sec. 3.1, "Improvement 1"): storage order [Block, Header, K/V, Token]; the
  *     head dimension is innermost and every layer has its own array of blocks (the paper omits both).
+ *   - Token-first KV layout (Sec. 3.1: the layout of mainstream engines, the paper's starting point): K and V each
+ *     occupy one contiguous region of the layer's pool, and inside a region a token's headers are stored together:
+ *     order [K/V, Block, Token, Header], head dimension innermost.
  *   - FFN partition (Sec. 3.2, Eq. 1): up_proj split column-wise, down_proj split row-wise in the paper's
  *     [in,out] algebra FFN = f(I x U) x D.  Weights are stored [out,in] row-major here, so the paper's columns
  *     of U are rows of up/gate (contiguous) and the paper's rows of D are columns of down (strided).
@@ -39,6 +42,15 @@ typedef struct {
 } oracle_model;
 
 enum { ORACLE_OK = 0, ORACLE_INVALID_ARG = 1, ORACLE_NO_FREE_BLOCKS = 4, ORACLE_BAD_BLOCK_ID = 5 };
+enum { ORACLE_HEADER_CENTRIC = 0, ORACLE_TOKEN_FIRST = 1 };
+
+/* Element offset inside one layer of a worker's pool (NB blocks, Hs headers per worker, T tokens per block). */
+static int64_t pool_offset(int order, int64_t NB, int Hs, int T, int D, int64_t blk, int hl, int c, int tok, int d) {
+    if (order == ORACLE_TOKEN_FIRST) /* [K/V][Block][Token][Header][dim] */
+        return ((((int64_t)c * NB + blk) * T + tok) * Hs + hl) * (int64_t)D + d;
+    /* [Block][Header][K/V][Token][dim] */
+    return ((((blk * Hs + hl) * 2 + c) * T + tok) * (int64_t)D) + d;
+}
 
 /* ---- Sec. 3.1: which headers worker W_i keeps (1-indexed, inclusive range) ---- */
 void oracle_header_range(int H, int TP, int i, int* first, int* last) {
@@ -71,11 +83,12 @@ int64_t oracle_padded_tokens(int S, const int32_t* seq_lens, int T) { return tok
  * Logical KV: KV[l][g][h][c][d]; g = padded global token (sequence s, token t -> token_base(s) + t, every
  * sequence rounded up to whole blocks, slack tokens included), h = K/V head 0..Hkv-1, c = 0 (K) / 1 (V).
  * Pool of worker r (0-indexed pointer array, worker r+1 in the paper's numbering):
- *   pool[r][l*layer_stride + ((((blk*Hs + hl)*2 + c)*T + tok)*D + d)],  Hs = Hkv/TP headers per worker.
+ *   pool[r][l*layer_stride + pool_offset(order, ...)],  Hs = Hkv/TP headers per worker, NB blocks per layer.
  * dir = 0: logical -> pools (shard).  dir = 1: pools -> logical (reconstruct).
  */
-static void kv_walk(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
-                    const int32_t* seq_lens, const int32_t* bt, int maxb, uint16_t* const* pools, int dir) {
+static void kv_walk(uint16_t* KV, const oracle_model* m, int T, int TP, int NB, int order,
+                    int64_t layer_stride_elems, int S, const int32_t* seq_lens, const int32_t* bt, int maxb,
+                    uint16_t* const* pools, int dir) {
     const int Hs = m->Hkv / TP;
     const int64_t G = token_base(seq_lens, S, T);
 #pragma omp parallel for schedule(static)
@@ -95,7 +108,7 @@ static void kv_walk(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t 
                     for (int c = 0; c < 2; ++c) {
                         for (int d = 0; d < m->D; ++d) {
                             const int64_t lo = ((((int64_t)l * G + g0 + t) * m->Hkv + (header - 1)) * 2 + c) * m->D + d;
-                            const int64_t po = ((((blk * Hs + hl) * 2 + c) * T + tok) * (int64_t)m->D) + d;
+                            const int64_t po = pool_offset(order, NB, Hs, T, m->D, blk, hl, c, tok, d);
                             if (dir == 0) pool[po] = KV[lo];
                             else KV[lo] = pool[po];
                         }
@@ -106,26 +119,29 @@ static void kv_walk(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t 
     }
 }
 
-void oracle_kv_shard(const uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
-                     const int32_t* seq_lens, const int32_t* bt, int maxb, uint16_t* const* pools) {
-    kv_walk((uint16_t*)KV, m, T, TP, layer_stride_elems, S, seq_lens, bt, maxb, pools, 0);
+void oracle_kv_shard(const uint16_t* KV, const oracle_model* m, int T, int TP, int NB, int order,
+                     int64_t layer_stride_elems, int S, const int32_t* seq_lens, const int32_t* bt, int maxb,
+                     uint16_t* const* pools) {
+    kv_walk((uint16_t*)KV, m, T, TP, NB, order, layer_stride_elems, S, seq_lens, bt, maxb, pools, 0);
 }
 
-void oracle_kv_reconstruct(uint16_t* KV, const oracle_model* m, int T, int TP, int64_t layer_stride_elems, int S,
-                           const int32_t* seq_lens, const int32_t* bt, int maxb, const uint16_t* const* pools) {
-    kv_walk(KV, m, T, TP, layer_stride_elems, S, seq_lens, bt, maxb, (uint16_t* const*)pools, 1);
+void oracle_kv_reconstruct(uint16_t* KV, const oracle_model* m, int T, int TP, int NB, int order,
+                           int64_t layer_stride_elems, int S, const int32_t* seq_lens, const int32_t* bt, int maxb,
+                           const uint16_t* const* pools) {
+    kv_walk(KV, m, T, TP, NB, order, layer_stride_elems, S, seq_lens, bt, maxb, (uint16_t* const*)pools, 1);
 }
 
 /* TP a -> b on the KV cache: un-shard the TP=a pools into the logical array, shard that for TP=b. */
-int oracle_kv_transform(const oracle_model* m, int T, int S, const int32_t* seq_lens, int maxb, int a,
-                        int64_t src_layer_stride, const int32_t* src_bt, const uint16_t* const* src_pools, int b,
-                        int64_t dst_layer_stride, const int32_t* dst_bt, uint16_t* const* dst_pools) {
+int oracle_kv_transform(const oracle_model* m, int T, int S, const int32_t* seq_lens, int maxb, int a, int NB_src,
+                        int src_order, int64_t src_layer_stride, const int32_t* src_bt,
+                        const uint16_t* const* src_pools, int b, int NB_dst, int dst_order, int64_t dst_layer_stride,
+                        const int32_t* dst_bt, uint16_t* const* dst_pools) {
     const int64_t G = token_base(seq_lens, S, T);
     const int64_t n = (int64_t)m->L * G * m->Hkv * 2 * m->D;
     uint16_t* KV = (uint16_t*)malloc((size_t)(n > 0 ? n : 1) * sizeof(uint16_t));
     if (!KV) return ORACLE_INVALID_ARG;
-    oracle_kv_reconstruct(KV, m, T, a, src_layer_stride, S, seq_lens, src_bt, maxb, src_pools);
-    oracle_kv_shard(KV, m, T, b, dst_layer_stride, S, seq_lens, dst_bt, maxb, dst_pools);
+    oracle_kv_reconstruct(KV, m, T, a, NB_src, src_order, src_layer_stride, S, seq_lens, src_bt, maxb, src_pools);
+    oracle_kv_shard(KV, m, T, b, NB_dst, dst_order, dst_layer_stride, S, seq_lens, dst_bt, maxb, dst_pools);
     free(KV);
     return ORACLE_OK;
 }
@@ -283,9 +299,10 @@ void oracle_assign_blocks(int S, const int32_t* seq_lens, int T, const int32_t* 
  * (skipped) or a block id is out of range (skipped, BAD_BLOCK_ID).  Element loops through the logical
  * coordinates (header -> source worker / destination worker), no run copies.
  */
-void oracle_kv_copy_pairs(const oracle_model* m, int T, int a, int NB_src, int64_t src_layer_stride,
-                          const uint16_t* const* src_pools, int b, int NB_dst, int64_t dst_layer_stride,
-                          uint16_t* const* dst_pools, const int32_t* pairs, int num_pairs, int32_t* status) {
+void oracle_kv_copy_pairs(const oracle_model* m, int T, int a, int NB_src, int src_order, int64_t src_layer_stride,
+                          const uint16_t* const* src_pools, int b, int NB_dst, int dst_order,
+                          int64_t dst_layer_stride, uint16_t* const* dst_pools, const int32_t* pairs, int num_pairs,
+                          int32_t* status) {
     const int Ha = m->Hkv / a, Hb = m->Hkv / b;
     for (int k = 0; k < num_pairs; ++k) {
         const int64_t p = pairs[2 * k], q = pairs[2 * k + 1];
@@ -306,8 +323,8 @@ void oracle_kv_copy_pairs(const oracle_model* m, int T, int a, int NB_src, int64
                 for (int c = 0; c < 2; ++c)
                     for (int tok = 0; tok < T; ++tok)
                         for (int d = 0; d < m->D; ++d)
-                            dp[((((q * Hb + (header - fb)) * 2 + c) * T + tok) * (int64_t)m->D) + d] =
-                                sp[((((p * Ha + (header - fa)) * 2 + c) * T + tok) * (int64_t)m->D) + d];
+                            dp[pool_offset(dst_order, NB_dst, Hb, T, m->D, q, header - fb, c, tok, d)] =
+                                sp[pool_offset(src_order, NB_src, Ha, T, m->D, p, header - fa, c, tok, d)];
             }
     }
 }

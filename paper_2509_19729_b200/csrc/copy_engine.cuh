@@ -2,12 +2,16 @@
 //
 // A work item is a small 2-D copy: n_rows runs of row_bytes bytes, run i read at src + i*src_pitch and written at
 // dst + i*dst_pitch (n_rows == 1 is a plain contiguous chunk).  All addresses, pitches and row_bytes are
-// multiples of 16 bytes.  Two ways to move an item:
-//   * cta_copy_item:    every thread of the CTA moves 16-byte vectors, all loads of an unrolled batch issued
-//                       before the first store, streaming cache hints;
-//   * WarpBulkRing:     one warp drives a ring of shared-memory stages with the bulk-copy engine (TMA, 1-D
-//                       cp.async.bulk, no multicast): global -> shared completes on an mbarrier, shared -> global is
-//                       tracked by the issuing thread's bulk groups.  Every wait is bounded.
+// multiples of 16 bytes.  Three ways to move items:
+//   * cta_copy_item      every thread of the CTA moves 16-byte vectors, all loads of an unrolled batch issued
+//                        before the first store, streaming cache hints;
+//   * warp_bulk_ring     each warp drives its own ring of shared-memory stages with the bulk-copy engine (TMA, 1-D
+//                        cp.async.bulk, no multicast): global -> shared completes on an mbarrier, shared -> global is
+//                        tracked by the issuing thread's bulk groups; loads lead stores by a fixed lag;
+//   * pair_bulk_ring     a producer warp and a consumer warp share one ring: the producer only issues loads (waits
+//                        on "empty" barriers), the consumer only issues stores (waits on "full" barriers), so the
+//                        split of the ring between loads and stores in flight adapts by itself.
+// Every wait on an mbarrier is bounded; bulk-group waits only wait for the thread's own stores.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -19,6 +23,14 @@ struct Item {
     char* dst;
     int64_t src_pitch, dst_pitch;
     int32_t n_rows, row_bytes;
+};
+
+// Shape of the bulk rings (runtime, chosen by the launcher).
+struct RingShape {
+    int32_t stages;       // stages per ring
+    int32_t lag;          // warp ring: loads lead stores by this many items; pair ring: stores kept in flight
+    int32_t stage_bytes;  // bytes per stage
+    int32_t hint;         // bit 0: loads evict-first in L2, bit 1: stores evict-first in L2
 };
 
 // ------------------------------------------------------------------ vector load/store path
@@ -64,7 +76,7 @@ __device__ __forceinline__ void cta_copy_item(const Item& it) {
     }
 }
 
-// ------------------------------------------------------------------ bulk-copy (TMA) path
+// ------------------------------------------------------------------ bulk-copy (TMA) primitives
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -73,6 +85,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -91,32 +106,72 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(smem_dst)),
-                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
 }
-__device__ __forceinline__ void bulk_s2g(void* gdst, const void* smem_src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)),
-                 "r"(bytes)
-                 : "memory");
+__device__ __forceinline__ void bulk_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar, bool hint,
+                                         uint64_t policy) {
+    if (hint)
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                smem_u32(smem_dst)),
+            "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+            : "memory");
+    else
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_u32(smem_dst)),
+                     "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                     : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* gdst, const void* smem_src, uint32_t bytes, bool hint, uint64_t policy) {
+    if (hint)
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
+                     "r"(smem_u32(smem_src)), "r"(bytes), "l"(policy)
+                     : "memory");
+    else
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                     "r"(smem_u32(smem_src)), "r"(bytes)
+                     : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+// Wait until at most n of this thread's bulk groups still have shared-memory reads outstanding (n in 0..15).
+__device__ __forceinline__ void bulk_wait_read(int n) {
+    switch (n) {
+        case 0: asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.bulk.wait_group.read 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.bulk.wait_group.read 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.bulk.wait_group.read 6;" ::: "memory"); break;
+        case 7: asm volatile("cp.async.bulk.wait_group.read 7;" ::: "memory"); break;
+        case 8: asm volatile("cp.async.bulk.wait_group.read 8;" ::: "memory"); break;
+        case 9: asm volatile("cp.async.bulk.wait_group.read 9;" ::: "memory"); break;
+        case 10: asm volatile("cp.async.bulk.wait_group.read 10;" ::: "memory"); break;
+        case 11: asm volatile("cp.async.bulk.wait_group.read 11;" ::: "memory"); break;
+        case 12: asm volatile("cp.async.bulk.wait_group.read 12;" ::: "memory"); break;
+        case 13: asm volatile("cp.async.bulk.wait_group.read 13;" ::: "memory"); break;
+        case 14: asm volatile("cp.async.bulk.wait_group.read 14;" ::: "memory"); break;
+        default: asm volatile("cp.async.bulk.wait_group.read 15;" ::: "memory"); break;
+    }
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// One warp's ring of NS shared-memory stages.  Loads run LAG items ahead of stores, so up to LAG loads and
-// NS - LAG stores are in flight per warp.  `item_of(w)` must return the same Item in every lane.
+constexpr int kMaxStages = 16;
+
+// ------------------------------------------------------------------ one ring per warp
+// Loads run `lag` items ahead of stores, so up to `lag` loads and `stages - lag` stores are in flight per warp.
+// `item_of(w)` must return the same Item in every lane.  bars: `stages` mbarriers of this warp.
 // Returns false if a bounded wait ran out (the caller records AMOEBA_ERR_TIMEOUT).
-template <int NS, int LAG, class ItemFn>
+template <class ItemFn>
 __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, int64_t first, int64_t stride,
-                                               char* stages, int stage_bytes, uint64_t* bars) {
-    static_assert(LAG >= 1 && LAG < NS, "loads must lead stores by 1..NS-1 stages");
+                                               char* stages, uint64_t* bars, const RingShape rs) {
     const int lane = threadIdx.x & 31;
+    const int NS = rs.stages, LAG = rs.lag;
+    const bool hl = rs.hint & 1, hs = rs.hint & 2;
+    const uint64_t policy = policy_evict_first();
     if (lane == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(&bars[s], 1);
         fence_async_smem();
@@ -125,38 +180,115 @@ __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, 
     const int64_t n_local = n_items > first ? (n_items - first + stride - 1) / stride : 0;
     bool ok = true;
     int64_t loads_issued = 0, loads_waited = 0;
+    int s_load = 0, s_store = 0;       // ring slots of the next load / next store
+    uint32_t store_parity = 0;         // phase parity of the slot the next store waits on
     for (int64_t k = 0; k < n_local + LAG && ok; ++k) {
         if (k < n_local) {
-            const int s = (int)(k % NS);
-            if (k >= NS) bulk_wait_read<NS - LAG - 1>();  // this lane's stores out of stage s have read it
-            __syncwarp();                                 // ... and so have every other lane's
+            if (k >= NS) bulk_wait_read(NS - LAG - 1);  // this lane's stores out of this slot have read it
+            __syncwarp();                               // ... and so have every other lane's
             const Item it = item_of(first + k * stride);
-            if (lane == 0) mbar_arrive_expect_tx(&bars[s], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
+            if (lane == 0) mbar_arrive_expect_tx(&bars[s_load], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
             __syncwarp();
-            char* st = stages + (int64_t)s * stage_bytes;
+            char* st = stages + (int64_t)s_load * rs.stage_bytes;
             for (int r = lane; r < it.n_rows; r += 32)
-                bulk_g2s(st + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, &bars[s]);
+                bulk_g2s(st + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, &bars[s_load], hl,
+                         policy);
             ++loads_issued;
+            if (++s_load == NS) s_load = 0;
         }
-        const int64_t j = k - LAG;
-        if (j >= 0) {
-            const int s = (int)(j % NS);
-            ok = mbar_wait_bounded(&bars[s], (uint32_t)((j / NS) & 1));
+        if (k >= LAG) {
+            ok = mbar_wait_bounded(&bars[s_store], store_parity);
             ok = __all_sync(0xffffffffu, ok);
-            ++loads_waited;
             if (ok) {
-                const Item it = item_of(first + j * stride);
-                const char* st = stages + (int64_t)s * stage_bytes;
+                ++loads_waited;
+                const Item it = item_of(first + (k - LAG) * stride);
+                const char* st = stages + (int64_t)s_store * rs.stage_bytes;
                 for (int r = lane; r < it.n_rows; r += 32)
-                    bulk_s2g(it.dst + r * it.dst_pitch, st + (int64_t)r * it.row_bytes, it.row_bytes);
+                    bulk_s2g(it.dst + r * it.dst_pitch, st + (int64_t)r * it.row_bytes, it.row_bytes, hs, policy);
             }
             bulk_commit();
+            if (++s_store == NS) {
+                s_store = 0;
+                store_parity ^= 1;
+            }
         }
     }
-    bulk_wait_all();  // this lane's stores are complete and visible
+    bulk_wait_all();  // this lane's stores are complete
     if (!ok) {        // give the loads still in flight a bounded chance to land before the CTA's smem goes away
         for (int64_t j = loads_waited; j < loads_issued; ++j)
             mbar_wait_bounded(&bars[j % NS], (uint32_t)((j / NS) & 1), 1u << 16);
+    }
+    __syncwarp();
+    return ok;
+}
+
+// ------------------------------------------------------------------ producer warp + consumer warp on one ring
+// `role` 0 = producer (loads), 1 = consumer (stores).  full/empty: `stages` mbarriers each, initialised by
+// pair_ring_init before both warps start.  rs.lag = number of store groups the consumer keeps in flight before it
+// hands a slot back.
+__device__ __forceinline__ void pair_ring_init(uint64_t* full, uint64_t* empty, int stages) {
+    for (int s = 0; s < stages; ++s) {
+        mbar_init(&full[s], 1);
+        mbar_init(&empty[s], 1);
+    }
+    fence_async_smem();
+}
+
+template <class ItemFn>
+__device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t n_items, int64_t first,
+                                               int64_t stride, char* stages, uint64_t* full, uint64_t* empty,
+                                               const RingShape rs) {
+    const int lane = threadIdx.x & 31;
+    const int NS = rs.stages, D = rs.lag;
+    const uint64_t policy = policy_evict_first();
+    const int64_t n_local = n_items > first ? (n_items - first + stride - 1) / stride : 0;
+    bool ok = true;
+    int slot = 0;
+    uint32_t parity = 0;
+    if (role == 0) {
+        const bool hl = rs.hint & 1;
+        for (int64_t k = 0; k < n_local && ok; ++k) {
+            if (k >= NS) {  // wait until the consumer has handed this slot back (its previous use)
+                ok = mbar_wait_bounded(&empty[slot], parity ^ 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
+            const Item it = item_of(first + k * stride);
+            if (lane == 0) mbar_arrive_expect_tx(&full[slot], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
+            __syncwarp();
+            char* st = stages + (int64_t)slot * rs.stage_bytes;
+            for (int r = lane; r < it.n_rows; r += 32)
+                bulk_g2s(st + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, &full[slot], hl,
+                         policy);
+            if (++slot == NS) {
+                slot = 0;
+                parity ^= 1;
+            }
+        }
+    } else {
+        const bool hs = rs.hint & 2;
+        int release = 0;  // slot of the oldest store not yet handed back
+        for (int64_t k = 0; k < n_local && ok; ++k) {
+            ok = mbar_wait_bounded(&full[slot], parity);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const Item it = item_of(first + k * stride);
+            const char* st = stages + (int64_t)slot * rs.stage_bytes;
+            for (int r = lane; r < it.n_rows; r += 32)
+                bulk_s2g(it.dst + r * it.dst_pitch, st + (int64_t)r * it.row_bytes, it.row_bytes, hs, policy);
+            bulk_commit();
+            if (k >= D) {  // the store issued D items ago has read its slot: hand it back
+                bulk_wait_read(D);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[release]);
+                if (++release == NS) release = 0;
+            }
+            if (++slot == NS) {
+                slot = 0;
+                parity ^= 1;
+            }
+        }
+        bulk_wait_all();
     }
     __syncwarp();
     return ok;

@@ -83,26 +83,31 @@ __global__ void __launch_bounds__(256) kv_reshard_ldst(const __grid_constant__ K
     }
 }
 
-template <int NS, int LAG>
-__global__ void __launch_bounds__(1024) kv_reshard_bulk(const __grid_constant__ KvParams p, int stage_bytes) {
+// Dynamic shared memory: [kBarrierBytes of mbarriers][rings x stages x stage_bytes].
+__global__ void __launch_bounds__(1024) kv_reshard_bulk(const __grid_constant__ KvParams p, const RingShape rs) {
     extern __shared__ __align__(128) char smem[];
     const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * NS;
-    char* stages = smem + 1024 + (int64_t)warp * NS * stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)warp * rs.stages * rs.stage_bytes;
     const KvItems items{p, clamp_pairs(p)};
-    const bool ok = warp_bulk_ring<NS, LAG>(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
-                                            (int64_t)gridDim.x * nwarps, stages, stage_bytes, bars);
+    const bool ok = warp_bulk_ring(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
+                                   (int64_t)gridDim.x * nwarps, stages, bars, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
-template <int NS, int LAG>
-static cudaError_t launch_bulk(const KvParams& p, int grid, int warps, int stage_bytes, cudaStream_t stream) {
-    const size_t smem = 1024 + (size_t)warps * NS * stage_bytes;
-    cudaError_t e = cudaFuncSetAttribute(kv_reshard_bulk<NS, LAG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    kv_reshard_bulk<NS, LAG><<<grid, warps * 32, smem, stream>>>(p, stage_bytes);
-    return cudaGetLastError();
+// Warps 2r and 2r+1 are the producer and the consumer of ring r.
+__global__ void __launch_bounds__(1024) kv_reshard_pair(const __grid_constant__ KvParams p, const RingShape rs) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
+    uint64_t* empty = full + rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
+    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
+    __syncthreads();
+    const KvItems items{p, clamp_pairs(p)};
+    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
+                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
 }  // namespace amoeba
@@ -153,21 +158,21 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t max_items = (int64_t)pairs_cap * p.n_layers * p.runs_per_block * p.chunks_per_run;
     cudaError_t e;
-    const int path = plan->opt.copy_path ? plan->opt.copy_path : kDefaultCopyPath;
+    const KernelOpts& opt = plan->opt.kv;
+    const int path = opt.copy_path ? opt.copy_path : kKvDefaults.copy_path;
     if (path == 1) {
-        const int per_sm = plan->opt.ctas_per_sm ? plan->opt.ctas_per_sm : 8;
+        const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 16;
         const int grid = (int)std::min<int64_t>(max_items, (int64_t)dev.sms * per_sm);
         kv_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
         e = cudaGetLastError();
     } else {
-        const BulkShape bs = bulk_shape(dev, plan->opt, (int)plan->chunk_bytes);
-        const int grid = (int)std::min<int64_t>((max_items + bs.warps - 1) / bs.warps, (int64_t)dev.sms * bs.ctas_per_sm);
-        switch (bs.stages) {
-            case 2: e = launch_bulk<2, 1>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
-            case 3: e = launch_bulk<3, 2>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
-            case 4: e = launch_bulk<4, 2>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
-            case 6: e = launch_bulk<6, 3>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
-            default: e = launch_bulk<8, 4>(p, grid, bs.warps, (int)plan->chunk_bytes, stream); break;
+        const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)plan->chunk_bytes);
+        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+        auto kernel = path == 3 ? kv_reshard_pair : kv_reshard_bulk;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+        if (e == cudaSuccess) {
+            kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring);
+            e = cudaGetLastError();
         }
     }
     if (e != cudaSuccess) return AMOEBA_ERR_CUDA;

@@ -3,18 +3,26 @@
 #include <algorithm>
 #include <cuda_runtime.h>
 
+#include "copy_engine.cuh"
 #include "plan.hpp"
 
 namespace amoeba {
 
-constexpr int kDefaultCopyPath = 2;  // 1 = vector ld/st, 2 = bulk-copy ring (chosen from measurements)
+// Defaults, chosen from sweeps over all benchmark configurations on B200: the producer/consumer ring, 8 KiB work
+// items, 5 rings of 4 stages per CTA (160 KiB of stages per SM - more in flight lowers DRAM efficiency, less starves
+// it), two stores in flight before a slot is handed back, both directions marked evict-first in L2.
+struct KernelDefaults {
+    int copy_path, stages, lag, warps, hint;
+};
+constexpr KernelDefaults kKvDefaults{3, 4, 2, 5, 4};
+constexpr KernelDefaults kWDefaults{3, 4, 2, 5, 4};
 
 struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;  // bytes of dynamic shared memory one CTA may opt in to
 };
 
-// Properties of the current device (two attribute queries; no allocation, no synchronisation).
+// Properties of the current device (attribute queries; no allocation, no synchronisation).
 inline bool device_info(DeviceInfo* out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
@@ -24,20 +32,43 @@ inline bool device_info(DeviceInfo* out) {
     return out->sms > 0;
 }
 
+constexpr int kBarrierBytes = 1024;  // head of dynamic shared memory: up to 128 mbarriers
+
 struct BulkShape {
-    int stages, warps, ctas_per_sm;
+    RingShape ring;
+    int path;         // 2 = ring per warp, 3 = producer/consumer pair per ring
+    int rings;        // rings per CTA
+    int threads;      // CTA size
+    int ctas_per_sm;
+    size_t smem;
 };
 
-// Ring depth and warps per CTA for the bulk-copy kernels: as many independent warp rings as fit in shared memory.
-inline BulkShape bulk_shape(const DeviceInfo& dev, const Options& opt, int stage_bytes) {
-    BulkShape s;
-    s.stages = opt.stages ? opt.stages : 4;
-    if (s.stages != 2 && s.stages != 3 && s.stages != 4 && s.stages != 6 && s.stages != 8) s.stages = 4;
-    s.ctas_per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 1;
-    const int budget = (dev.smem_optin - 1024 * s.ctas_per_sm) / s.ctas_per_sm - 1024;
-    while (s.stages > 2 && (int64_t)s.stages * stage_bytes > budget) s.stages = s.stages == 3 ? 2 : s.stages == 4 ? 3 : s.stages == 6 ? 4 : 6;
-    s.warps = (int)std::max<int64_t>(1, std::min<int64_t>(16, budget / ((int64_t)s.stages * stage_bytes)));
-    return s;
+// Ring depth, lag and rings per CTA for the bulk-copy kernels: the requested shape, shrunk until it fits the
+// shared memory one CTA may use and the barrier area.
+inline BulkShape bulk_shape(const DeviceInfo& dev, const KernelOpts& opt, const KernelDefaults& def, int path,
+                            int stage_bytes) {
+    BulkShape b;
+    b.path = path;
+    b.ctas_per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 1;
+    int stages = std::min(kMaxStages, std::max(2, opt.stages ? opt.stages : def.stages));
+    const int budget = dev.smem_optin / b.ctas_per_sm - kBarrierBytes - (b.ctas_per_sm > 1 ? 1024 : 0);
+    while (stages > 2 && (int64_t)stages * stage_bytes > budget) --stages;
+    int lag = opt.lag ? opt.lag : (opt.stages ? stages / 2 : def.lag);
+    lag = std::max(1, std::min(lag, stages - 1));
+    const int bars_per_ring = path == 3 ? 2 * stages : stages;
+    int rings = opt.warps ? opt.warps : def.warps;
+    rings = (int)std::min<int64_t>(rings, budget / ((int64_t)stages * stage_bytes));
+    rings = std::min(rings, kBarrierBytes / 8 / bars_per_ring);
+    rings = std::max(1, std::min(rings, path == 3 ? 16 : 32));
+    b.rings = rings;
+    b.threads = 32 * rings * (path == 3 ? 2 : 1);
+    b.ring.stages = stages;
+    b.ring.lag = lag;
+    b.ring.stage_bytes = stage_bytes;
+    const int hint = opt.hint ? opt.hint : (def.hint ? def.hint : 1);
+    b.ring.hint = hint - 1;
+    b.smem = kBarrierBytes + (size_t)rings * stages * stage_bytes;
+    return b;
 }
 
 }  // namespace amoeba

@@ -43,9 +43,10 @@ static int64_t chunk_of(int64_t total, int64_t cap) {
 }
 
 amoeba_status finalize_chunks(amoeba_plan* p) {
-    const int64_t cap = p->opt.chunk_bytes > 0 ? p->opt.chunk_bytes : 16384;
-    if (cap < 16 || cap % 16) return AMOEBA_ERR_INVALID_ARG;
-    p->chunk_bytes = chunk_of(p->run_bytes, cap);
+    const int64_t kv_cap = p->opt.kv.chunk_bytes > 0 ? p->opt.kv.chunk_bytes : kDefaultKvChunk;
+    const int64_t cap = p->opt.w.chunk_bytes > 0 ? p->opt.w.chunk_bytes : kDefaultWChunk;
+    if (cap < 16 || cap % 16 || kv_cap < 16 || kv_cap % 16) return AMOEBA_ERR_INVALID_ARG;
+    p->chunk_bytes = chunk_of(p->run_bytes, kv_cap);
     p->wdev.clear();
     int64_t item = 0;
     for (const amoeba_weight_desc& d : p->wdescs) {
@@ -207,9 +208,9 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
         p->weight_bytes_per_layer += d.row_bytes * d.n_rows;
     }
 
-    if (const char* env = std::getenv("AMOEBA_COPY_PATH")) {
-        if (env[0] == 'l') p->opt.copy_path = 1;
-        if (env[0] == 't') p->opt.copy_path = 2;
+    if (const char* env = std::getenv("AMOEBA_COPY_PATH")) {  // "ldst", "bulk" (ring per warp), "pair"
+        const int path = env[0] == 'l' ? 1 : env[0] == 'b' || env[0] == 't' ? 2 : env[0] == 'p' ? 3 : 0;
+        p->opt.kv.copy_path = p->opt.w.copy_path = path;
     }
     st = finalize_chunks(p);
     if (st != AMOEBA_OK) {
@@ -283,27 +284,46 @@ amoeba_status amoeba_plan_weight_desc(const amoeba_plan* plan, int32_t index, am
 }
 
 amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t value) {
-    if (!plan || value < 0) return AMOEBA_ERR_INVALID_ARG;
-    Options old = plan->opt;
-    switch (option) {
-        case AMOEBA_OPT_COPY_PATH:
-            if (value > 2) return AMOEBA_ERR_INVALID_ARG;
-            plan->opt.copy_path = (int)value;
-            break;
-        case AMOEBA_OPT_CTAS_PER_SM:
-            if (value > 32) return AMOEBA_ERR_INVALID_ARG;
-            plan->opt.ctas_per_sm = (int)value;
-            break;
-        case AMOEBA_OPT_CHUNK_BYTES:
-            if (value > 65536) return AMOEBA_ERR_INVALID_ARG;
-            plan->opt.chunk_bytes = value;
-            break;
-        case AMOEBA_OPT_STAGES:
-            if (value > 16) return AMOEBA_ERR_INVALID_ARG;
-            plan->opt.stages = (int)value;
-            break;
-        default:
-            return AMOEBA_ERR_INVALID_ARG;
+    if (!plan || value < 0 || option < 0) return AMOEBA_ERR_INVALID_ARG;
+    const Options old = plan->opt;
+    const int which = option / AMOEBA_OPT_WEIGHTS_ONLY;  // 0 both kernels, 1 weights only, 2 KV only
+    const int id = option % AMOEBA_OPT_WEIGHTS_ONLY;
+    if (which > 2) return AMOEBA_ERR_INVALID_ARG;
+    KernelOpts* targets[2] = {which != 1 ? &plan->opt.kv : nullptr, which != 2 ? &plan->opt.w : nullptr};
+    for (KernelOpts* k : targets) {
+        if (!k) continue;
+        switch (id) {
+            case AMOEBA_OPT_COPY_PATH:
+                if (value > 3) return AMOEBA_ERR_INVALID_ARG;
+                k->copy_path = (int)value;
+                break;
+            case AMOEBA_OPT_CTAS_PER_SM:
+                if (value > 32) return AMOEBA_ERR_INVALID_ARG;
+                k->ctas_per_sm = (int)value;
+                break;
+            case AMOEBA_OPT_CHUNK_BYTES:
+                if (value > 65536) return AMOEBA_ERR_INVALID_ARG;
+                k->chunk_bytes = value;
+                break;
+            case AMOEBA_OPT_STAGES:
+                if (value > 16) return AMOEBA_ERR_INVALID_ARG;
+                k->stages = (int)value;
+                break;
+            case AMOEBA_OPT_LAG:
+                if (value > 15) return AMOEBA_ERR_INVALID_ARG;
+                k->lag = (int)value;
+                break;
+            case AMOEBA_OPT_WARPS:
+                if (value > 16) return AMOEBA_ERR_INVALID_ARG;
+                k->warps = (int)value;
+                break;
+            case AMOEBA_OPT_L2_HINT:
+                if (value > 4) return AMOEBA_ERR_INVALID_ARG;
+                k->hint = (int)value;
+                break;
+            default:
+                return AMOEBA_ERR_INVALID_ARG;
+        }
     }
     amoeba_status st = finalize_chunks(plan);
     if (st != AMOEBA_OK) {

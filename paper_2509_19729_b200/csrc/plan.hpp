@@ -10,6 +10,8 @@ namespace amoeba {
 constexpr int kNumTensors = 7;  // q,k,v,o,gate,up,down
 constexpr int kMaxWeightDescs = 160;
 constexpr int kMaxWeightPtrs = 2048;  // per launch: layers * (a + b) * kNumTensors pointers
+constexpr int64_t kDefaultKvChunk = 8192;   // upper bound of one KV copy work item
+constexpr int64_t kDefaultWChunk = 8192;    // upper bound of one weight copy work item
 
 // One weight copy descriptor as the kernels see it (per layer, relative to that layer's buffers).
 struct WDescDev {
@@ -25,11 +27,19 @@ struct WDescDev {
     int32_t pad;
 };
 
-struct Options {
-    int copy_path = 0;    // 0 default, 1 vector ld/st, 2 bulk-copy ring
-    int ctas_per_sm = 0;  // 0 default
+// Tuning knobs of one copy kernel; 0 = use the kernel's default.
+struct KernelOpts {
+    int copy_path = 0;    // 1 vector ld/st, 2 bulk-copy ring per warp, 3 bulk-copy producer/consumer ring
+    int ctas_per_sm = 0;
     int64_t chunk_bytes = 0;
-    int stages = 0;
+    int stages = 0;       // ring depth
+    int lag = 0;          // loads ahead of stores (path 2) / stores kept in flight (path 3)
+    int warps = 0;        // rings per CTA
+    int hint = 0;         // 1 + bit mask: bit 0 loads evict-first, bit 1 stores evict-first (0 = default)
+};
+
+struct Options {
+    KernelOpts kv, w;
 };
 
 }  // namespace amoeba
@@ -40,7 +50,7 @@ struct amoeba_plan {
     int32_t heads_src, heads_dst;  // K/V headers per source / destination worker
     int32_t heads_per_run, runs_per_block;
     int64_t unit_bytes;  // one (block, header): 2 * T * D * e
-    int64_t run_bytes, chunk_bytes;
+    int64_t run_bytes, chunk_bytes;  // chunk_bytes: KV work item
     int64_t src_block_bytes, dst_block_bytes, src_layer_stride, dst_layer_stride;
     // weights
     std::vector<amoeba_weight_desc> wdescs;  // public form

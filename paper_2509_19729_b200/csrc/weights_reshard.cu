@@ -54,28 +54,31 @@ __global__ void __launch_bounds__(256) w_reshard_ldst(const __grid_constant__ WP
     for (int64_t w = blockIdx.x; w < n; w += gridDim.x) cta_copy_item<UNROLL>(items(w));
 }
 
-template <int NS, int LAG>
-__global__ void __launch_bounds__(1024) w_reshard_bulk(const __grid_constant__ WParams p, int stage_bytes,
+__global__ void __launch_bounds__(1024) w_reshard_bulk(const __grid_constant__ WParams p, const RingShape rs,
                                                         int32_t* status) {
     extern __shared__ __align__(128) char smem[];
     const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * NS;
-    char* stages = smem + 1024 + (int64_t)warp * NS * stage_bytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)warp * rs.stages * rs.stage_bytes;
     const WItems items{p};
-    const bool ok = warp_bulk_ring<NS, LAG>(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
-                                            (int64_t)gridDim.x * nwarps, stages, stage_bytes, bars);
+    const bool ok = warp_bulk_ring(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
+                                   (int64_t)gridDim.x * nwarps, stages, bars, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
-template <int NS, int LAG>
-static cudaError_t launch_bulk(const WParams& p, int grid, int warps, int stage_bytes, int32_t* status,
-                               cudaStream_t stream) {
-    const size_t smem = 1024 + (size_t)warps * NS * stage_bytes;
-    cudaError_t e = cudaFuncSetAttribute(w_reshard_bulk<NS, LAG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    w_reshard_bulk<NS, LAG><<<grid, warps * 32, smem, stream>>>(p, stage_bytes, status);
-    return cudaGetLastError();
+__global__ void __launch_bounds__(1024) w_reshard_pair(const __grid_constant__ WParams p, const RingShape rs,
+                                                        int32_t* status) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
+    uint64_t* empty = full + rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
+    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
+    __syncthreads();
+    const WItems items{p};
+    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
+                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
 static void* const* slots(const amoeba_layer_weights* w) { return reinterpret_cast<void* const*>(w); }
@@ -105,7 +108,8 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
     DeviceInfo dev;
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int path = plan->opt.copy_path ? plan->opt.copy_path : kDefaultCopyPath;
+    const KernelOpts& opt = plan->opt.w;
+    const int path = opt.copy_path ? opt.copy_path : kWDefaults.copy_path;
     int stage_bytes = 16;
     for (const WDescDev& d : plan->wdev)
         stage_bytes = std::max<int64_t>(stage_bytes, (int64_t)d.rows_per_item * d.chunk_bytes);
@@ -132,19 +136,18 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
         const int64_t n_items = (int64_t)p.items_per_layer * nl;
         cudaError_t e;
         if (path == 1) {
-            const int per_sm = plan->opt.ctas_per_sm ? plan->opt.ctas_per_sm : 8;
+            const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 16;
             const int grid = (int)std::min<int64_t>(n_items, (int64_t)dev.sms * per_sm);
             w_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
             e = cudaGetLastError();
         } else {
-            const BulkShape bs = bulk_shape(dev, plan->opt, stage_bytes);
-            const int grid = (int)std::min<int64_t>((n_items + bs.warps - 1) / bs.warps, (int64_t)dev.sms * bs.ctas_per_sm);
-            switch (bs.stages) {
-                case 2: e = launch_bulk<2, 1>(p, grid, bs.warps, stage_bytes, d_status, stream); break;
-                case 3: e = launch_bulk<3, 2>(p, grid, bs.warps, stage_bytes, d_status, stream); break;
-                case 4: e = launch_bulk<4, 2>(p, grid, bs.warps, stage_bytes, d_status, stream); break;
-                case 6: e = launch_bulk<6, 3>(p, grid, bs.warps, stage_bytes, d_status, stream); break;
-                default: e = launch_bulk<8, 4>(p, grid, bs.warps, stage_bytes, d_status, stream); break;
+            const BulkShape bs = bulk_shape(dev, opt, kWDefaults, path, stage_bytes);
+            const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+            auto kernel = path == 3 ? w_reshard_pair : w_reshard_bulk;
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+            if (e == cudaSuccess) {
+                kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring, d_status);
+                e = cudaGetLastError();
             }
         }
         if (e != cudaSuccess) return AMOEBA_ERR_CUDA;

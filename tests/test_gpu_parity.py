@@ -7,7 +7,8 @@ from harness import check_case, make_case, run_case
 
 pytestmark = pytest.mark.gpu
 
-LDST, BULK = 1, 2
+LDST, BULK, PAIR = 1, 2, 3
+PATHS = [LDST, BULK, PAIR]
 SMALL40 = dict(L=2, hidden=320, Hq=40, Hkv=40, D=16, I=640)  # 40-head shape: divisors 1,2,4,5,8,10,20,40
 GQA = dict(L=3, hidden=512, Hq=16, Hkv=8, D=128, I=1792)
 
@@ -22,7 +23,7 @@ def _need_gpu():
     assert A.library_path().exists()
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 def test_tiny_config_end_to_end(path):
     cfg = wl.CONFIGS["tiny_2to1"]
     lens = wl.draw_seq_lens(cfg, name="tiny_2to1")
@@ -30,7 +31,7 @@ def test_tiny_config_end_to_end(path):
     check_case(c, run_case(c, path))
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("a,b", [(1, 2), (2, 1), (1, 4), (4, 1), (2, 8), (8, 2), (4, 4), (1, 1), (8, 1), (1, 8)])
 def test_gqa_shapes_all_directions(path, a, b):
     lens = [1, 16, 17, 300, 0, 77, 1024, 5]
@@ -38,7 +39,7 @@ def test_gqa_shapes_all_directions(path, a, b):
     check_case(c, run_case(c, path))
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("a,b", [(4, 5), (5, 8), (8, 5), (10, 4), (10, 20), (20, 1), (5, 5)])
 def test_non_nested_partitions(path, a, b):
     lens = [33, 7, 0, 64, 129]
@@ -46,14 +47,14 @@ def test_non_nested_partitions(path, a, b):
     check_case(c, run_case(c, path))
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("fq,fg", [(False, False), (True, False), (False, True)])
 def test_unfused_weight_buffers(path, fq, fg):
     c = make_case(GQA, 2, 4, [40], fused_qkv=fq, fused_gate_up=fg, kv=True, seed=5)
     check_case(c, run_case(c, path))
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 def test_free_mask_compaction_and_foreign_blocks(path):
     lens = list(np.random.default_rng(3).integers(1, 600, size=200))
     c = make_case(dict(GQA, L=1), 4, 1, lens, dst_form="mask", dst_occupied=0.3, src_free=0.3, weights=False, seed=9)
@@ -61,7 +62,7 @@ def test_free_mask_compaction_and_foreign_blocks(path):
     check_case(c, s)  # foreign (occupied) blocks keep the fill: whole-pool comparison
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("chunk", [1024, 4096, 8192, 32768])
 def test_chunk_sizes_and_ragged_tails(path, chunk):
     import paper_2509_19729_b200 as A
@@ -71,13 +72,28 @@ def test_chunk_sizes_and_ragged_tails(path, chunk):
     check_case(c, run_case(c, path, options=[(A.OPT_CHUNK_BYTES, chunk)]))
 
 
-@pytest.mark.parametrize("stages", [2, 3, 4, 6, 8])
-def test_bulk_ring_depths(stages):
+@pytest.mark.parametrize("path", [BULK, PAIR])
+@pytest.mark.parametrize("stages,lag,warps", [(2, 1, 1), (3, 2, 2), (4, 2, 3), (6, 3, 0), (8, 1, 2), (12, 11, 1),
+                                              (16, 8, 1), (5, 4, 16)])
+def test_bulk_ring_shapes(path, stages, lag, warps):
     import paper_2509_19729_b200 as A
 
     c = make_case(GQA, 1, 4, [500, 20, 1000], seed=stages)
-    check_case(c, run_case(c, BULK, options=[(A.OPT_STAGES, stages)]))
-    check_case(c, run_case(c, BULK, options=[(A.OPT_STAGES, stages), (A.OPT_CHUNK_BYTES, 4096), (A.OPT_CTAS_PER_SM, 2)]))
+    opts = [(A.OPT_STAGES, stages), (A.OPT_LAG, lag), (A.OPT_WARPS, warps)]
+    check_case(c, run_case(c, path, options=opts))
+    check_case(c, run_case(c, path, options=opts + [(A.OPT_CHUNK_BYTES, 4096), (A.OPT_CTAS_PER_SM, 2),
+                                                    (A.OPT_L2_HINT, 4)]))
+
+
+def test_per_kernel_options():
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 2, 4, [300, 20], seed=77)
+    opts = [(A.OPT_COPY_PATH + A.OPT_KV_ONLY, PAIR), (A.OPT_COPY_PATH + A.OPT_WEIGHTS_ONLY, LDST),
+            (A.OPT_CHUNK_BYTES + A.OPT_WEIGHTS_ONLY, 2048), (A.OPT_L2_HINT + A.OPT_KV_ONLY, 2)]
+    s = run_case(c, None, options=opts)
+    assert A.amoeba_plan_kv_info(s.plan).chunk_bytes == 8192  # the weights-only chunk option left KV alone
+    check_case(c, s)
 
 
 def test_long_single_row_and_many_sequences():
@@ -115,7 +131,7 @@ def test_invalid_lengths_and_pairs_cap():
     check_case(c, run_case(c, LDST))
 
 
-@pytest.mark.parametrize("path", [LDST, BULK])
+@pytest.mark.parametrize("path", PATHS)
 def test_bad_block_ids_are_skipped(path):
     lens = [160, 48]
     base = make_case(GQA, 2, 1, lens, weights=False, seed=4)

@@ -394,3 +394,122 @@ def test_workload_generators():
     x = np.array([1.0, -2.5, 3.1415926, 1e-3], dtype=np.float32)
     assert np.allclose(wl.from_bits(wl.to_bits(x, "bf16"), "bf16"), x, rtol=2 ** -8)
     assert np.allclose(wl.from_bits(wl.to_bits(x, "fp16"), "fp16"), x, rtol=2 ** -10)
+
+
+# ---------------- token-first storage order (Sec. 3.1: the mainstream-engine layout the paper starts from) ----------------
+@pytest.mark.parametrize("TP", [1, 2, 4])
+def test_token_first_memory_order_and_two_regions(oracle, TP):
+    m, T, NB = SMALL, 4, 7
+    seq_lens = [5, 0, 9, 4]
+    bt, nblk = _state(seq_lens, T, NB)
+    G = int(nblk.sum()) * T
+    n = m["L"] * G * m["Hkv"] * 2 * m["D"]
+    KV = np.arange(n, dtype=np.uint16).reshape(m["L"], G, m["Hkv"], 2, m["D"])
+    FILL = 0xFFFF
+    pools = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=FILL, order=oracle.TOKEN_FIRST)
+    Hs = m["Hkv"] // TP
+    region = NB * T * Hs * m["D"]  # one of K / V for one layer
+    tok_block = {}
+    g0 = 0
+    for s, nb in enumerate(nblk):
+        for t in range(nb * T):
+            tok_block[g0 + t] = (bt[s, t // T], t % T)
+        g0 += nb * T
+    seen = 0
+    for r, pool in enumerate(pools):
+        assert pool.size == m["L"] * 2 * region
+        written = np.flatnonzero(pool != FILL)
+        seen += written.size
+        l, g, h, c, d = np.unravel_index(pool[written].astype(np.int64), KV.shape)
+        blk = np.array([tok_block[x][0] for x in g])
+        tok = np.array([tok_block[x][1] for x in g])
+        # memory order == lexicographic order of (layer, K/V, block, token, header, dim)
+        keys = np.stack([l, c, blk, tok, h, d], axis=1)
+        assert np.array_equal(np.lexsort(keys.T[::-1]), np.arange(len(keys)))
+        # K and V live in two separate contiguous regions of each layer
+        assert np.array_equal(c, (written // region) % 2)
+        assert np.array_equal(l, written // (2 * region))
+        # a token's headers are stored together: Hs*D consecutive words share (block, token)
+        runs = (written // (Hs * m["D"]))
+        for run in np.unique(runs)[:50]:
+            sel = runs == run
+            assert len(set(zip(blk[sel].tolist(), tok[sel].tolist(), c[sel].tolist()))) == 1 and sel.sum() == Hs * m["D"]
+    assert seen == n
+
+
+@pytest.mark.parametrize("TP", [1, 2, 4])
+def test_token_first_equals_numpy_split(oracle, TP):
+    m, T, NB = SMALL, 4, 9
+    seq_lens = [7, 3, 0, 16, 1]
+    bt, nblk = _state(seq_lens, T, NB, seed=3)
+    G = int(nblk.sum()) * T
+    KV = np.random.default_rng(0).integers(0, 65536, size=(m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    pools = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=0, order=oracle.TOKEN_FIRST)
+    parts = np.split(KV, TP, axis=2)
+    Hs = m["Hkv"] // TP
+    for r in range(TP):
+        pool = pools[r].reshape(m["L"], 2, NB, T, Hs, m["D"])
+        g0 = 0
+        for s, nb in enumerate(nblk):
+            for i in range(nb):
+                blk_logical = parts[r][:, g0 + i * T:g0 + (i + 1) * T]  # [L, T, Hs, 2, D]
+                assert np.array_equal(pool[:, :, bt[s, i]], blk_logical.transpose(0, 3, 1, 2, 4))
+            g0 += nb * T
+    assert np.array_equal(oracle.kv_reconstruct(pools, m, T, TP, NB, seq_lens, bt, order=oracle.TOKEN_FIRST), KV)
+
+
+@pytest.mark.parametrize("a,b,so,do", [(1, 4, 1, 1), (4, 2, 1, 1), (2, 2, 1, 0), (2, 4, 0, 1), (4, 1, 1, 0), (1, 2, 0, 1)])
+def test_storage_order_conversions_round_trip(oracle, a, b, so, do):
+    m, T = SMALL, 4
+    seq_lens = [9, 4, 0, 13, 2]
+    NB_a, NB_b = 10, 13
+    bt_a, nblk = _state(seq_lens, T, NB_a, seed=7)
+    G = int(nblk.sum()) * T
+    KV = np.random.default_rng(2).integers(0, 65536, size=(m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    pools_a = oracle.kv_shard(KV, m, T, a, NB_a, seq_lens, bt_a, order=so)
+    free_b = np.random.default_rng(3).permutation(NB_b).astype(np.int32)
+    bt_b, pairs, N, left, st = oracle.assign_blocks(seq_lens, T, bt_a, NB_a, NB_b, free_list=free_b)
+    pools_b = [np.full(m["L"] * oracle.pool_elems_per_layer(m, T, b, NB_b), 0xA5A5, np.uint16) for _ in range(b)]
+    oracle.kv_transform(m, T, seq_lens, a, NB_a, bt_a, pools_a, b, NB_b, bt_b, pools_b, src_order=so, dst_order=do)
+    direct = oracle.kv_shard(KV, m, T, b, NB_b, seq_lens, bt_b, order=do)
+    for x, y in zip(pools_b, direct):
+        assert np.array_equal(x, y)
+    via_pairs = [np.full_like(p, 0xA5A5) for p in pools_b]
+    assert oracle.kv_copy_pairs(m, T, a, NB_a, pools_a, b, NB_b, via_pairs, pairs, N, src_order=so, dst_order=do) == 0
+    for x, y in zip(pools_b, via_pairs):
+        assert np.array_equal(x, y)
+    # back again with the original ids: physical bytes identical
+    bt_a2, _, _, _, st2 = oracle.assign_blocks(seq_lens, T, bt_b, NB_b, NB_a, free_list=bt_a[bt_a >= 0])
+    back = [np.full_like(p, 0xA5A5) for p in pools_a]
+    oracle.kv_transform(m, T, seq_lens, b, NB_b, bt_b, pools_b, a, NB_a, bt_a2, back, src_order=do, dst_order=so)
+    for x, y in zip(back, pools_a):
+        assert np.array_equal(x, y)
+
+
+def test_decode_attention_from_token_first_strides(oracle):
+    """The same decode-step attention, read through the token-first strides, gives the same bits."""
+    cfg = wl.CONFIGS["tiny_2to1"]
+    m, T = cfg["model"], wl.BLOCK_TOKENS
+    st = wl.draw_kv_state(cfg, name="tiny_2to1")
+    seq_lens, bt = st["seq_lens"], st["src_bt"]
+    G = int(st["blocks_per_seq"].sum()) * T
+    KV = wl.draw_kv_logical(cfg, G, range(m["L"]))
+    TP, NB = 2, st["NB_src"]
+    Hs = m["Hkv"] // TP
+    tf = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, order=oracle.TOKEN_FIRST)
+    hc = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, order=oracle.HEADER_CENTRIC)
+    q = wl.rng(7, "q").standard_normal(size=(m["D"],)).astype(np.float32)
+
+    def attend(K, V):
+        s = (K.view(np.float16).astype(np.float32) @ q) / np.float32(np.sqrt(m["D"]))
+        p = np.exp(s - s.max())
+        return (p / p.sum()) @ V.view(np.float16).astype(np.float32)
+
+    for l, s, h in itertools.product(range(m["L"]), range(len(seq_lens)), range(m["Hkv"])):
+        blocks = bt[s, :st["blocks_per_seq"][s]]
+        a_tf = tf[h // Hs].reshape(m["L"], 2, NB, T, Hs, m["D"])[l][:, blocks][:, :, :, h % Hs]  # [2, nblk, T, D]
+        a_hc = hc[h // Hs].reshape(m["L"], NB, Hs, 2, T, m["D"])[l, blocks, h % Hs]        # [nblk, 2, T, D]
+        n = seq_lens[s]
+        K1, V1 = (np.ascontiguousarray(a_tf[c].reshape(-1, m["D"])[:n]) for c in (0, 1))
+        K2, V2 = (np.ascontiguousarray(a_hc[:, c].reshape(-1, m["D"])[:n]) for c in (0, 1))
+        assert np.array_equal(attend(K1, V1).view(np.uint32), attend(K2, V2).view(np.uint32))
