@@ -32,9 +32,12 @@ DEFAULT_CONFIG = "llama3_8b_1to4"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes (read + written) per algorithmic byte of kv_reshard, from the ncu capture summarised in
-# profiles/ (None until a capture exists for the default copy path).
-NCU_KV_TRAFFIC_RATIO = None
+# DRAM bytes (read + written) per algorithmic byte of kv_reshard_pair (the default copy path), from the ncu capture
+# summarised in profiles/kv_reshard_pair_llama3_8b_1to4_1layer.md: taken on a one-layer slice and scaled by the
+# bytes of a full launch (every layer repeats the same work on disjoint memory).  Only quoted for that workload
+# with default kernel options.
+NCU_KV_TRAFFIC_RATIO = 0.9895
+NCU_KV_TRAFFIC_CONFIG = "llama3_8b_1to4"
 
 
 def peaks():
@@ -118,9 +121,10 @@ def barrier(world: int):
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=48, w_layers=2, threads=1):
-    """A bounded sample of the workload for the CPU oracle: the first n_seqs sequences over kv_layers layers of
-    KV, and w_layers layers of weights.  Returns a closure that runs one oracle a->b pass and the bytes it moves."""
+def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=None, w_layers=4, threads=1):
+    """A bounded sample of the workload for the CPU oracle: the first n_seqs sequences (None = all) over kv_layers
+    layers of KV, and w_layers layers of weights; values are uniform 16-bit words (the movement does not depend on
+    them).  Returns a closure that runs one oracle a->b pass and the bytes it moves."""
     import oracle
 
     oracle.build()
@@ -128,16 +132,17 @@ def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=48, w_layers=2, threads=1):
     cfg = wl.CONFIGS[cfg_name]
     m, a, b, T = dict(cfg["model"]), cfg["a"], cfg["b"], wl.BLOCK_TOKENS
     lens = wl.draw_seq_lens(cfg, name=cfg_name)[:n_seqs]
+    kv_layers, w_layers = min(kv_layers, cfg.get("kv_layers") or m["L"]), min(w_layers, m["L"])
     m_kv = dict(m, L=kv_layers)
     st = wl.draw_kv_state(cfg, name=cfg_name, seq_lens=lens)
     G = int(st["blocks_per_seq"].sum()) * T
-    KV = wl.draw_kv_logical(dict(cfg, model=m_kv), G, range(kv_layers))
+    KV = wl.draw_kv_logical(dict(cfg, model=m_kv), G, range(kv_layers), dist="words")
     src = oracle.kv_shard(KV, m_kv, T, a, st["NB_src"], lens, st["src_bt"])
     del KV
     free = dict(free_list=st.get("dst_free_list"), free_mask=st.get("dst_free_mask"))
     dst = [np.full(kv_layers * oracle.pool_elems_per_layer(m_kv, T, b, st["NB_dst"]), 0xA5A5, np.uint16)
            for _ in range(b)]
-    W = [oracle.weights_shard(wl.draw_weights_logical(cfg, l), m, a) for l in range(w_layers)]
+    W = [oracle.weights_shard(wl.draw_weights_logical(cfg, l, dist="words"), m, a) for l in range(w_layers)]
     Wd = [oracle.empty_shards(m, b) for _ in range(w_layers)]
     e = 2
     kv_bytes = 2 * st["n_live"] * kv_layers * m["Hkv"] * 2 * T * m["D"] * e
@@ -160,7 +165,7 @@ def run_reference(args, rank, world):
     """The reference arm: the CPU oracle as it stands, timed on the host cores on a bounded sample per step."""
     if rank != 0:
         return
-    run, nbytes, desc = oracle_sample(args.config)
+    run, nbytes, desc = oracle_sample(args.config, kv_layers=1, w_layers=2)
     for _ in range(args.warmup):
         run()
     t0 = time.perf_counter()
@@ -332,7 +337,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=list(wl.CONFIGS))
-    ap.add_argument("--copy-path", type=int, default=0, help="0 default, 1 vector ld/st, 2 bulk-copy ring")
+    ap.add_argument("--copy-path", type=int, default=0, help="0 default, 1 vector ld/st, 2 bulk-copy ring per warp, 3 producer/consumer bulk-copy ring")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
@@ -409,6 +414,8 @@ def main():
         return
 
     peak, peak_kind = peaks()
+    traffic_known = (NCU_KV_TRAFFIC_RATIO is not None and args.config == NCU_KV_TRAFFIC_CONFIG
+                     and not (args.copy_path or args.chunk or args.stages or args.ctas_per_sm))
     kv_gbs = kv_bytes / (kv_ms / 1e3) / 1e9
     w_gbs = w_bytes / (w_ms / 1e3) / 1e9 if w_bytes else None
     out = {
@@ -419,7 +426,7 @@ def main():
                    "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
                    "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
                    "l2_policy": "no flush: every step streams far more than the 126 MB L2",
-                   "copy_path": {0: "default", 1: "ldst", 2: "bulk"}[args.copy_path],
+                   "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],
                    "chunk_bytes": n_seq_layers[2]},
         "phases_ms": {"rewrite_block_tables": bt_ms, "reshard_kv": kv_ms, "reshard_weights": w_ms,
                       "reshard_kv_min": min(phase[1]), "reshard_weights_min": min(phase[2])},
@@ -428,7 +435,7 @@ def main():
                                 "reshard_weights": 100 * w_gbs / NOMINAL_HBM_GBS if w_gbs else None},
         "roofline": {"kernel": "kv_reshard", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
                      "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": None if NCU_KV_TRAFFIC_RATIO is None else NCU_KV_TRAFFIC_RATIO * kv_bytes},
+                     "traffic": NCU_KV_TRAFFIC_RATIO * kv_bytes if traffic_known else None},
         "roofline_weights": None if not w_gbs else {"kernel": "w_reshard", "bound": "hbm", "achieved": w_gbs,
                                                     "peak": peak, "unit": "GB/s", "frac": w_gbs / peak},
         "gpu_launches": int(launches), "clocks": clocks,

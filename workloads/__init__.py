@@ -131,24 +131,35 @@ def draw_kv_state(cfg: dict, seed: int = DEFAULT_SEED, name: str = "", seq_lens=
     return st
 
 
-def draw_kv_logical(cfg: dict, n_tokens: int, layers, seed: int = DEFAULT_SEED) -> np.ndarray:
-    """Logical KV values N(0,1) for the given layers: uint16 [len(layers), n_tokens, Hkv, 2, D]."""
+def draw_kv_logical(cfg: dict, n_tokens: int, layers, seed: int = DEFAULT_SEED, dist: str = "normal") -> np.ndarray:
+    """Logical KV values for the given layers: uint16 [len(layers), n_tokens, Hkv, 2, D].
+
+    dist "normal": N(0,1) rounded to the config's 16-bit float type; "words": uniform 16-bit words (several times
+    faster to draw; for timing runs, where the values do not matter)."""
     m = cfg["model"]
     out = np.empty((len(layers), n_tokens, m["Hkv"], 2, m["D"]), dtype=np.uint16)
     for i, l in enumerate(layers):
-        x = rng(seed, "kv", l).standard_normal(size=out.shape[1:], dtype=np.float32)
-        out[i] = to_bits(x, cfg["dtype"])
+        if dist == "words":
+            out[i] = rng(seed, "kv_words", l).integers(0, 65536, size=out.shape[1:], dtype=np.uint16)
+        else:
+            x = rng(seed, "kv", l).standard_normal(size=out.shape[1:], dtype=np.float32)
+            out[i] = to_bits(x, cfg["dtype"])
     return out
 
 
-def draw_weights_logical(cfg: dict, layer: int, seed: int = DEFAULT_SEED, std: float = 0.02) -> dict:
-    """One layer's logical weights N(0, std), [out,in] row-major, as uint16 words."""
+def draw_weights_logical(cfg: dict, layer: int, seed: int = DEFAULT_SEED, std: float = 0.02,
+                         dist: str = "normal") -> dict:
+    """One layer's logical weights, [out,in] row-major, as uint16 words: N(0, std) rounded to the config's 16-bit
+    float type, or (dist "words", for timing runs) uniform 16-bit words."""
     m = cfg["model"]
     hid, qr, kr, I = m["hidden"], m["Hq"] * m["D"], m["Hkv"] * m["D"], m["I"]
     shapes = {"q": (qr, hid), "k": (kr, hid), "v": (kr, hid), "o": (hid, qr), "gate": (I, hid), "up": (I, hid),
               "down": (hid, I)}
     out = {}
     for j, (n, s) in enumerate(shapes.items()):
+        if dist == "words":
+            out[n] = rng(seed, "w_words", layer, j).integers(0, 65536, size=s, dtype=np.uint16)
+            continue
         x = rng(seed, "w", layer, j).standard_normal(size=s, dtype=np.float32) * np.float32(std)
         out[n] = to_bits(x, cfg["dtype"])
     return out
