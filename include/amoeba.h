@@ -4,9 +4,10 @@
  * The library re-lays-out the state of one running LLM instance from a tensor-parallel partition of degree a to
  * one of degree b without recomputing anything (the transformation the Amoeba paper introduces in its Sec. 1 and
  * designs in Sec. 3.1 - 3.2).  The state is
- *   - the paged, head-sharded KV cache in the header-centric layout of Sec. 3.1 ("Improvement 1"):
+ *   - the paged, head-sharded KV cache, by default in the header-centric layout of Sec. 3.1 ("Improvement 1"):
  *       pool of worker r:  [layer][block][header of r][K/V][token][head_dim]
- *     where worker r (0-indexed here; W_{r+1} in the paper) owns the K/V headers r*Hkv/tp ... (r+1)*Hkv/tp - 1
+ *     (the token-first order [layer][K/V][block][token][header of r][head_dim] is accepted on either side, so a
+ *     transformation can also convert between the two), where worker r (0-indexed here; W_{r+1} in the paper) owns the K/V headers r*Hkv/tp ... (r+1)*Hkv/tp - 1
  *     (Sec. 3.1 "Base solution", 1-indexed there), and
  *   - the projection weights, stored [out,in] row-major and partitioned as in Sec. 3.2, Eq. 1:
  *     q/k/v/gate/up by output rows (the paper's column-wise split of U), o_proj/down_proj by input columns (the
@@ -51,7 +52,13 @@ typedef enum {
     AMOEBA_ERR_TOO_LARGE = 8       /* the problem needs more scratch than the library's built-in scratch array holds */
 } amoeba_status;
 
-enum { AMOEBA_KV_HEAD_MAJOR = 0 /* [block][header][K/V][token][dim], Sec. 3.1 Improvement 1 */ };
+/* Storage order of one layer of a worker's KV pool (Sec. 3.1).  HEAD_MAJOR is the paper's header-centric layout
+ * ("Improvement 1"); TOKEN_MAJOR is the token-first layout of mainstream engines that the paper starts from: K and V
+ * are two contiguous regions of the layer and a token's headers are stored together. */
+enum {
+    AMOEBA_KV_HEAD_MAJOR = 0, /* [block][header][K/V][token][dim] */
+    AMOEBA_KV_TOKEN_MAJOR = 1 /* [K/V][block][token][header][dim] */
+};
 enum { AMOEBA_MAX_TP = 32 }; /* and at most 22 intersecting (source worker, destination worker) pairs */
 
 /* Transformer shape.  elem_bytes is the size of one weight / KV element (2: fp16 or bf16). */
@@ -65,7 +72,7 @@ typedef struct {
     int32_t tp;            /* number of workers; must divide num_q_heads, num_kv_heads and intermediate */
     int32_t block_tokens;  /* tokens per KV block */
     int32_t num_blocks;    /* capacity of every worker's pool, in blocks, per layer */
-    int32_t kv_order;      /* AMOEBA_KV_HEAD_MAJOR */
+    int32_t kv_order;      /* AMOEBA_KV_HEAD_MAJOR or AMOEBA_KV_TOKEN_MAJOR; source and destination may differ */
     int32_t fused_qkv;     /* 1: worker buffer [q_r; k_r; v_r] (pointer in .q, .k/.v unused); 0: three buffers */
     int32_t fused_gate_up; /* 1: worker buffer [gate_r; up_r] (pointer in .gate, .up unused); 0: two buffers */
     int64_t kv_layer_stride_bytes; /* distance between layers inside a worker's pool; 0 = dense */
@@ -104,7 +111,7 @@ typedef struct {
     int32_t heads_per_run;   /* consecutive K/V headers that share one source and one destination worker */
     int32_t runs_per_block;  /* num_kv_heads / heads_per_run */
     int64_t run_bytes;       /* heads_per_run * 2 * block_tokens * head_dim * elem_bytes */
-    int64_t chunk_bytes;     /* size of one copy work item (divides run_bytes) */
+    int64_t chunk_bytes;     /* largest copy work item in bytes (both sides header-centric: it divides run_bytes) */
     int64_t src_block_bytes, dst_block_bytes;   /* one block in a source / destination worker's pool */
     int64_t src_layer_stride, dst_layer_stride; /* bytes between layers in a pool */
 } amoeba_kv_info;
@@ -212,7 +219,8 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
  *
  * For every pair k < min(*d_num_pairs, pairs_cap) with both ids >= 0, every layer in [layer_begin, layer_end) and
  * every K/V header h: the 2*block_tokens*head_dim elements of (block, header) are copied from
- * src_pools[h / (Hkv/a)] to dst_pools[h / (Hkv/b)] at the pool addresses of the header-centric layout.
+ * src_pools[h / (Hkv/a)] to dst_pools[h / (Hkv/b)], read at the addresses of the source layout's kv_order and
+ * written at those of the destination layout's kv_order.
  * src_pools / dst_pools are HOST arrays of a / b device pointers (read during the call only).
  * A pair with an id outside its pool is skipped and sets BAD_BLOCK_ID in *d_status.
  */

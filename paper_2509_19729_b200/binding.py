@@ -31,6 +31,8 @@ __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO
 OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT = range(7)
 OPT_WEIGHTS_ONLY, OPT_KV_ONLY = 16, 32  # add to an option id to set one kernel only
 COPY_PATH_LDST, COPY_PATH_BULK, COPY_PATH_PAIR = 1, 2, 3
+KV_HEAD_MAJOR, KV_TOKEN_MAJOR = 0, 1  # [block][header][K/V][token][dim] / [K/V][block][token][header][dim]
+__all__ += ["KV_HEAD_MAJOR", "KV_TOKEN_MAJOR"]
 TENSOR_NAMES = ("q", "k", "v", "o", "gate", "up", "down")
 
 
@@ -145,10 +147,12 @@ class Plan:
 
 
 def make_layout(model: dict, tp: int, num_blocks: int, block_tokens: int = 16, fused_qkv: bool = True,
-                fused_gate_up: bool = True, elem_bytes: int = 2, kv_layer_stride_bytes: int = 0) -> Layout:
-    """Layout from a shape dict with keys L, hidden, Hq, Hkv, D, I."""
+                fused_gate_up: bool = True, elem_bytes: int = 2, kv_layer_stride_bytes: int = 0,
+                kv_order: int = 0) -> Layout:
+    """Layout from a shape dict with keys L, hidden, Hq, Hkv, D, I; kv_order KV_HEAD_MAJOR or KV_TOKEN_MAJOR."""
     m = Model(model["L"], model["hidden"], model["Hq"], model["Hkv"], model["D"], model["I"], elem_bytes)
-    return Layout(m, tp, block_tokens, num_blocks, 0, int(fused_qkv), int(fused_gate_up), kv_layer_stride_bytes)
+    return Layout(m, tp, block_tokens, num_blocks, int(kv_order), int(fused_qkv), int(fused_gate_up),
+                  kv_layer_stride_bytes)
 
 
 def amoeba_status_string(status: int) -> str:

@@ -65,14 +65,35 @@ __device__ __forceinline__ void copy_vecs(const uint4* __restrict__ s, uint4* __
 // All threads of the CTA call this with the same item.
 template <int UNROLL>
 __device__ __forceinline__ void cta_copy_item(const Item& it) {
-    if (it.n_rows == 1) {
-        copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src), reinterpret_cast<uint4*>(it.dst), it.row_bytes >> 4,
-                          threadIdx.x, blockDim.x);
-    } else {  // one warp per row, lanes along the row
+    if (it.n_rows == 1 || (it.src_pitch == it.row_bytes && it.dst_pitch == it.row_bytes)) {
+        copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src), reinterpret_cast<uint4*>(it.dst),
+                          (it.n_rows * it.row_bytes) >> 4, threadIdx.x, blockDim.x);
+    } else if (it.row_bytes >= 512) {  // one warp per row, lanes along the row
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
         for (int r = warp; r < it.n_rows; r += nwarps)
             copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch),
                               reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch), it.row_bytes >> 4, lane, 32);
+    } else {  // short rows: the vectors of all rows are dealt to the threads of the CTA
+        const int vpr = it.row_bytes >> 4, n = it.n_rows * vpr;
+        for (int base = 0; base < n; base += blockDim.x * UNROLL) {
+            uint4 v[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n) {
+                    const int r = i / vpr, c = i - r * vpr;
+                    v[u] = ld_stream(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch) + c);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int i = base + u * blockDim.x + threadIdx.x;
+                if (i < n) {
+                    const int r = i / vpr, c = i - r * vpr;
+                    st_stream(reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch) + c, v[u]);
+                }
+            }
+        }
     }
 }
 
@@ -161,6 +182,30 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 constexpr int kMaxStages = 16;
 
+// One item between global memory and a shared-memory stage (rows packed densely in the stage).  A side whose rows
+// are adjacent in global memory (pitch == row_bytes, or a single row) moves as ONE bulk copy issued by lane 0;
+// otherwise lane r moves row r, r + 32, ...  All lanes of the warp call these with the same item.
+__device__ __forceinline__ void item_load(const Item& it, char* stage, uint64_t* bar, bool hint, uint64_t policy) {
+    const int lane = threadIdx.x & 31;
+    if (it.n_rows == 0) return;  // skipped item: the barrier phase completes with 0 bytes expected
+    if (it.n_rows == 1 || it.src_pitch == it.row_bytes) {
+        if (lane == 0) bulk_g2s(stage, it.src, (uint32_t)it.n_rows * (uint32_t)it.row_bytes, bar, hint, policy);
+    } else {
+        for (int r = lane; r < it.n_rows; r += 32)
+            bulk_g2s(stage + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, bar, hint, policy);
+    }
+}
+__device__ __forceinline__ void item_store(const Item& it, const char* stage, bool hint, uint64_t policy) {
+    const int lane = threadIdx.x & 31;
+    if (it.n_rows == 0) return;
+    if (it.n_rows == 1 || it.dst_pitch == it.row_bytes) {
+        if (lane == 0) bulk_s2g(it.dst, stage, (uint32_t)it.n_rows * (uint32_t)it.row_bytes, hint, policy);
+    } else {
+        for (int r = lane; r < it.n_rows; r += 32)
+            bulk_s2g(it.dst + r * it.dst_pitch, stage + (int64_t)r * it.row_bytes, it.row_bytes, hint, policy);
+    }
+}
+
 // ------------------------------------------------------------------ one ring per warp
 // Loads run `lag` items ahead of stores, so up to `lag` loads and `stages - lag` stores are in flight per warp.
 // `item_of(w)` must return the same Item in every lane.  bars: `stages` mbarriers of this warp.
@@ -189,10 +234,7 @@ __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, 
             const Item it = item_of(first + k * stride);
             if (lane == 0) mbar_arrive_expect_tx(&bars[s_load], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
             __syncwarp();
-            char* st = stages + (int64_t)s_load * rs.stage_bytes;
-            for (int r = lane; r < it.n_rows; r += 32)
-                bulk_g2s(st + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, &bars[s_load], hl,
-                         policy);
+            item_load(it, stages + (int64_t)s_load * rs.stage_bytes, &bars[s_load], hl, policy);
             ++loads_issued;
             if (++s_load == NS) s_load = 0;
         }
@@ -202,9 +244,7 @@ __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, 
             if (ok) {
                 ++loads_waited;
                 const Item it = item_of(first + (k - LAG) * stride);
-                const char* st = stages + (int64_t)s_store * rs.stage_bytes;
-                for (int r = lane; r < it.n_rows; r += 32)
-                    bulk_s2g(it.dst + r * it.dst_pitch, st + (int64_t)r * it.row_bytes, it.row_bytes, hs, policy);
+                item_store(it, stages + (int64_t)s_store * rs.stage_bytes, hs, policy);
             }
             bulk_commit();
             if (++s_store == NS) {
@@ -256,10 +296,7 @@ __device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t
             const Item it = item_of(first + k * stride);
             if (lane == 0) mbar_arrive_expect_tx(&full[slot], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
             __syncwarp();
-            char* st = stages + (int64_t)slot * rs.stage_bytes;
-            for (int r = lane; r < it.n_rows; r += 32)
-                bulk_g2s(st + (int64_t)r * it.row_bytes, it.src + r * it.src_pitch, it.row_bytes, &full[slot], hl,
-                         policy);
+            item_load(it, stages + (int64_t)slot * rs.stage_bytes, &full[slot], hl, policy);
             if (++slot == NS) {
                 slot = 0;
                 parity ^= 1;
@@ -273,9 +310,7 @@ __device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const Item it = item_of(first + k * stride);
-            const char* st = stages + (int64_t)slot * rs.stage_bytes;
-            for (int r = lane; r < it.n_rows; r += 32)
-                bulk_s2g(it.dst + r * it.dst_pitch, st + (int64_t)r * it.row_bytes, it.row_bytes, hs, policy);
+            item_store(it, stages + (int64_t)slot * rs.stage_bytes, hs, policy);
             bulk_commit();
             if (k >= D) {  // the store issued D items ago has read its slot: hand it back
                 bulk_wait_read(D);

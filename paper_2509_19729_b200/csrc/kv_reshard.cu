@@ -1,11 +1,14 @@
 // KV cache migration in the head dimension (Sec. 3.1) as an on-GPU gather/scatter between the pools of the
-// source workers (TP = a) and of the destination workers (TP = b), header-centric layout
-// [layer][block][header][K/V][token][dim] on both sides.
+// source workers (TP = a) and of the destination workers (TP = b).  Either side may use the header-centric order
+// [layer][block][header][K/V][token][dim] (Sec. 3.1, Improvement 1) or the token-first order
+// [layer][K/V][block][token][header][dim] of mainstream engines.
 //
-// Work decomposition: (layer, pair, run, chunk).  A run is heads_per_run = gcd(Hkv/a, Hkv/b) consecutive headers
-// of one block: contiguous in exactly one source pool and one destination pool.  Runs are cut into equal chunks
-// (the copy work items), dealt round-robin to a persistent grid; layer is the slowest index so that concurrently
-// running CTAs touch neighbouring DRAM pages.
+// Work decomposition: (layer, pair, K/V plane, header unit, row group, column chunk).  A header unit is a group of
+// consecutive headers that lives in exactly one source pool and one destination pool and is a regular 2-D copy on
+// both sides (see KvGeom): with both sides header-centric it is a run of gcd(Hkv/a, Hkv/b) headers, K and V
+// together, one contiguous row; with token-first on a side it is one row per token.  Units are cut into copy work
+// items, dealt round-robin to a persistent grid; layer is the slowest index so that concurrently running CTAs touch
+// neighbouring DRAM pages.
 #include <cuda_runtime.h>
 
 #include "copy_engine.cuh"
@@ -20,50 +23,67 @@ struct KvParams {
     const int32_t* pairs;      // [cap][2]
     const int32_t* num_pairs;  // device scalar
     int32_t* status;
-    int64_t unit_bytes, chunk_bytes, src_layer_stride, dst_layer_stride;
+    int64_t vec_bytes, src_layer_stride, dst_layer_stride;
+    int64_t row_bytes, src_row_pitch, dst_row_pitch;
     int32_t pairs_cap, layer_begin, n_layers;
-    int32_t nb_src, nb_dst;
-    int32_t heads_src, heads_dst, heads_per_run, runs_per_block, chunks_per_run;
+    int32_t nb_src, nb_dst, block_tokens;
+    int32_t src_token_major, dst_token_major;
+    int32_t heads_src, heads_dst, heads_per_unit, head_units, planes;
+    int32_t rows, rows_per_item, row_groups, col_chunks, chunk_bytes;
 };
+
+// Byte offset, inside one layer of a worker's pool, of token 0 of (block, local header, K/V plane).
+__device__ __forceinline__ int64_t pool_offset(bool token_major, int32_t nb, int32_t heads, int32_t T, int64_t vec,
+                                               int32_t blk, int32_t hl, int32_t c) {
+    return token_major ? ((((int64_t)c * nb + blk) * T) * heads + hl) * vec
+                       : ((((int64_t)blk * heads + hl) * 2 + c) * T) * vec;
+}
 
 struct KvItems {
     const KvParams& p;
     int32_t n_pairs;
-    __device__ __forceinline__ int64_t count() const {
-        return (int64_t)n_pairs * p.n_layers * p.runs_per_block * p.chunks_per_run;
+    __device__ __forceinline__ int64_t items_per_pair() const {
+        return (int64_t)p.planes * p.head_units * p.row_groups * p.col_chunks;
     }
+    __device__ __forceinline__ int64_t count() const { return (int64_t)n_pairs * p.n_layers * items_per_pair(); }
     // n_rows == 0 marks a skipped pair.
     __device__ __forceinline__ Item operator()(int64_t w) const {
-        const int32_t chunk = (int32_t)(w % p.chunks_per_run);
-        int64_t t = w / p.chunks_per_run;
-        const int32_t run = (int32_t)(t % p.runs_per_block);
-        t /= p.runs_per_block;
+        const int32_t col = (int32_t)(w % p.col_chunks);
+        int64_t t = w / p.col_chunks;
+        const int32_t rg = (int32_t)(t % p.row_groups);
+        t /= p.row_groups;
+        const int32_t hu = (int32_t)(t % p.head_units);
+        t /= p.head_units;
+        const int32_t c = (int32_t)(t % p.planes);
+        t /= p.planes;
         const int32_t pair = (int32_t)(t % n_pairs);
         const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
         const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
         Item it;
-        it.n_rows = 1;
-        it.row_bytes = (int32_t)p.chunk_bytes;
-        it.src_pitch = it.dst_pitch = 0;
-        if (ids.x < 0 || ids.y < 0) {  // the table rewrite already reported this one
-            it.n_rows = 0;
-            it.src = nullptr;
-            it.dst = nullptr;
-            return it;
-        }
+        it.src_pitch = p.src_row_pitch;
+        it.dst_pitch = p.dst_row_pitch;
+        it.n_rows = 0;
+        it.row_bytes = 0;
+        it.src = nullptr;
+        it.dst = nullptr;
+        if (ids.x < 0 || ids.y < 0) return it;  // the table rewrite already reported this one
         if (ids.x >= p.nb_src || ids.y >= p.nb_dst) {
-            if (run == 0 && chunk == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
-            it.n_rows = 0;
-            it.src = nullptr;
-            it.dst = nullptr;
+            if (hu == 0 && c == 0 && rg == 0 && col == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
             return it;
         }
-        const int32_t h0 = run * p.heads_per_run;  // first header of the run
+        const int32_t h0 = hu * p.heads_per_unit;  // first header of the unit
         const int32_t ra = h0 / p.heads_src, ha = h0 - ra * p.heads_src;
         const int32_t rb = h0 / p.heads_dst, hb = h0 - rb * p.heads_dst;
-        const int64_t in_run = (int64_t)chunk * p.chunk_bytes;
-        it.src = p.src[ra] + layer * p.src_layer_stride + ((int64_t)ids.x * p.heads_src + ha) * p.unit_bytes + in_run;
-        it.dst = p.dst[rb] + layer * p.dst_layer_stride + ((int64_t)ids.y * p.heads_dst + hb) * p.unit_bytes + in_run;
+        const int32_t r0 = rg * p.rows_per_item;
+        const int64_t in_row = (int64_t)col * p.chunk_bytes;
+        it.n_rows = min(p.rows_per_item, p.rows - r0);
+        it.row_bytes = p.chunk_bytes;
+        it.src = p.src[ra] + layer * p.src_layer_stride +
+                 pool_offset(p.src_token_major, p.nb_src, p.heads_src, p.block_tokens, p.vec_bytes, ids.x, ha, c) +
+                 r0 * p.src_row_pitch + in_row;
+        it.dst = p.dst[rb] + layer * p.dst_layer_stride +
+                 pool_offset(p.dst_token_major, p.nb_dst, p.heads_dst, p.block_tokens, p.vec_bytes, ids.y, hb, c) +
+                 r0 * p.dst_row_pitch + in_row;
         return it;
     }
 };
@@ -138,8 +158,22 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     p.pairs = d_pairs;
     p.num_pairs = d_num_pairs;
     p.status = d_status;
-    p.unit_bytes = plan->unit_bytes;
-    p.chunk_bytes = plan->chunk_bytes;
+    const KvGeom& g = plan->kv;
+    p.vec_bytes = plan->vec_bytes;
+    p.row_bytes = g.row_bytes;
+    p.src_row_pitch = g.src_row_pitch;
+    p.dst_row_pitch = g.dst_row_pitch;
+    p.block_tokens = plan->src.block_tokens;
+    p.src_token_major = plan->src.kv_order == AMOEBA_KV_TOKEN_MAJOR;
+    p.dst_token_major = plan->dst.kv_order == AMOEBA_KV_TOKEN_MAJOR;
+    p.heads_per_unit = g.heads_per_unit;
+    p.head_units = g.head_units;
+    p.planes = g.planes;
+    p.rows = g.rows;
+    p.rows_per_item = g.rows_per_item;
+    p.row_groups = g.row_groups;
+    p.col_chunks = g.col_chunks;
+    p.chunk_bytes = g.chunk_bytes;
     p.src_layer_stride = plan->src_layer_stride;
     p.dst_layer_stride = plan->dst_layer_stride;
     p.pairs_cap = pairs_cap;
@@ -149,14 +183,11 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     p.nb_dst = plan->dst.num_blocks;
     p.heads_src = plan->heads_src;
     p.heads_dst = plan->heads_dst;
-    p.heads_per_run = plan->heads_per_run;
-    p.runs_per_block = plan->runs_per_block;
-    p.chunks_per_run = (int32_t)(plan->run_bytes / plan->chunk_bytes);
 
     DeviceInfo dev;
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * p.runs_per_block * p.chunks_per_run;
+    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * g.planes * g.head_units * g.row_groups * g.col_chunks;
     cudaError_t e;
     const KernelOpts& opt = plan->opt.kv;
     const int path = opt.copy_path ? opt.copy_path : kKvDefaults.copy_path;
@@ -166,7 +197,7 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
         kv_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
         e = cudaGetLastError();
     } else {
-        const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)plan->chunk_bytes);
+        const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)g.item_bytes);
         const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
         auto kernel = path == 3 ? kv_reshard_pair : kv_reshard_bulk;
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);

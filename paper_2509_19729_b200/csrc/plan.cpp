@@ -26,7 +26,7 @@ static amoeba_status check_layout(const amoeba_layout& l) {
         m.intermediate <= 0 || l.tp <= 0 || l.block_tokens <= 0 || l.num_blocks <= 0 || l.kv_layer_stride_bytes < 0)
         return AMOEBA_ERR_INVALID_ARG;
     if (m.elem_bytes != 2) return AMOEBA_ERR_UNSUPPORTED;
-    if (l.kv_order != AMOEBA_KV_HEAD_MAJOR) return AMOEBA_ERR_UNSUPPORTED;
+    if (l.kv_order != AMOEBA_KV_HEAD_MAJOR && l.kv_order != AMOEBA_KV_TOKEN_MAJOR) return AMOEBA_ERR_UNSUPPORTED;
     if (l.tp > AMOEBA_MAX_TP) return AMOEBA_ERR_UNSUPPORTED;
     // Even partition of the headers and of the FFN width over the workers; K/V header replication for
     // tp > num_kv_heads is not a re-layout of existing state and is not handled.
@@ -46,7 +46,37 @@ amoeba_status finalize_chunks(amoeba_plan* p) {
     const int64_t kv_cap = p->opt.kv.chunk_bytes > 0 ? p->opt.kv.chunk_bytes : kDefaultKvChunk;
     const int64_t cap = p->opt.w.chunk_bytes > 0 ? p->opt.w.chunk_bytes : kDefaultWChunk;
     if (cap < 16 || cap % 16 || kv_cap < 16 || kv_cap % 16) return AMOEBA_ERR_INVALID_ARG;
-    p->chunk_bytes = chunk_of(p->run_bytes, kv_cap);
+    // KV work items: cut a unit's rows into column chunks (long rows) or group whole rows (short rows).
+    KvGeom& g = p->kv;
+    const bool src_tok = p->src.kv_order == AMOEBA_KV_TOKEN_MAJOR, dst_tok = p->dst.kv_order == AMOEBA_KV_TOKEN_MAJOR;
+    const int32_t T = p->src.block_tokens;
+    if (!src_tok && !dst_tok) {  // a run of headers with K and V is contiguous on both sides
+        g.planes = 1;
+        g.heads_per_unit = p->heads_per_run;
+        g.rows = 1;
+        g.row_bytes = p->run_bytes;
+        g.src_row_pitch = g.dst_row_pitch = p->run_bytes;
+    } else {
+        g.planes = 2;
+        g.heads_per_unit = (src_tok && dst_tok) ? p->heads_per_run : 1;
+        g.rows = T;
+        g.row_bytes = g.heads_per_unit * p->vec_bytes;
+        g.src_row_pitch = src_tok ? p->heads_src * p->vec_bytes : p->vec_bytes;
+        g.dst_row_pitch = dst_tok ? p->heads_dst * p->vec_bytes : p->vec_bytes;
+    }
+    g.head_units = p->src.model.num_kv_heads / g.heads_per_unit;
+    if (g.row_bytes > kv_cap) {
+        g.rows_per_item = 1;
+        g.chunk_bytes = (int32_t)chunk_of(g.row_bytes, kv_cap);
+        g.col_chunks = (int32_t)(g.row_bytes / g.chunk_bytes);
+    } else {
+        g.rows_per_item = (int32_t)std::min<int64_t>(g.rows, std::max<int64_t>(1, kv_cap / g.row_bytes));
+        g.chunk_bytes = (int32_t)g.row_bytes;
+        g.col_chunks = 1;
+    }
+    g.row_groups = (g.rows + g.rows_per_item - 1) / g.rows_per_item;
+    g.item_bytes = (int64_t)g.rows_per_item * g.chunk_bytes;
+    p->chunk_bytes = g.item_bytes;
     p->wdev.clear();
     int64_t item = 0;
     for (const amoeba_weight_desc& d : p->wdescs) {
@@ -162,6 +192,7 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
     p->heads_dst = m.num_kv_heads / b;
     p->heads_per_run = std::gcd(p->heads_src, p->heads_dst);
     p->runs_per_block = m.num_kv_heads / p->heads_per_run;
+    p->vec_bytes = (int64_t)m.head_dim * e;
     p->unit_bytes = 2 * (int64_t)src->block_tokens * m.head_dim * e;
     p->run_bytes = p->heads_per_run * p->unit_bytes;
     p->src_block_bytes = p->heads_src * p->unit_bytes;
@@ -173,7 +204,9 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
         delete p;
         return AMOEBA_ERR_INVALID_ARG;
     }
-    if (p->unit_bytes % 16 || p->src_layer_stride % 16 || p->dst_layer_stride % 16) {
+    const bool any_token_major = src->kv_order == AMOEBA_KV_TOKEN_MAJOR || dst->kv_order == AMOEBA_KV_TOKEN_MAJOR;
+    if (p->unit_bytes % 16 || p->src_layer_stride % 16 || p->dst_layer_stride % 16 ||
+        (any_token_major && p->vec_bytes % 16)) {
         delete p;
         return AMOEBA_ERR_ALIGNMENT;
     }

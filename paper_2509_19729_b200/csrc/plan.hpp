@@ -42,6 +42,26 @@ struct Options {
     KernelOpts kv, w;
 };
 
+// How the KV copy of one (block pair, layer) is cut into 2-D work items.  A "unit" is the largest piece that is a
+// regular 2-D copy on both sides: `rows` rows of `row_bytes`, consecutive rows `src_row_pitch` / `dst_row_pitch`
+// apart.  It covers `heads_per_unit` consecutive headers and either both of K and V (planes == 1) or one of them.
+//   both sides header-centric : unit = one run of headers, K and V together, one contiguous row
+//   both sides token-first    : unit = one run of headers of K or of V; one row per token
+//   mixed orders              : unit = one header of K or of V; one row per token (head_dim elements)
+struct KvGeom {
+    int32_t planes;          // 1: a unit spans K and V; 2: K and V are separate units
+    int32_t heads_per_unit;  // consecutive headers per unit
+    int32_t head_units;      // num_kv_heads / heads_per_unit
+    int32_t rows;            // rows per unit (1 or block_tokens)
+    int64_t row_bytes;
+    int64_t src_row_pitch, dst_row_pitch;
+    int32_t rows_per_item;   // rows one work item covers (1 when a row is split into column chunks)
+    int32_t row_groups;      // ceil(rows / rows_per_item)
+    int32_t col_chunks;      // work items along a row
+    int32_t chunk_bytes;     // bytes per column chunk (divides row_bytes)
+    int64_t item_bytes;      // largest work item
+};
+
 }  // namespace amoeba
 
 struct amoeba_plan {
@@ -50,7 +70,9 @@ struct amoeba_plan {
     int32_t heads_src, heads_dst;  // K/V headers per source / destination worker
     int32_t heads_per_run, runs_per_block;
     int64_t unit_bytes;  // one (block, header): 2 * T * D * e
-    int64_t run_bytes, chunk_bytes;  // chunk_bytes: KV work item
+    int64_t run_bytes, chunk_bytes;  // chunk_bytes: largest KV work item
+    int64_t vec_bytes;   // one (token, header): D * e
+    amoeba::KvGeom kv;
     int64_t src_block_bytes, dst_block_bytes, src_layer_stride, dst_layer_stride;
     // weights
     std::vector<amoeba_weight_desc> wdescs;  // public form

@@ -36,11 +36,14 @@ class Session:
     def __init__(self, model: dict, a: int, b: int, NB_src: int, NB_dst: int, num_seqs: int, max_blocks_per_seq: int,
                  pairs_cap: int, kv_layers: Optional[int] = None, kv: bool = True, weights: bool = True,
                  fused_qkv: bool = True, fused_gate_up: bool = True, block_tokens: int = 16, device="cuda:0",
-                 dst_fill: Optional[int] = 0xA5):
+                 dst_fill: Optional[int] = 0xA5, src_kv_order: int = A.KV_HEAD_MAJOR,
+                 dst_kv_order: int = A.KV_HEAD_MAJOR):
         self.model, self.a, self.b = model, a, b
         self.device = torch.device(device)
-        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up)
-        self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up)
+        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up,
+                                        kv_order=src_kv_order)
+        self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up,
+                                        kv_order=dst_kv_order)
         self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
         self.info = A.amoeba_plan_kv_info(self.plan)
         self.L = model["L"]

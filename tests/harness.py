@@ -16,10 +16,11 @@ class Case:
 
 def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_slack=0.25, dst_occupied=0.3, seed=0,
               fused_qkv=True, fused_gate_up=True, weights=True, kv=True, dtype="bf16", free_override=None,
-              src_bt_override=None, pairs_cap=None):
+              src_bt_override=None, pairs_cap=None, src_order=0, dst_order=0):
     """Seeded inputs + the oracle's expected outputs for one TP a->b transformation."""
     c = Case()
     c.model, c.a, c.b, c.T, c.fq, c.fg = model, a, b, T, fused_qkv, fused_gate_up
+    c.src_order, c.dst_order = src_order, dst_order  # 0 header-centric, 1 token-first (same codes on both sides)
     cfg = dict(model=model, dtype=dtype, S=len(seq_lens), src_free=src_free, dst_form=dst_form, dst_slack=dst_slack,
                dst_occupied=dst_occupied)
     st = wl.draw_kv_state(cfg, seed=seed, name="case", seq_lens=np.maximum(np.asarray(seq_lens), 0), T=T)
@@ -40,7 +41,8 @@ def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_sl
         G = int(st["blocks_per_seq"].sum()) * T
         c.KV = g.integers(0, 65536, size=(L, G, model["Hkv"], 2, model["D"]), dtype=np.uint16)
         valid_lens = np.maximum(c.seq_lens, 0)
-        c.src_pools = oracle.kv_shard(c.KV, model, T, a, c.NB_src, valid_lens, st["src_bt"], fill=0x5A5A)
+        c.src_pools = oracle.kv_shard(c.KV, model, T, a, c.NB_src, valid_lens, st["src_bt"], fill=0x5A5A,
+                                      order=src_order)
     # expected tables
     c.exp_dst_bt, c.exp_pairs, c.exp_n, c.exp_left, c.exp_status = oracle.assign_blocks(
         c.seq_lens, T, c.src_bt, c.NB_src, c.NB_dst, free_list=c.free_list, free_mask=c.free_mask,
@@ -50,10 +52,10 @@ def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_sl
                            for _ in range(b)]
         if c.exp_status == 0:
             oracle.kv_transform(model, T, c.seq_lens, a, c.NB_src, c.src_bt, c.src_pools, b, c.NB_dst, c.exp_dst_bt,
-                                c.exp_dst_pools)
+                                c.exp_dst_pools, src_order=src_order, dst_order=dst_order)
         else:
             st2 = oracle.kv_copy_pairs(model, T, a, c.NB_src, c.src_pools, b, c.NB_dst, c.exp_dst_pools, c.exp_pairs,
-                                       c.exp_n, status=c.exp_status)
+                                       c.exp_n, status=c.exp_status, src_order=src_order, dst_order=dst_order)
             assert st2 == c.exp_status
     c.weights = weights
     if weights:
@@ -74,7 +76,8 @@ def run_case(c, copy_path=None, options=(), device="cuda:0", steps=1):
     from paper_2509_19729_b200.session import Session
 
     s = Session(c.model, c.a, c.b, c.NB_src, c.NB_dst, len(c.seq_lens), c.maxb, c.pairs_cap, kv=c.kv,
-                weights=c.weights, fused_qkv=c.fq, fused_gate_up=c.fg, block_tokens=c.T, device=device)
+                weights=c.weights, fused_qkv=c.fq, fused_gate_up=c.fg, block_tokens=c.T, device=device,
+                src_kv_order=c.src_order, dst_kv_order=c.dst_order)
     if copy_path is not None:
         s.set_option(A.OPT_COPY_PATH, copy_path)
     for opt, val in options:

@@ -15,12 +15,33 @@ pytestmark = pytest.mark.gpu
 FULL = ["llama3_8b_1to4", "llama3_8b_2to8", "llama2_7b_1to2", "llama2_13b_4to1", "llama3_70b_slice_8to2"]
 
 
-def _block_view(pool, n_layers, NB):
-    return pool.view(n_layers, NB, -1)  # [layer][block][bytes of one block in this worker's pool]
+CASES = [(n, "head") for n in FULL] + [("llama3_8b_1to4", "token"), ("llama3_70b_slice_8to2", "token2head"),
+                                       ("llama2_7b_1to2", "head2token")]
 
 
-@pytest.mark.parametrize("name", FULL)
-def test_full_size_config(name, oracle):
+class _BlockView:
+    """One worker's pool addressed as [layer, block] -> the bytes of that block, as a pool holding only that block
+    would store them (header-centric: one slab per block; token-first: the block's K slab then its V slab)."""
+
+    def __init__(self, pool, n_layers, NB, token_first):
+        self.tf = token_first
+        self.v = pool.view(n_layers, 2, NB, -1) if token_first else pool.view(n_layers, NB, -1)
+
+    def __getitem__(self, idx):
+        l, blk = idx
+        return self.v[l, :, blk].reshape(-1) if self.tf else self.v[l, blk]
+
+    def layer_blocks(self, l, NB, ids):
+        """int64 words of the given blocks of layer l, [len(ids), words]."""
+        import torch
+
+        if self.tf:
+            return torch.cat([self.v[l, c].view(torch.int64).view(NB, -1).index_select(0, ids) for c in range(2)], 1)
+        return self.v[l].view(torch.int64).view(NB, -1).index_select(0, ids)
+
+
+@pytest.mark.parametrize("name,kv_order", CASES)
+def test_full_size_config(name, kv_order, oracle):
     import torch
 
     import bench
@@ -29,7 +50,8 @@ def test_full_size_config(name, oracle):
     cfg = wl.CONFIGS[name]
     m, a, b, T = cfg["model"], cfg["a"], cfg["b"], wl.BLOCK_TOKENS
     device = torch.device("cuda:0")
-    s, st = bench.build_session(name, device)
+    so, do = bench.KV_ORDERS[kv_order]
+    s, st = bench.build_session(name, device, kv_order=kv_order)
     try:
         s.status.zero_()
         s.step()
@@ -47,8 +69,8 @@ def test_full_size_config(name, oracle):
 
         # ---- KV: sampled blocks, each re-laid-out by the oracle on its own
         Lkv = s.kv_layers
-        src_v = [_block_view(p, Lkv, st["NB_src"]) for p in s.src_pools]
-        dst_v = [_block_view(p, Lkv, st["NB_dst"]) for p in s.dst_pools]
+        src_v = [_BlockView(p, Lkv, st["NB_src"], so == 1) for p in s.src_pools]
+        dst_v = [_BlockView(p, Lkv, st["NB_dst"], do == 1) for p in s.dst_pools]
         g = np.random.default_rng(7)
         one = dict(m, L=1)
         seqs = np.flatnonzero(st["blocks_per_seq"] > 0)
@@ -59,7 +81,7 @@ def test_full_size_config(name, oracle):
             sid, did = int(st["src_bt"][q, i]), int(dst_bt[q, i])
             src1 = [v[l, sid].cpu().numpy().view(np.uint16).copy() for v in src_v]  # NB = 1 pools
             exp1 = [np.zeros(d[l, did].numel() // 2, np.uint16) for d in dst_v]
-            oracle.kv_transform(one, T, [T], a, 1, [[0]], src1, b, 1, [[0]], exp1)
+            oracle.kv_transform(one, T, [T], a, 1, [[0]], src1, b, 1, [[0]], exp1, src_order=so, dst_order=do)
             for r in range(b):
                 got = dst_v[r][l, did].cpu().numpy().view(np.uint16)
                 assert np.array_equal(got, exp1[r]), (name, l, q, i, r)
@@ -77,10 +99,8 @@ def test_full_size_config(name, oracle):
         live_src = torch.as_tensor(exp_pairs[:, 0].astype(np.int64), device=device)
         live_dst = torch.as_tensor(exp_pairs[:, 1].astype(np.int64), device=device)
         for l in sorted(set(int(x) for x in g.integers(Lkv, size=3))):
-            ssum = sum(int(v[l].view(torch.int64).view(st["NB_src"], -1).index_select(0, live_src).sum().item())
-                       for v in src_v)
-            dsum = sum(int(v[l].view(torch.int64).view(st["NB_dst"], -1).index_select(0, live_dst).sum().item())
-                       for v in dst_v)
+            ssum = sum(int(v.layer_blocks(l, st["NB_src"], live_src).sum().item()) for v in src_v)
+            dsum = sum(int(v.layer_blocks(l, st["NB_dst"], live_dst).sum().item()) for v in dst_v)
             assert (ssum - dsum) % (1 << 64) == 0
 
         # ---- weights: whole comparison of sampled layers

@@ -199,3 +199,43 @@ def test_side_stream():
         s.step(st)
     st.synchronize()
     check_case(c, s)
+
+
+# ---- token-first storage order (Sec. 3.1: the layout of mainstream engines) on either or both sides
+HC, TF = 0, 1
+ORDERS = [(TF, TF), (TF, HC), (HC, TF)]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("so,do", ORDERS)
+@pytest.mark.parametrize("a,b", [(1, 4), (4, 1), (2, 8), (8, 2), (2, 2), (1, 1)])
+def test_token_first_orders_gqa(path, so, do, a, b):
+    lens = [1, 16, 17, 300, 0, 77, 513, 5]
+    c = make_case(GQA, a, b, lens, weights=False, seed=a * 16 + b + 100 * so + 1000 * do, src_order=so, dst_order=do)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("so,do", ORDERS)
+@pytest.mark.parametrize("a,b", [(4, 5), (8, 5), (10, 4), (20, 1), (5, 5)])
+def test_token_first_non_nested_partitions(path, so, do, a, b):
+    c = make_case(SMALL40, a, b, [33, 7, 0, 64, 129], T=8, weights=False, seed=a * 64 + b, src_order=so, dst_order=do)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("so,do", ORDERS)
+@pytest.mark.parametrize("chunk", [256, 1024, 4096, 32768])
+def test_token_first_chunk_sizes(path, so, do, chunk):
+    """Work items from a quarter of a token row up to several rows: column chunks, row groups and ragged groups."""
+    import paper_2509_19729_b200 as A
+
+    wide = dict(L=2, hidden=256, Hq=16, Hkv=16, D=64, I=512)  # 1->2: token rows of 8 headers = 1 KiB
+    c = make_case(wide, 1, 2, [100, 3, 48], T=12, weights=False, seed=chunk, src_order=so, dst_order=do)
+    check_case(c, run_case(c, path, options=[(A.OPT_CHUNK_BYTES, chunk)]))
+
+
+def test_token_first_full_transformation_with_weights_and_mask():
+    lens = list(np.random.default_rng(4).integers(1, 400, size=60))
+    c = make_case(GQA, 2, 4, lens, dst_form="mask", dst_occupied=0.3, src_free=0.3, seed=21, src_order=TF, dst_order=TF)
+    check_case(c, run_case(c))

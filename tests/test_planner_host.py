@@ -122,3 +122,36 @@ def test_no_device_means_cuda_error_not_a_fallback():
     with pytest.raises(A.AmoebaError) as e:  # non-null fake addresses, aligned: passes validation, then no device
         A.amoeba_reshard_kv(plan, [4096, 8192], [12288], 4096, 4096, 4, 0, 1, 4096, stream=0)
     assert e.value.status == A.ERR_CUDA
+
+
+@pytest.mark.parametrize("so,do", [(0, 0), (1, 1), (1, 0), (0, 1)])
+@pytest.mark.parametrize("a,b", [(1, 4), (8, 2), (4, 5), (2, 2)])
+def test_kv_geometry_covers_each_block_once_for_both_orders(so, do, a, b):
+    """The planner's work-item size never exceeds the cap and the plan accepts both storage orders on both sides."""
+    import paper_2509_19729_b200 as A
+
+    model = dict(L=2, hidden=320, Hq=40, Hkv=40, D=16, I=640)
+    src = A.make_layout(model, a, 64, block_tokens=8, kv_order=so)
+    dst = A.make_layout(model, b, 64, block_tokens=8, kv_order=do)
+    plan = A.amoeba_plan_create(src, dst)
+    info = A.amoeba_plan_kv_info(plan)
+    assert 16 <= info.chunk_bytes <= 8192 and info.chunk_bytes % 16 == 0
+    for cap in (16, 64, 4096):
+        A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, cap)
+        assert A.amoeba_plan_kv_info(plan).chunk_bytes <= max(cap, 16)
+    kv_rw, _ = A.amoeba_plan_bytes(plan, 10)
+    assert kv_rw == 2 * 10 * 2 * 40 * 2 * 8 * 16 * 2  # both ways x blocks x layers x Hkv x (K,V) x T x D x e
+
+
+def test_unknown_kv_order_is_unsupported():
+    import paper_2509_19729_b200 as A
+
+    model = dict(L=1, hidden=64, Hq=4, Hkv=4, D=16, I=128)
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_plan_create(A.make_layout(model, 1, 8, kv_order=2), A.make_layout(model, 2, 8))
+    assert e.value.status == A.ERR_UNSUPPORTED
+    # token-first needs head_dim * elem_bytes to be a multiple of 16
+    odd = dict(model, D=4)
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_plan_create(A.make_layout(odd, 1, 8, kv_order=1), A.make_layout(odd, 2, 8, kv_order=1))
+    assert e.value.status == A.ERR_ALIGNMENT
