@@ -140,6 +140,8 @@ enum {
     AMOEBA_OPT_LAG = 4,         /* path 2: loads issued ahead of stores; path 3: stores kept in flight (< stages) */
     AMOEBA_OPT_WARPS = 5,       /* bulk-copy rings per CTA */
     AMOEBA_OPT_L2_HINT = 6,     /* 1 = none, 2 = loads evict-first, 3 = stores evict-first, 4 = both */
+    AMOEBA_OPT_TENSOR_MAPS = 7, /* KV, bulk-copy paths, token-first sides: 1 = one bulk copy per token row,
+                                   2 = one tiled (tensor-map) copy per work item */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };

@@ -11,6 +11,8 @@
 //   * pair_bulk_ring     a producer warp and a consumer warp share one ring: the producer only issues loads (waits
 //                        on "empty" barriers), the consumer only issues stores (waits on "full" barriers), so the
 //                        split of the ring between loads and stores in flight adapts by itself.
+// In the ring kernels a side of an item may also be one box of a tensor map (tiled TMA), which gathers or scatters
+// many short rows with a single copy instruction.
 // Every wait on an mbarrier is bounded; bulk-group waits only wait for the thread's own stores.
 #pragma once
 #include <cstdint>
@@ -23,6 +25,12 @@ struct Item {
     char* dst;
     int64_t src_pitch, dst_pitch;
     int32_t n_rows, row_bytes;
+    // Bulk-copy rings only: when non-null, that side of the item is one box of a 5-D tensor map instead of rows
+    // (coordinates {0, tok, 0, head, layer}); the box holds exactly n_rows * row_bytes bytes and arrives in / leaves
+    // shared memory in the same dense order as the packed rows.
+    const void* src_map;
+    const void* dst_map;
+    int32_t src_tok, src_head, dst_tok, dst_head, layer;
 };
 
 // Shape of the bulk rings (runtime, chosen by the launcher).
@@ -156,6 +164,37 @@ __device__ __forceinline__ void bulk_s2g(void* gdst, const void* smem_src, uint3
                      "r"(smem_u32(smem_src)), "r"(bytes)
                      : "memory");
 }
+// Tiled (tensor-map) copies of one 5-D box; the innermost coordinate is always 0, so the 16-byte rule on it holds.
+__device__ __forceinline__ void tensor_g2s(void* smem_dst, const void* map, int32_t c1, int32_t c3, int32_t c4,
+                                           uint64_t* bar, bool hint, uint64_t policy) {
+    if (hint)
+        asm volatile(
+            "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+            "[%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;" ::"r"(smem_u32(smem_dst)),
+            "l"(map), "r"(0), "r"(c1), "r"(0), "r"(c3), "r"(c4), "r"(smem_u32(bar)), "l"(policy)
+            : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(smem_u32(smem_dst)),
+            "l"(map), "r"(0), "r"(c1), "r"(0), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+            : "memory");
+}
+__device__ __forceinline__ void tensor_s2g(const void* map, int32_t c1, int32_t c3, int32_t c4, const void* smem_src,
+                                           bool hint, uint64_t policy) {
+    if (hint)
+        asm volatile(
+            "cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group.L2::cache_hint "
+            "[%0, {%1, %2, %3, %4, %5}], [%6], %7;" ::"l"(map),
+            "r"(0), "r"(c1), "r"(0), "r"(c3), "r"(c4), "r"(smem_u32(smem_src)), "l"(policy)
+            : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group "
+            "[%0, {%1, %2, %3, %4, %5}], [%6];" ::"l"(map),
+            "r"(0), "r"(c1), "r"(0), "r"(c3), "r"(c4), "r"(smem_u32(smem_src))
+            : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Wait until at most n of this thread's bulk groups still have shared-memory reads outstanding (n in 0..15).
 __device__ __forceinline__ void bulk_wait_read(int n) {
@@ -188,7 +227,9 @@ constexpr int kMaxStages = 16;
 __device__ __forceinline__ void item_load(const Item& it, char* stage, uint64_t* bar, bool hint, uint64_t policy) {
     const int lane = threadIdx.x & 31;
     if (it.n_rows == 0) return;  // skipped item: the barrier phase completes with 0 bytes expected
-    if (it.n_rows == 1 || it.src_pitch == it.row_bytes) {
+    if (it.src_map) {
+        if (lane == 0) tensor_g2s(stage, it.src_map, it.src_tok, it.src_head, it.layer, bar, hint, policy);
+    } else if (it.n_rows == 1 || it.src_pitch == it.row_bytes) {
         if (lane == 0) bulk_g2s(stage, it.src, (uint32_t)it.n_rows * (uint32_t)it.row_bytes, bar, hint, policy);
     } else {
         for (int r = lane; r < it.n_rows; r += 32)
@@ -198,7 +239,9 @@ __device__ __forceinline__ void item_load(const Item& it, char* stage, uint64_t*
 __device__ __forceinline__ void item_store(const Item& it, const char* stage, bool hint, uint64_t policy) {
     const int lane = threadIdx.x & 31;
     if (it.n_rows == 0) return;
-    if (it.n_rows == 1 || it.dst_pitch == it.row_bytes) {
+    if (it.dst_map) {
+        if (lane == 0) tensor_s2g(it.dst_map, it.dst_tok, it.dst_head, it.layer, stage, hint, policy);
+    } else if (it.n_rows == 1 || it.dst_pitch == it.row_bytes) {
         if (lane == 0) bulk_s2g(it.dst, stage, (uint32_t)it.n_rows * (uint32_t)it.row_bytes, hint, policy);
     } else {
         for (int r = lane; r < it.n_rows; r += 32)

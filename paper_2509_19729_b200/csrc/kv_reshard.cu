@@ -9,7 +9,11 @@
 // together, one contiguous row; with token-first on a side it is one row per token.  Units are cut into copy work
 // items, dealt round-robin to a persistent grid; layer is the slowest index so that concurrently running CTAs touch
 // neighbouring DRAM pages.
+#include <cuda.h>
 #include <cuda_runtime.h>
+
+#include <cstring>
+#include <mutex>
 
 #include "copy_engine.cuh"
 #include "launch.hpp"
@@ -30,6 +34,15 @@ struct KvParams {
     int32_t src_token_major, dst_token_major;
     int32_t heads_src, heads_dst, heads_per_unit, head_units, planes;
     int32_t rows, rows_per_item, row_groups, col_chunks, chunk_bytes;
+    // box items (tensor-map path)
+    int32_t heads_per_run, runs_per_block, box_heads, box_tokens, box_sub_runs, box_tok_groups;
+};
+
+// Tensor maps of the token-first pools, one per worker: dimensions {dim, token of the layer's K or V region,
+// K/V, local header, layer}, box {head_dim, box_tokens, 2, box_heads, 1}.
+struct KvMaps {
+    CUtensorMap src[AMOEBA_MAX_TP];
+    CUtensorMap dst[AMOEBA_MAX_TP];
 };
 
 // Byte offset, inside one layer of a worker's pool, of token 0 of (block, local header, K/V plane).
@@ -60,6 +73,7 @@ struct KvItems {
         const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
         const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
         Item it;
+        it.src_map = it.dst_map = nullptr;
         it.src_pitch = p.src_row_pitch;
         it.dst_pitch = p.dst_row_pitch;
         it.n_rows = 0;
@@ -84,6 +98,65 @@ struct KvItems {
         it.dst = p.dst[rb] + layer * p.dst_layer_stride +
                  pool_offset(p.dst_token_major, p.nb_dst, p.heads_dst, p.block_tokens, p.vec_bytes, ids.y, hb, c) +
                  r0 * p.dst_row_pitch + in_row;
+        return it;
+    }
+};
+
+// Box items: (layer, pair, run, sub-run of headers, token group); K and V travel together.
+struct KvBoxItems {
+    const KvParams& p;
+    const KvMaps& maps;
+    int32_t n_pairs;
+    __device__ __forceinline__ int64_t count() const {
+        return (int64_t)n_pairs * p.n_layers * p.runs_per_block * p.box_sub_runs * p.box_tok_groups;
+    }
+    __device__ __forceinline__ Item operator()(int64_t w) const {
+        const int32_t tg = (int32_t)(w % p.box_tok_groups);
+        int64_t t = w / p.box_tok_groups;
+        const int32_t sub = (int32_t)(t % p.box_sub_runs);
+        t /= p.box_sub_runs;
+        const int32_t run = (int32_t)(t % p.runs_per_block);
+        t /= p.runs_per_block;
+        const int32_t pair = (int32_t)(t % n_pairs);
+        const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
+        const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
+        Item it;
+        it.src_map = it.dst_map = nullptr;
+        it.n_rows = 0;
+        it.row_bytes = 0;
+        it.src = nullptr;
+        it.dst = nullptr;
+        it.src_pitch = it.dst_pitch = (int64_t)p.block_tokens * p.vec_bytes;  // header-centric side: (header, K/V) rows
+        if (ids.x < 0 || ids.y < 0) return it;
+        if (ids.x >= p.nb_src || ids.y >= p.nb_dst) {
+            if (run == 0 && sub == 0 && tg == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+            return it;
+        }
+        const int32_t h0 = run * p.heads_per_run + sub * p.box_heads;
+        const int32_t ra = h0 / p.heads_src, ha = h0 - ra * p.heads_src;
+        const int32_t rb = h0 / p.heads_dst, hb = h0 - rb * p.heads_dst;
+        const int32_t t0 = tg * p.box_tokens;
+        it.n_rows = 2 * p.box_heads;
+        it.row_bytes = (int32_t)(p.box_tokens * p.vec_bytes);
+        it.layer = layer;
+        if (p.src_token_major) {
+            it.src_map = &maps.src[ra];
+            it.src_tok = ids.x * p.block_tokens + t0;
+            it.src_head = ha;
+        } else {
+            it.src = p.src[ra] + layer * p.src_layer_stride +
+                     pool_offset(false, p.nb_src, p.heads_src, p.block_tokens, p.vec_bytes, ids.x, ha, 0) +
+                     t0 * p.vec_bytes;
+        }
+        if (p.dst_token_major) {
+            it.dst_map = &maps.dst[rb];
+            it.dst_tok = ids.y * p.block_tokens + t0;
+            it.dst_head = hb;
+        } else {
+            it.dst = p.dst[rb] + layer * p.dst_layer_stride +
+                     pool_offset(false, p.nb_dst, p.heads_dst, p.block_tokens, p.vec_bytes, ids.y, hb, 0) +
+                     t0 * p.vec_bytes;
+        }
         return it;
     }
 };
@@ -130,6 +203,72 @@ __global__ void __launch_bounds__(1024) kv_reshard_pair(const __grid_constant__ 
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
+// The same two ring kernels over box items (a side that is token-first goes through its tensor map).
+__global__ void __launch_bounds__(1024) kv_reshard_bulk_box(const __grid_constant__ KvParams p,
+                                                            const __grid_constant__ KvMaps maps, const RingShape rs) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)warp * rs.stages * rs.stage_bytes;
+    const KvBoxItems items{p, maps, clamp_pairs(p)};
+    const bool ok = warp_bulk_ring(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
+                                   (int64_t)gridDim.x * nwarps, stages, bars, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
+}
+
+__global__ void __launch_bounds__(1024) kv_reshard_pair_box(const __grid_constant__ KvParams p,
+                                                            const __grid_constant__ KvMaps maps, const RingShape rs) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
+    uint64_t* empty = full + rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
+    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
+    __syncthreads();
+    const KvBoxItems items{p, maps, clamp_pairs(p)};
+    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
+                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link against the driver.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// Tensor map of one worker's token-first pool [layer][K/V][block][token][header][dim] (16-bit elements), with the
+// dimensions ordered {dim, token, K/V, header, layer} so that a box lands in shared memory as
+// [header][K/V][token][dim]: the header-centric order of the same data.
+static bool encode_pool_map(CUtensorMap* out, const void* pool, const amoeba_layout& lay, int64_t layer_stride,
+                            int32_t heads, int64_t vec_bytes, const KvBoxGeom& bx) {
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return false;
+    const cuuint64_t T = (cuuint64_t)lay.block_tokens, NB = (cuuint64_t)lay.num_blocks;
+    const cuuint64_t dims[5] = {(cuuint64_t)lay.model.head_dim, NB * T, 2, (cuuint64_t)heads,
+                                (cuuint64_t)lay.model.num_layers};
+    const cuuint64_t strides[4] = {(cuuint64_t)heads * vec_bytes,           // next token
+                                   NB * T * (cuuint64_t)heads * vec_bytes,   // K region -> V region
+                                   (cuuint64_t)vec_bytes,                    // next header of the same token
+                                   (cuuint64_t)layer_stride};
+    const cuuint32_t box[5] = {(cuuint32_t)lay.model.head_dim, (cuuint32_t)bx.tokens, 2, (cuuint32_t)bx.heads, 1};
+    const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
+    return encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 5, const_cast<void*>(pool), dims, strides, box, elem_strides,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace amoeba
 
 using namespace amoeba;
@@ -174,6 +313,13 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     p.row_groups = g.row_groups;
     p.col_chunks = g.col_chunks;
     p.chunk_bytes = g.chunk_bytes;
+    const KvBoxGeom& bx = plan->kvbox;
+    p.heads_per_run = plan->heads_per_run;
+    p.runs_per_block = plan->runs_per_block;
+    p.box_heads = bx.heads;
+    p.box_tokens = bx.tokens;
+    p.box_sub_runs = bx.sub_runs;
+    p.box_tok_groups = bx.tok_groups;
     p.src_layer_stride = plan->src_layer_stride;
     p.dst_layer_stride = plan->dst_layer_stride;
     p.pairs_cap = pairs_cap;
@@ -187,15 +333,41 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     DeviceInfo dev;
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * g.planes * g.head_units * g.row_groups * g.col_chunks;
     cudaError_t e;
     const KernelOpts& opt = plan->opt.kv;
     const int path = opt.copy_path ? opt.copy_path : kKvDefaults.copy_path;
+    const bool token_side = p.src_token_major || p.dst_token_major;
+    const bool boxes = path != 1 && token_side && bx.usable && opt.tensor_maps != 1;
+    const int64_t items_per_pair = boxes ? (int64_t)p.runs_per_block * bx.sub_runs * bx.tok_groups
+                                         : (int64_t)g.planes * g.head_units * g.row_groups * g.col_chunks;
+    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * items_per_pair;
     if (path == 1) {
         const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 16;
         const int grid = (int)std::min<int64_t>(max_items, (int64_t)dev.sms * per_sm);
         kv_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
         e = cudaGetLastError();
+    } else if (boxes) {
+        KvMaps maps;  // encoded per call: the pool addresses are arguments of this call
+        std::memset(&maps, 0, sizeof(maps));
+        if (p.src_token_major)
+            for (int r = 0; r < plan->src.tp; ++r)
+                if (!encode_pool_map(&maps.src[r], src_pools[r], plan->src, plan->src_layer_stride, plan->heads_src,
+                                     plan->vec_bytes, bx))
+                    return AMOEBA_ERR_CUDA;
+        if (p.dst_token_major)
+            for (int r = 0; r < plan->dst.tp; ++r)
+                if (!encode_pool_map(&maps.dst[r], dst_pools[r], plan->dst, plan->dst_layer_stride, plan->heads_dst,
+                                     plan->vec_bytes, bx))
+                    return AMOEBA_ERR_CUDA;
+        const int stage_bytes = (int)((bx.item_bytes + 127) / 128 * 128);  // tiled copies want 128-byte aligned stages
+        const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, stage_bytes);
+        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+        auto kernel = path == 3 ? kv_reshard_pair_box : kv_reshard_bulk_box;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+        if (e == cudaSuccess) {
+            kernel<<<grid, bs.threads, bs.smem, stream>>>(p, maps, bs.ring);
+            e = cudaGetLastError();
+        }
     } else {
         const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)g.item_bytes);
         const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);

@@ -77,6 +77,31 @@ amoeba_status finalize_chunks(amoeba_plan* p) {
     g.row_groups = (g.rows + g.rows_per_item - 1) / g.rows_per_item;
     g.item_bytes = (int64_t)g.rows_per_item * g.chunk_bytes;
     p->chunk_bytes = g.item_bytes;
+
+    // Box items for the tensor-map path (only meaningful when a side is token-first).
+    KvBoxGeom& bx = p->kvbox;
+    bx = KvBoxGeom{};
+    const int32_t D = p->src.model.head_dim;
+    if ((src_tok || dst_tok) && D <= 256 && p->vec_bytes % 16 == 0) {
+        bx.usable = 1;
+        auto largest_divisor = [](int64_t n, int64_t limit) {
+            int64_t best = 1;
+            for (int64_t d = 1; d <= n && d <= limit; ++d)
+                if (n % d == 0) best = d;
+            return best;
+        };
+        if (p->unit_bytes <= kv_cap) {
+            bx.tokens = T;
+            bx.heads = (int32_t)largest_divisor(p->heads_per_run, std::min<int64_t>(128, kv_cap / p->unit_bytes));
+        } else {
+            bx.heads = 1;
+            bx.tokens = (int32_t)largest_divisor(T, std::min<int64_t>(256, std::max<int64_t>(1, kv_cap / (2 * p->vec_bytes))));
+        }
+        if (T > 256 && bx.tokens == T) bx.tokens = (int32_t)largest_divisor(T, 256);
+        bx.sub_runs = p->heads_per_run / bx.heads;
+        bx.tok_groups = T / bx.tokens;
+        bx.item_bytes = 2 * (int64_t)bx.heads * bx.tokens * p->vec_bytes;
+    }
     p->wdev.clear();
     int64_t item = 0;
     for (const amoeba_weight_desc& d : p->wdescs) {
@@ -353,6 +378,10 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
             case AMOEBA_OPT_L2_HINT:
                 if (value > 4) return AMOEBA_ERR_INVALID_ARG;
                 k->hint = (int)value;
+                break;
+            case AMOEBA_OPT_TENSOR_MAPS:
+                if (value > 2) return AMOEBA_ERR_INVALID_ARG;
+                k->tensor_maps = (int)value;
                 break;
             default:
                 return AMOEBA_ERR_INVALID_ARG;

@@ -27,6 +27,20 @@ struct WDescDev {
     int32_t pad;
 };
 
+// Box geometry of the KV copy when a side is token-first and the bulk-copy kernels address it through a tensor map
+// (tiled TMA): a work item is `heads` consecutive headers x K and V x `tokens` consecutive tokens of one block.  On a
+// token-first side that is one 5-D box {dim, token, K/V, header, layer} of the worker's pool; on a header-centric
+// side it is 2*heads rows of tokens*vec_bytes, consecutive rows block_tokens*vec_bytes apart.  In shared memory
+// both are the same dense [header][K/V][token][dim] tile, so one load and one store move the item.
+struct KvBoxGeom {
+    int32_t usable;      // 0: shape outside the tensor-map limits, row copies are used instead
+    int32_t heads;       // headers per item (divides the run length)
+    int32_t tokens;      // tokens per item (divides block_tokens)
+    int32_t sub_runs;    // items along a run of headers
+    int32_t tok_groups;  // items along the tokens of a block
+    int64_t item_bytes;
+};
+
 // Tuning knobs of one copy kernel; 0 = use the kernel's default.
 struct KernelOpts {
     int copy_path = 0;    // 1 vector ld/st, 2 bulk-copy ring per warp, 3 bulk-copy producer/consumer ring
@@ -36,6 +50,7 @@ struct KernelOpts {
     int lag = 0;          // loads ahead of stores (path 2) / stores kept in flight (path 3)
     int warps = 0;        // rings per CTA
     int hint = 0;         // 1 + bit mask: bit 0 loads evict-first, bit 1 stores evict-first (0 = default)
+    int tensor_maps = 0;  // KV only: 1 = row copies on token-first sides, 2 = tensor-map boxes (0 = default)
 };
 
 struct Options {
@@ -73,6 +88,7 @@ struct amoeba_plan {
     int64_t run_bytes, chunk_bytes;  // chunk_bytes: largest KV work item
     int64_t vec_bytes;   // one (token, header): D * e
     amoeba::KvGeom kv;
+    amoeba::KvBoxGeom kvbox;
     int64_t src_block_bytes, dst_block_bytes, src_layer_stride, dst_layer_stride;
     // weights
     std::vector<amoeba_weight_desc> wdescs;  // public form

@@ -35,6 +35,7 @@ struct WItems {
         const int32_t r0 = rg * d.rows_per_item;
         const int64_t off = (int64_t)cc * d.chunk_bytes;
         Item it;
+        it.src_map = it.dst_map = nullptr;
         it.n_rows = min(d.rows_per_item, d.n_rows - r0);
         it.row_bytes = (int32_t)min((int64_t)d.chunk_bytes, d.row_bytes - off);
         it.src_pitch = d.src_pitch;

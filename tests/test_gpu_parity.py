@@ -204,35 +204,55 @@ def test_side_stream():
 # ---- token-first storage order (Sec. 3.1: the layout of mainstream engines) on either or both sides
 HC, TF = 0, 1
 ORDERS = [(TF, TF), (TF, HC), (HC, TF)]
+# (copy path, token-first addressing in the bulk-copy kernels: 1 = one bulk copy per token row, 2 = tensor-map boxes)
+VARIANTS = [(LDST, 0), (BULK, 1), (BULK, 2), (PAIR, 1), (PAIR, 2)]
 
 
-@pytest.mark.parametrize("path", PATHS)
+def _opts(tm, extra=()):
+    import paper_2509_19729_b200 as A
+
+    return ([(A.OPT_TENSOR_MAPS, tm)] if tm else []) + list(extra)
+
+
+@pytest.mark.parametrize("path,tm", VARIANTS)
 @pytest.mark.parametrize("so,do", ORDERS)
 @pytest.mark.parametrize("a,b", [(1, 4), (4, 1), (2, 8), (8, 2), (2, 2), (1, 1)])
-def test_token_first_orders_gqa(path, so, do, a, b):
+def test_token_first_orders_gqa(path, tm, so, do, a, b):
     lens = [1, 16, 17, 300, 0, 77, 513, 5]
     c = make_case(GQA, a, b, lens, weights=False, seed=a * 16 + b + 100 * so + 1000 * do, src_order=so, dst_order=do)
-    check_case(c, run_case(c, path))
+    check_case(c, run_case(c, path, options=_opts(tm)))
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path,tm", VARIANTS)
 @pytest.mark.parametrize("so,do", ORDERS)
 @pytest.mark.parametrize("a,b", [(4, 5), (8, 5), (10, 4), (20, 1), (5, 5)])
-def test_token_first_non_nested_partitions(path, so, do, a, b):
+def test_token_first_non_nested_partitions(path, tm, so, do, a, b):
     c = make_case(SMALL40, a, b, [33, 7, 0, 64, 129], T=8, weights=False, seed=a * 64 + b, src_order=so, dst_order=do)
-    check_case(c, run_case(c, path))
+    check_case(c, run_case(c, path, options=_opts(tm)))
 
 
-@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("path,tm", VARIANTS)
 @pytest.mark.parametrize("so,do", ORDERS)
 @pytest.mark.parametrize("chunk", [256, 1024, 4096, 32768])
-def test_token_first_chunk_sizes(path, so, do, chunk):
-    """Work items from a quarter of a token row up to several rows: column chunks, row groups and ragged groups."""
+def test_token_first_chunk_sizes(path, tm, so, do, chunk):
+    """Work items from a quarter of a token row up to several rows (row copies) and from one token of one header up to
+    a whole run of headers (boxes): column chunks, row groups, ragged groups, token groups, header groups."""
     import paper_2509_19729_b200 as A
 
     wide = dict(L=2, hidden=256, Hq=16, Hkv=16, D=64, I=512)  # 1->2: token rows of 8 headers = 1 KiB
     c = make_case(wide, 1, 2, [100, 3, 48], T=12, weights=False, seed=chunk, src_order=so, dst_order=do)
-    check_case(c, run_case(c, path, options=[(A.OPT_CHUNK_BYTES, chunk)]))
+    check_case(c, run_case(c, path, options=_opts(tm, [(A.OPT_CHUNK_BYTES, chunk)])))
+
+
+@pytest.mark.parametrize("so,do", ORDERS)
+def test_token_first_bad_block_ids_are_skipped(so, do):
+    """A pair with an id outside its pool moves nothing and reports BAD_BLOCK_ID, with boxes as with rows."""
+    lens = [40, 40, 40]
+    c0 = make_case(dict(GQA, L=1), 2, 4, lens, weights=False, seed=3)
+    bt = c0.src_bt.copy()
+    bt[1, 1] = c0.NB_src + 5
+    c = make_case(dict(GQA, L=1), 2, 4, lens, weights=False, seed=3, src_bt_override=bt, src_order=so, dst_order=do)
+    check_case(c, run_case(c))
 
 
 def test_token_first_full_transformation_with_weights_and_mask():
