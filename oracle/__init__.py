@@ -243,3 +243,27 @@ def assign_blocks(seq_lens, T, src_bt, NB_src, NB_dst, free_list=None, free_mask
                                pairs.ctypes.data_as(C.POINTER(C.c_int32)), pairs_cap, C.byref(npairs),
                                C.byref(nfree), C.byref(st))
     return dst_bt, pairs[:npairs.value].copy(), npairs.value, nfree.value, st.value
+
+
+
+def kv_merge_inplace(m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride=None):
+    """In-place merge of N instances of TP=a into one of TP=N*a (Sec. 3.1, Improvement 1).
+
+    seq_lens [N][S], bt [N][S][maxb]; pools: list of N*a uint16 arrays, pools[i*a + r] = worker r of instance i
+    (header-centric, NB blocks per layer), rewritten in place into worker r*N+i of the merged instance (NB*N blocks of
+    Hkv/(N*a) headers).  Returns (new_bt [N][S][maxb], live [N][NB], status)."""
+    sl = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    b = np.ascontiguousarray(bt, dtype=np.int32)
+    assert sl.ndim == 2 and b.ndim == 3 and sl.shape[0] == N and b.shape[:2] == sl.shape and len(pools) == N * a
+    S, maxb = b.shape[1], b.shape[2]
+    stride = pool_elems_per_layer(m, T, a, NB) if layer_stride is None else layer_stride
+    new_bt = np.empty_like(b)
+    live = np.empty((N, NB), dtype=np.uint8)
+    st = C.c_int32(status)
+    mm = _model(m)
+    lib().oracle_kv_merge_inplace(C.byref(mm), T, N, a, NB, C.c_int64(stride), S,
+                                  sl.ctypes.data_as(C.POINTER(C.c_int32)), maxb,
+                                  b.ctypes.data_as(C.POINTER(C.c_int32)), _ptr_array(pools),
+                                  new_bt.ctypes.data_as(C.POINTER(C.c_int32)),
+                                  live.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(st))
+    return new_bt, live, st.value

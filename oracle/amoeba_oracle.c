@@ -26,6 +26,16 @@
  *     paper gives no order; the reading used here is sequences in index order, logical blocks in order, each
  *     taking the next id of the ordered free list (list order, or ascending id when a mask is given).
  *
+ *   - In-place migration (Sec. 3.1, "Improvement 1"; the scenario of Sec. 3.1's example, N x TP1 -> TP N, here
+ *     N x TP a -> TP N*a): every worker keeps its memory.  A worker retains, for the requests of its own instance, the
+ *     headers the target TP assigns to it, sends the other headers to their workers, and the room they leave is
+ *     reused "through block reshaping": an old block of Hkv/a headers becomes N new blocks of Hkv/(N*a) headers.
+ *     The paper names no block numbering; the reading used here: the worker r of instance i becomes worker r*N+i of
+ *     the merged instance (so that, with a = 1, W_i keeps header group i as in the paper's example), and block p of
+ *     instance i becomes block p*N+i of the merged instance (on every worker: the block table stays shared).  With
+ *     the header-centric layout that new block is, on the worker that retains it, exactly the retained segment of
+ *     the old block: nothing of it moves.
+ *
  * Elements are opaque 16-bit words (fp16 or bf16 makes no difference to movement).
  */
 #include <stdint.h>
@@ -327,4 +337,86 @@ void oracle_kv_copy_pairs(const oracle_model* m, int T, int a, int NB_src, int s
                                 sp[pool_offset(src_order, NB_src, Ha, T, m->D, p, header - fa, c, tok, d)];
             }
     }
+}
+
+
+/*
+ * In-place merge of N instances of TP = a into one instance of TP = N*a (Sec. 3.1, Improvement 1).
+ *
+ * in : seq_lens[N][S], bt[N][S][maxb] (each instance's own block table over its own pool of NB blocks; -1 padded;
+ *      an instance with fewer than S sequences pads with length 0);
+ *      pools[i*a + r] = pool of worker r (0-indexed) of instance i, header-centric, [L][NB][Hkv/a][K/V][T][D],
+ *      layer_stride elements between layers.
+ * out: the same pools, now read as pools of the merged instance: pools[i*a + r] is worker r*N+i (0-indexed) with
+ *      [L][NB*N][Hkv/(N*a)][K/V][T][D]; new_bt[N][S][maxb] = the merged instance's block table rows of the N
+ *      request sets (entry p -> p*N+i); live[N][NB] = 1 for every old block named by instance i's table.
+ *
+ * Every word is read from a snapshot of the old pools and written to its new place, element by element through
+ * the logical coordinates (instance, block, token, header, K/V, dim); words whose new place equals their old place
+ * are written with the value they already have.  Words of blocks no table names are never touched.
+ *
+ * Errors.  Whole call (nothing moves, new_bt all -1, live all 0): a negative length or a sequence longer than maxb
+ * blocks -> INVALID_ARG.  Per block -> BAD_BLOCK_ID: an id outside [0, NB) or -1 inside a sequence gives new_bt
+ * entry -1 and the block does not move; an id named twice by one instance moves once, both entries get p*N+i.
+ * status is sticky.
+ */
+void oracle_kv_merge_inplace(const oracle_model* m, int T, int N, int a, int NB, int64_t layer_stride, int S,
+                             const int32_t* seq_lens, int maxb, const int32_t* bt, uint16_t* const* pools,
+                             int32_t* new_bt, uint8_t* live, int32_t* status) {
+    const int TPn = N * a;               /* target TP */
+    const int Ha = m->Hkv / a;           /* headers per worker before */
+    const int Hn = m->Hkv / TPn;         /* headers per worker after */
+    const int64_t pool_elems = (int64_t)m->L * layer_stride;
+    for (int64_t k = 0; k < (int64_t)N * S * maxb; ++k) new_bt[k] = -1;
+    for (int64_t k = 0; k < (int64_t)N * NB; ++k) live[k] = 0;
+    for (int64_t k = 0; k < (int64_t)N * S; ++k)
+        if (seq_lens[k] < 0 || blocks_of(seq_lens[k], T) > maxb) {
+            if (*status == 0) *status = ORACLE_INVALID_ARG;
+            return;
+        }
+    /* snapshot of every pool before anything moves */
+    uint16_t** old = (uint16_t**)malloc(sizeof(uint16_t*) * (size_t)(N * a));
+    for (int w = 0; w < N * a; ++w) {
+        old[w] = (uint16_t*)malloc((size_t)pool_elems * sizeof(uint16_t));
+        memcpy(old[w], pools[w], (size_t)pool_elems * sizeof(uint16_t));
+    }
+    for (int i = 0; i < N; ++i) {
+        for (int s = 0; s < S; ++s) {
+            for (int64_t j = 0; j < blocks_of(seq_lens[i * S + s], T); ++j) {
+                const int64_t e = ((int64_t)i * S + s) * maxb + j;
+                const int64_t p = bt[e];
+                if (p < 0 || p >= NB) {
+                    if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+                    continue;
+                }
+                new_bt[e] = (int32_t)(p * N + i);
+                if (live[(int64_t)i * NB + p]) { /* named twice by this instance: already moved */
+                    if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+                    continue;
+                }
+                live[(int64_t)i * NB + p] = 1;
+                for (int l = 0; l < m->L; ++l)
+                    for (int header = 1; header <= m->Hkv; ++header) {
+                        /* before: worker wa of instance i (1-indexed within the instance) */
+                        const int wa = oracle_worker_of_header(m->Hkv, a, header);
+                        int fa, fn, last;
+                        oracle_header_range(m->Hkv, a, wa, &fa, &last);
+                        /* after: worker wn of the merged instance, which is worker (wn-1)/N of instance (wn-1)%N */
+                        const int wn = oracle_worker_of_header(m->Hkv, TPn, header);
+                        oracle_header_range(m->Hkv, TPn, wn, &fn, &last);
+                        const int inst_after = (wn - 1) % N, rank_after = (wn - 1) / N;
+                        const uint16_t* sp = old[i * a + (wa - 1)] + (int64_t)l * layer_stride;
+                        uint16_t* dp = pools[inst_after * a + rank_after] + (int64_t)l * layer_stride;
+                        for (int c = 0; c < 2; ++c)
+                            for (int tok = 0; tok < T; ++tok)
+                                for (int d = 0; d < m->D; ++d)
+                                    dp[pool_offset(ORACLE_HEADER_CENTRIC, (int64_t)NB * N, Hn, T, m->D, p * N + i,
+                                                   header - fn, c, tok, d)] =
+                                        sp[pool_offset(ORACLE_HEADER_CENTRIC, NB, Ha, T, m->D, p, header - fa, c, tok, d)];
+                    }
+            }
+        }
+    }
+    for (int w = 0; w < N * a; ++w) free(old[w]);
+    free(old);
 }
