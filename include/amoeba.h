@@ -231,6 +231,45 @@ AMOEBA_API amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
 
 /*
+ * In-place merge of N instances of TP = a into one instance of TP = N*a  (Sec. 3.1, "Improvement 1": in-place
+ * migration with the header-centric layout; the freed parts of a block are reused through block reshaping)
+ *
+ * The plan's source layout describes every one of the N instances (tp = a, num_blocks = NB); its destination layout
+ * describes the merged instance: tp = N*a, num_blocks = NB*N, same model, block_tokens and layer stride; both
+ * header-centric (with the token-first order the retained headers of a block are not one segment: UNSUPPORTED, as
+ * the paper argues).  Every worker keeps its memory: pools[i*a + r], before the call the pool of worker r of instance
+ * i with NB blocks of Hkv/a headers, is after the call the pool of worker r*N+i of the merged instance with NB*N
+ * blocks of Hkv/(N*a) headers.  Block p of instance i becomes block p*N+i of the merged instance; on the worker that
+ * retains its headers that is the same memory, so those bytes do not move.  The paper gives no numbering; this one
+ * keeps the block table shared by all workers and needs no free list.
+ *
+ * amoeba_merge_block_tables: d_src_bt int32 [N][num_seqs][max_blocks_per_seq] and d_seq_lens int32 [N][num_seqs] are
+ * the N instances' tables (an instance with fewer sequences pads with length 0).  Writes d_dst_bt (same shape:
+ * entry p -> p*N+i, -1 past each sequence's blocks) and d_live: uint8 [N][NB] rounded up to a multiple of 16 bytes
+ * (amoeba_merge_live_bytes), 1 for every block an instance's table names, which amoeba_merge_kv_inplace reads.
+ * Device-detected errors: a negative length or a sequence needing more than max_blocks_per_seq blocks -> whole call
+ * INVALID_ARG (d_dst_bt all -1, d_live all 0, so nothing moves); an id outside [0, NB) or -1 inside a sequence ->
+ * BAD_BLOCK_ID, table entry -1, block not moved; an id named twice by one instance -> BAD_BLOCK_ID, moved once.
+ *
+ * amoeba_merge_kv_inplace: pools is a HOST array of N*a device pointers.  For every layer in [layer_begin, layer_end),
+ * every old block id p and every two instances i != k, the headers of block p that instance i's worker r holds for
+ * merged worker r*N+k move to that worker's memory (pools[k*a + r]), into the place of the headers it gives up for
+ * worker r*N+i; where both blocks are live the two segments are exchanged through shared memory (both are read
+ * completely before either is written), where one is live it is copied, where neither is nothing happens.  Bytes of
+ * blocks no table names, and vacated segments nothing is received into, keep their values.  Moves (N-1)/N of the live
+ * bytes and needs no second pool.  The vector load/store copy path does not apply; the bulk-copy rings are used.
+ */
+AMOEBA_API amoeba_status amoeba_merge_live_bytes(const amoeba_plan* plan, int64_t* bytes);
+AMOEBA_API amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt, const int32_t* d_seq_lens,
+                                        int32_t num_seqs, int32_t max_blocks_per_seq, int32_t* d_dst_bt,
+                                        uint8_t* d_live, int32_t* d_status, void* cuda_stream);
+AMOEBA_API amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                      int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
+/* Bytes read + written by amoeba_merge_kv_inplace when n_live_blocks old blocks (summed over the instances) are
+ * live, over all layers: 2 * (N-1)/N of their size. */
+AMOEBA_API amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_live_blocks, int64_t* kv_bytes_rw);
+
+/*
  * amoeba_reshard_weights  (model weight transformation, Sec. 3.2: the copy that re-partitions the weights; Eq. 1
  * fixes which rows / columns each worker holds)
  *

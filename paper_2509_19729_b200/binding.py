@@ -102,6 +102,10 @@ def _load():
         "amoeba_rewrite_block_tables_builtin_scratch": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP]),
         "amoeba_reshard_kv": (I32, [VP, P(VP), P(VP), VP, VP, I32, I32, I32, VP, VP]),
         "amoeba_reshard_weights": (I32, [VP, P(LayerWeights), P(LayerWeights), I32, I32, VP, VP]),
+        "amoeba_merge_live_bytes": (I32, [VP, P(I64)]),
+        "amoeba_merge_bytes": (I32, [VP, I64, P(I64)]),
+        "amoeba_merge_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, VP, VP]),
+        "amoeba_merge_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
         "amoeba_launch_count": (I64, []),
         "amoeba_status_string": (C.c_char_p, [I32]),
     }
@@ -275,6 +279,38 @@ def amoeba_reshard_weights(plan: Plan, src, dst, layer_begin: int, layer_end: in
         raise AmoebaError(ERR_INVALID_ARG, "amoeba_reshard_weights (need [tp][num_layers] entries)")
     _check(_load().amoeba_reshard_weights(plan.handle, src, dst, layer_begin, layer_end, _ptr(status),
                                           _stream(stream)), "amoeba_reshard_weights")
+
+
+def amoeba_merge_live_bytes(plan: Plan) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_merge_live_bytes(plan.handle, C.byref(out)), "amoeba_merge_live_bytes")
+    return out.value
+
+
+def amoeba_merge_bytes(plan: Plan, n_live_blocks: int) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_merge_bytes(plan.handle, n_live_blocks, C.byref(out)), "amoeba_merge_bytes")
+    return out.value
+
+
+def amoeba_merge_block_tables(plan: Plan, src_bt, seq_lens, num_seqs: int, max_blocks_per_seq: int, dst_bt, live,
+                              status, stream=None) -> None:
+    _check(_load().amoeba_merge_block_tables(plan.handle, _ptr(src_bt), _ptr(seq_lens), num_seqs, max_blocks_per_seq,
+                                             _ptr(dst_bt), _ptr(live), _ptr(status), _stream(stream)),
+           "amoeba_merge_block_tables")
+
+
+def amoeba_merge_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int, layer_end: int, status,
+                            stream=None) -> None:
+    """pools: N*a tensors or addresses, pools[i*a + r] = worker r of instance i."""
+    if len(pools) != plan.dst.tp:
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_merge_kv_inplace (need N*a pools)")
+    pp = (C.c_void_p * len(pools))(*[_ptr(x) for x in pools])
+    _check(_load().amoeba_merge_kv_inplace(plan.handle, pp, _ptr(live), layer_begin, layer_end, _ptr(status),
+                                           _stream(stream)), "amoeba_merge_kv_inplace")
+
+
+__all__ += ["amoeba_merge_live_bytes", "amoeba_merge_bytes", "amoeba_merge_block_tables", "amoeba_merge_kv_inplace"]
 
 
 def amoeba_launch_count() -> int:

@@ -213,6 +213,85 @@ extern "C" amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// Block tables of the in-place merge of N instances (Sec. 3.1, Improvement 1): block p of instance i becomes block
+// p*N+i of the merged instance, and the blocks each instance's table names are marked live for the KV kernel.
+// One launch; no CTA waits on another: every CTA decides the whole-call error by scanning all sequence lengths itself
+// (a few KB), the live bytes are zeroed by a memset that precedes the launch on the stream.
+namespace amoeba {
+
+__global__ void __launch_bounds__(256) merge_tables(const int32_t* __restrict__ src_bt,
+                                                    const int32_t* __restrict__ seq_lens, int32_t n_inst,
+                                                    int32_t num_seqs, int32_t block_tokens,
+                                                    int32_t max_blocks_per_seq, int32_t nb, int32_t* __restrict__ dst_bt,
+                                                    uint32_t* live_words, int32_t* status) {
+    const int64_t rows = (int64_t)n_inst * num_seqs;
+    int bad_len = 0;
+    for (int64_t k = threadIdx.x; k < rows; k += blockDim.x) {
+        const int32_t len = seq_lens[k];
+        bad_len |= len < 0 || ((int64_t)len + block_tokens - 1) / block_tokens > max_blocks_per_seq;
+    }
+    const bool call_failed = __syncthreads_or(bad_len) != 0;
+    if (call_failed && blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_INVALID_ARG);
+
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int32_t segs_per_row = (max_blocks_per_seq + kSegment - 1) / kSegment;
+    bool bad = false;
+    for (int64_t unit = warp; unit < rows * segs_per_row; unit += n_warps) {
+        const int64_t row = unit / segs_per_row;  // instance * num_seqs + sequence
+        const int32_t inst = (int32_t)(row / num_seqs);
+        const int32_t col0 = (int32_t)(unit - row * segs_per_row) * kSegment;
+        const int32_t nblk = call_failed ? 0 : (int32_t)(((int64_t)seq_lens[row] + block_tokens - 1) / block_tokens);
+        for (int32_t i = col0 + lane; i < min(col0 + kSegment, max_blocks_per_seq); i += 32) {
+            int32_t out = -1;
+            if (i < nblk) {
+                const int32_t p = src_bt[row * max_blocks_per_seq + i];
+                if (p >= 0 && p < nb) {
+                    out = p * n_inst + inst;
+                    const int64_t idx = (int64_t)inst * nb + p;  // byte of the live array
+                    const uint32_t bit = 1u << (8 * (idx & 3));
+                    if (atomicOr(live_words + (idx >> 2), bit) & bit) bad = true;  // named twice by this instance
+                } else {
+                    bad = true;
+                }
+            }
+            dst_bt[row * max_blocks_per_seq + i] = out;
+        }
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+}
+
+}  // namespace amoeba
+
+extern "C" amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
+                                                   const int32_t* d_seq_lens, int32_t num_seqs,
+                                                   int32_t max_blocks_per_seq, int32_t* d_dst_bt, uint8_t* d_live,
+                                                   int32_t* d_status, void* cuda_stream) {
+    if (!plan || num_seqs < 0 || max_blocks_per_seq <= 0 || !d_live || !d_status) return AMOEBA_ERR_INVALID_ARG;
+    if (num_seqs > 0 && (!d_src_bt || !d_seq_lens || !d_dst_bt)) return AMOEBA_ERR_INVALID_ARG;
+    const int n = merge_instances(plan);
+    if (!n) return AMOEBA_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(d_live) % 16) return AMOEBA_ERR_ALIGNMENT;
+    int64_t live_bytes = 0;
+    amoeba_merge_live_bytes(plan, &live_bytes);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(d_live, 0, (size_t)live_bytes, stream) != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    if (num_seqs == 0) return AMOEBA_OK;
+    DeviceInfo dev;
+    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    const int64_t units = (int64_t)n * num_seqs * ((max_blocks_per_seq + kSegment - 1) / kSegment);
+    const int grid = (int)std::min<int64_t>((units + 7) / 8, (int64_t)dev.sms * 4);
+    merge_tables<<<grid, 256, 0, stream>>>(d_src_bt, d_seq_lens, n, num_seqs, plan->src.block_tokens,
+                                           max_blocks_per_seq, plan->src.num_blocks, d_dst_bt,
+                                           reinterpret_cast<uint32_t*>(d_live), d_status);
+    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    return AMOEBA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // Variant for callers that cannot allocate device memory: the scratch is an array in the library's device image.
 namespace amoeba {
 

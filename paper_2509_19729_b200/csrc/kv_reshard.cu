@@ -231,6 +231,93 @@ __global__ void __launch_bounds__(1024) kv_reshard_pair_box(const __grid_constan
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------- in-place merge of N instances (Sec. 3.1, Impr. 1)
+// Pools: [instance i][worker r] -> pools[i*a + r]; old block p of such a pool is N segments of Hkv/(N*a) headers;
+// segment k is what merged worker r*N+k keeps.  For i < k the pair of segments (pool (i,r), block p, segment k) and
+// (pool (k,r), block p, segment i) trade places; segment i of pool (i,r) stays.  A work item is one chunk of such a
+// pair: both live -> a two-row item whose rows are read from A and B and written to B and A (the rings read a whole
+// item into a stage before they write any of it); one live -> a plain copy; none -> skipped.
+struct MergeParams {
+    char* pools[AMOEBA_MAX_TP];
+    const uint8_t* live;  // [N][nb]
+    int64_t layer_stride, block_bytes, seg_bytes, chunk_bytes;
+    int32_t n_inst, a, nb, layer_begin, n_layers, chunks_per_seg, n_pairs;
+};
+
+struct MergeItems {
+    const MergeParams& p;
+    __device__ __forceinline__ int64_t count() const {
+        return (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
+    }
+    __device__ __forceinline__ Item operator()(int64_t w) const {
+        const int32_t chunk = (int32_t)(w % p.chunks_per_seg);
+        int64_t t = w / p.chunks_per_seg;
+        int32_t pr = (int32_t)(t % p.n_pairs);
+        t /= p.n_pairs;
+        const int32_t r = (int32_t)(t % p.a);
+        t /= p.a;
+        const int32_t blk = (int32_t)(t % p.nb);
+        const int32_t layer = p.layer_begin + (int32_t)(t / p.nb);
+        int32_t i = 0;  // pr-th pair (i, k) with i < k, in lexicographic order
+        while (pr >= p.n_inst - 1 - i) {
+            pr -= p.n_inst - 1 - i;
+            ++i;
+        }
+        const int32_t k = i + 1 + pr;
+        const bool live_i = p.live[(int64_t)i * p.nb + blk] != 0, live_k = p.live[(int64_t)k * p.nb + blk] != 0;
+        Item it;
+        it.src_map = it.dst_map = nullptr;
+        it.n_rows = 0;
+        it.row_bytes = (int32_t)p.chunk_bytes;
+        it.src = nullptr;
+        it.dst = nullptr;
+        it.src_pitch = it.dst_pitch = 0;
+        if (!live_i && !live_k) return it;
+        const int64_t base = layer * p.layer_stride + (int64_t)blk * p.block_bytes + (int64_t)chunk * p.chunk_bytes;
+        char* A = p.pools[i * p.a + r] + base + k * p.seg_bytes;  // leaves instance i's worker for merged worker r*N+k
+        char* B = p.pools[k * p.a + r] + base + i * p.seg_bytes;  // leaves instance k's worker for merged worker r*N+i
+        if (live_i && live_k) {
+            it.n_rows = 2;
+            it.src = A;
+            it.src_pitch = B - A;
+            it.dst = B;
+            it.dst_pitch = A - B;
+        } else {
+            it.n_rows = 1;
+            it.src = live_i ? A : B;
+            it.dst = live_i ? B : A;
+        }
+        return it;
+    }
+};
+
+__global__ void __launch_bounds__(1024) kv_merge_bulk(const __grid_constant__ MergeParams p, const RingShape rs,
+                                                      int32_t* status) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem) + warp * rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)warp * rs.stages * rs.stage_bytes;
+    const MergeItems items{p};
+    const bool ok = warp_bulk_ring(items, items.count(), (int64_t)blockIdx.x * nwarps + warp,
+                                   (int64_t)gridDim.x * nwarps, stages, bars, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
+}
+
+__global__ void __launch_bounds__(1024) kv_merge_pair(const __grid_constant__ MergeParams p, const RingShape rs,
+                                                      int32_t* status) {
+    extern __shared__ __align__(128) char smem[];
+    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
+    uint64_t* empty = full + rs.stages;
+    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
+    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
+    __syncthreads();
+    const MergeItems items{p};
+    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
+                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime so that the library does not link against the driver.
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -377,6 +464,63 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
             kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring);
             e = cudaGetLastError();
         }
+    }
+    if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    return AMOEBA_OK;
+}
+
+extern "C" amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status,
+                                                 void* cuda_stream) {
+    if (!plan || !pools || !d_live || !d_status) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_model& m = plan->src.model;
+    if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    const int n = merge_instances(plan);
+    if (!n) return AMOEBA_ERR_UNSUPPORTED;
+    const int a = plan->src.tp;
+    MergeParams p{};
+    for (int w = 0; w < n * a; ++w) {
+        if (!pools[w]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(pools[w]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        for (int v = 0; v < w; ++v)
+            if (pools[v] == pools[w]) return AMOEBA_ERR_INVALID_ARG;  // every worker has its own memory
+        p.pools[w] = static_cast<char*>(pools[w]);
+    }
+    if (layer_begin == layer_end) return AMOEBA_OK;
+    const KernelOpts& opt = plan->opt.kv;
+    const int64_t cap = std::max<int64_t>(16, (opt.chunk_bytes > 0 ? opt.chunk_bytes : kDefaultKvChunk) / 2);
+    p.live = d_live;
+    p.layer_stride = plan->src_layer_stride;
+    p.block_bytes = plan->src_block_bytes;
+    p.seg_bytes = plan->dst_block_bytes;  // one new block = one segment of an old block
+    p.chunk_bytes = p.seg_bytes;          // largest divisor of the segment that is a multiple of 16 and <= cap
+    for (int64_t parts = std::max<int64_t>(1, (p.seg_bytes + cap - 1) / cap); parts <= p.seg_bytes / 16; ++parts)
+        if (p.seg_bytes % parts == 0 && (p.seg_bytes / parts) % 16 == 0) {
+            p.chunk_bytes = p.seg_bytes / parts;
+            break;
+        }
+    if (p.chunk_bytes > 65536) return AMOEBA_ERR_UNSUPPORTED;
+    p.chunks_per_seg = (int32_t)(p.seg_bytes / p.chunk_bytes);
+    p.n_inst = n;
+    p.a = a;
+    p.nb = plan->src.num_blocks;
+    p.layer_begin = layer_begin;
+    p.n_layers = layer_end - layer_begin;
+    p.n_pairs = n * (n - 1) / 2;
+
+    DeviceInfo dev;
+    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int path = opt.copy_path == 2 ? 2 : 3;  // a swap needs a staged copy: the rings only
+    const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)(2 * p.chunk_bytes));
+    const int64_t n_items = (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
+    const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+    auto kernel = path == 3 ? kv_merge_pair : kv_merge_bulk;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+    if (e == cudaSuccess) {
+        kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring, d_status);
+        e = cudaGetLastError();
     }
     if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();

@@ -132,6 +132,16 @@ amoeba_status finalize_chunks(amoeba_plan* p) {
     return AMOEBA_OK;
 }
 
+int merge_instances(const amoeba_plan* p) {
+    const amoeba_layout &s = p->src, &d = p->dst;
+    if (s.kv_order != AMOEBA_KV_HEAD_MAJOR || d.kv_order != AMOEBA_KV_HEAD_MAJOR) return 0;
+    if (d.tp % s.tp) return 0;
+    const int64_t n = d.tp / s.tp;
+    if (n < 2 || (int64_t)d.num_blocks != (int64_t)s.num_blocks * n) return 0;
+    if (p->src_layer_stride != p->dst_layer_stride) return 0;
+    return (int)n;
+}
+
 struct Range {
     int64_t lo, hi;
 };
@@ -393,6 +403,24 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
         finalize_chunks(plan);
     }
     return st;
+}
+
+amoeba_status amoeba_merge_live_bytes(const amoeba_plan* plan, int64_t* bytes) {
+    if (!plan || !bytes) return AMOEBA_ERR_INVALID_ARG;
+    const int n = merge_instances(plan);
+    if (!n) return AMOEBA_ERR_UNSUPPORTED;
+    *bytes = ((int64_t)n * plan->src.num_blocks + 15) / 16 * 16;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_live_blocks, int64_t* kv_bytes_rw) {
+    if (!plan || !kv_bytes_rw || n_live_blocks < 0) return AMOEBA_ERR_INVALID_ARG;
+    const int n = merge_instances(plan);
+    if (!n) return AMOEBA_ERR_UNSUPPORTED;
+    const amoeba_model& m = plan->src.model;
+    // one old block on all a workers of its instance: Hkv headers; (n-1)/n of them move, read once and written once
+    *kv_bytes_rw = 2 * n_live_blocks * m.num_layers * (m.num_kv_heads / n) * (n - 1) * plan->unit_bytes;
+    return AMOEBA_OK;
 }
 
 int64_t amoeba_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
