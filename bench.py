@@ -161,11 +161,40 @@ def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=None, w_layers=4, threads=1
     return run, kv_bytes + w_bytes, desc
 
 
+def oracle_merge_sample(cfg_name: str, kv_layers=1, n_seqs=16):
+    """A bounded sample of a merge workload for the CPU oracle: the first n_seqs sequences of every instance over
+    kv_layers layers.  Returns a closure that runs one oracle in-place merge and the bytes the merge moves."""
+    import oracle
+
+    oracle.build()
+    cfg = wl.MERGE_CONFIGS[cfg_name]
+    m, N, a, T = dict(cfg["model"], L=kv_layers), cfg["N"], cfg["a"], wl.BLOCK_TOKENS
+    st = wl.draw_merge_state(dict(cfg, S=min(n_seqs, cfg["S"])), name=cfg_name)
+    per = oracle.pool_elems_per_layer(m, T, a, st["NB"])
+    g = wl.rng(wl.DEFAULT_SEED, "merge_sample")
+    pools = [g.integers(0, 65536, size=kv_layers * per, dtype=np.uint16) for _ in range(N * a)]
+    nbytes = 2 * st["n_live"] * kv_layers * (m["Hkv"] // N) * (N - 1) * 2 * T * m["D"] * 2
+
+    def run():
+        _, _, status = oracle.kv_merge_inplace(m, T, N, a, st["NB"], st["seq_lens"], st["src_bt"], pools)
+        assert status == 0
+
+    desc = (f"{cfg_name}: first {min(n_seqs, cfg['S'])} of {cfg['S']} sequences per instance ({st['n_live']} blocks) x "
+            f"{kv_layers} of {cfg['model']['L']} layers")
+    return run, nbytes, desc
+
+
 def run_reference(args, rank, world):
     """The reference arm: the CPU oracle as it stands, timed on the host cores on a bounded sample per step."""
     if rank != 0:
         return
-    run, nbytes, desc = oracle_sample(args.config, kv_layers=1, w_layers=2)
+    if args.config in wl.MERGE_CONFIGS:
+        run, nbytes, desc = oracle_merge_sample(args.config)
+        cfg = dict(wl.MERGE_CONFIGS[args.config])
+        cfg["a"], cfg["b"] = f"{cfg['N']}x{cfg['a']}", cfg["N"] * cfg["a"]
+    else:
+        run, nbytes, desc = oracle_sample(args.config, kv_layers=1, w_layers=2)
+        cfg = wl.CONFIGS[args.config]
     for _ in range(args.warmup):
         run()
     t0 = time.perf_counter()
@@ -173,7 +202,6 @@ def run_reference(args, rank, world):
         run()
     dt = (time.perf_counter() - t0) / args.steps
     val = nbytes / dt / 1e9
-    cfg = wl.CONFIGS[args.config]
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
@@ -215,6 +243,109 @@ def build_session(cfg_name: str, device, layers=None, kv=True, weights=True, see
             p.fill_(0xA5)
     torch.cuda.synchronize()
     return s, st
+
+
+def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, fill=True):
+    import torch
+
+    from paper_2509_19729_b200.session import MergeSession
+
+    cfg = wl.MERGE_CONFIGS[cfg_name]
+    m = dict(cfg["model"])
+    if layers is not None:
+        m["L"] = layers
+    st = wl.draw_merge_state(cfg, seed=seed, name=cfg_name)
+    s = MergeSession(m, cfg["N"], cfg["a"], st["NB"], cfg["S"], st["maxb"], device=device)
+    s.set_tables(st["seq_lens"], st["src_bt"])
+    if fill:
+        for i, p in enumerate(s.pools):
+            wl.hash_fill_(p, seed, 300 + i)
+    torch.cuda.synchronize()
+    return s, st
+
+
+def run_merge(args, rank, world, local):
+    """In-place merge workload: one step = merged block tables + the in-place KV exchange of all layers.  (A second
+    step over the same tables exchanges the same segments back: every step moves the same bytes.)"""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    cfg = wl.MERGE_CONFIGS[args.config]
+    s, st = build_merge_session(args.config, device, layers=args.layers)
+    for opt, val in ((A.OPT_COPY_PATH, args.copy_path), (A.OPT_CHUNK_BYTES, args.chunk), (A.OPT_STAGES, args.stages),
+                     (A.OPT_CTAS_PER_SM, args.ctas_per_sm)):
+        if val:
+            s.set_option(opt, val)
+    nbytes = s.bytes_rw(st["n_live"])
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(args.warmup):
+        s.status.zero_()
+        s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0, f"device status {int(s.status.item())}"
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = A.amoeba_launch_count()
+    marks = []
+    t_begin, t_end = ev(), ev()
+    torch.cuda.synchronize()
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        m3 = [ev() for _ in range(3)]
+        m3[0].record(stream)
+        s.merge_block_tables()
+        m3[1].record(stream)
+        s.merge_kv()
+        m3[2].record(stream)
+        marks.append(m3)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    barrier(world)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0
+    sec = t_begin.elapsed_time(t_end) / 1e3 / args.steps
+    bt_ms = statistics.mean(m3[0].elapsed_time(m3[1]) for m3 in marks)
+    kv_ms = statistics.mean(m3[1].elapsed_time(m3[2]) for m3 in marks)
+    sec_all, bytes_all = aggregate(world, sec, nbytes, device)
+    pool_bytes = sum(p.numel() for p in s.pools)
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    kv_gbs = nbytes / (kv_ms / 1e3) / 1e9
+    N, a = cfg["N"], cfg["a"]
+    out = {
+        "metric": METRIC, "value": bytes_all / sec_all / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{N}x{a}->{N * a} in place", "layers": s.kv_layers,
+                   "sequences_per_instance": cfg["S"], "live_blocks": st["n_live"], "pool_blocks": st["NB"],
+                   "block_tokens": wl.BLOCK_TOKENS, "kv_bytes_rw": nbytes, "weight_bytes_rw": 0,
+                   "pool_bytes": pool_bytes, "extra_kv_memory_bytes": 0,
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
+        "phases_ms": {"merge_block_tables": bt_ms, "merge_kv_inplace": kv_ms},
+        "phases_gbs": {"merge_kv_inplace": kv_gbs},
+        "roofline": {"kernel": "kv_merge_pair", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": None,
+    }
+    del s
+    torch.cuda.empty_cache()
+    if not args.no_cpu_baseline and world == 1:
+        run, ob, desc = oracle_merge_sample(args.config, kv_layers=2, n_seqs=10**9)
+        t0 = time.perf_counter()
+        run()
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": ob / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc,
+                               "seconds": dt}
+    print(json.dumps(out))
 
 
 def host_free_bytes() -> int:
@@ -341,7 +472,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=list(wl.CONFIGS))
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=list(wl.CONFIGS) + list(wl.MERGE_CONFIGS))
     ap.add_argument("--copy-path", type=int, default=0, help="0 default, 1 vector ld/st, 2 bulk-copy ring per warp, 3 producer/consumer bulk-copy ring")
     ap.add_argument("--chunk", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
@@ -359,6 +490,10 @@ def main():
     rank, world, local = dist_setup(args.gpus if args.impl == "ours" else 0)
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+
+    if args.config in wl.MERGE_CONFIGS:
+        run_merge(args, rank, world, local)
         return
 
     import torch

@@ -136,3 +136,54 @@ class Session:
         """(KV bytes, weight bytes) read+written by one step with n_blocks live blocks over the held KV layers."""
         kv, w = A.amoeba_plan_bytes(self.plan, n_blocks)
         return kv * self.kv_layers // self.L if self.src_pools else 0, w if self.src_w else 0
+
+
+
+class MergeSession:
+    """Buffers of one in-place merge of N instances of TP=a into one instance of TP=N*a on one GPU.
+
+    pools[i*a + r] is the pool of worker r of instance i before the merge and of worker r*N+i of the merged instance
+    after it.  kv_layers: layers the pools hold (None = all)."""
+
+    def __init__(self, model: dict, N: int, a: int, NB: int, num_seqs: int, max_blocks_per_seq: int,
+                 kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0"):
+        self.model, self.N, self.a, self.NB = model, N, a, NB
+        self.device = torch.device(device)
+        self.src_layout = A.make_layout(model, a, NB, block_tokens)
+        self.dst_layout = A.make_layout(model, N * a, NB * N, block_tokens)
+        self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
+        self.L = model["L"]
+        self.kv_layers = self.L if kv_layers is None else kv_layers
+        self.num_seqs, self.maxb = num_seqs, max_blocks_per_seq
+        i32 = dict(dtype=torch.int32, device=self.device)
+        self.src_bt = torch.full((N, num_seqs, max_blocks_per_seq), -1, **i32)
+        self.dst_bt = torch.full((N, num_seqs, max_blocks_per_seq), -2, **i32)
+        self.seq_lens = torch.zeros((N, num_seqs), **i32)
+        self.status = torch.zeros(1, **i32)
+        self.live = torch.zeros(A.amoeba_merge_live_bytes(self.plan), dtype=torch.uint8, device=self.device)
+        per_layer = A.amoeba_layout_kv_pool_bytes(self.src_layout) // self.L
+        self.pools = [torch.empty(per_layer * self.kv_layers, dtype=torch.uint8, device=self.device)
+                      for _ in range(N * a)]
+
+    def set_tables(self, seq_lens, src_bt) -> None:
+        self.seq_lens.copy_(torch.as_tensor(seq_lens, dtype=torch.int32))
+        self.src_bt.copy_(torch.as_tensor(src_bt, dtype=torch.int32))
+
+    def merge_block_tables(self, stream=None) -> None:
+        A.amoeba_merge_block_tables(self.plan, self.src_bt, self.seq_lens, self.num_seqs, self.maxb, self.dst_bt,
+                                    self.live, self.status, stream)
+
+    def merge_kv(self, stream=None, layer_begin: int = 0, layer_end: Optional[int] = None) -> None:
+        A.amoeba_merge_kv_inplace(self.plan, self.pools, self.live, layer_begin,
+                                  self.kv_layers if layer_end is None else layer_end, self.status, stream)
+
+    def step(self, stream=None) -> None:
+        self.merge_block_tables(stream)
+        self.merge_kv(stream)
+
+    def set_option(self, option: int, value: int) -> None:
+        A.amoeba_plan_set_option(self.plan, option, value)
+
+    def bytes_rw(self, n_live: int) -> int:
+        """Bytes read + written by one merge with n_live live old blocks (summed over instances), held layers."""
+        return A.amoeba_merge_bytes(self.plan, n_live) * self.kv_layers // self.L

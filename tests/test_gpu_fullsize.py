@@ -115,3 +115,59 @@ def test_full_size_config(name, kv_order, oracle):
     finally:
         del s
         torch.cuda.empty_cache()
+
+
+def test_full_size_inplace_merge(oracle):
+    """The benchmark's in-place merge workload (4 x TP1 -> TP4) at full size: merged tables and live marks compared
+    whole; sampled old blocks (with whatever mix of live / free they have across the instances) compared with the
+    oracle's merge of just those blocks; word sums of the live blocks conserved per layer."""
+    import torch
+
+    import bench
+
+    name = "llama3_8b_merge_4x1to4"
+    cfg = wl.MERGE_CONFIGS[name]
+    m, N, a, T = cfg["model"], cfg["N"], cfg["a"], wl.BLOCK_TOKENS
+    device = torch.device("cuda:0")
+    s, st = bench.build_merge_session(name, device)
+    try:
+        NB, L = st["NB"], s.kv_layers
+        exp_bt, exp_live, exp_status = oracle.kv_merge_inplace(dict(m, L=0), T, N, a, NB, st["seq_lens"], st["src_bt"],
+                                                               [np.zeros(0, np.uint16) for _ in range(N * a)])
+        assert exp_status == 0
+        g = np.random.default_rng(11)
+        old_v = [p.view(L, NB, -1) for p in s.pools]            # [layer][old block][bytes]
+        samples = [(int(g.integers(L)), int(g.integers(NB))) for _ in range(64)]
+        before = {(l, p): [v[l, p].cpu().numpy().view(np.uint16).copy() for v in old_v] for l, p in samples}
+        live_old = [torch.as_tensor(np.flatnonzero(exp_live[i]).astype(np.int64), device=device) for i in range(N)]
+        sum_layers = sorted(set(int(x) for x in g.integers(L, size=2)))
+        sums_before = {l: sum(int(old_v[i * a + r][l].view(torch.int64).view(NB, -1).index_select(0, live_old[i]).sum())
+                              for i in range(N) for r in range(a)) for l in sum_layers}
+
+        s.status.zero_()
+        s.step()
+        torch.cuda.synchronize()
+        assert int(s.status.item()) == 0
+        assert np.array_equal(s.dst_bt.cpu().numpy(), exp_bt)
+        assert np.array_equal(s.live.cpu().numpy()[:N * NB].reshape(N, NB), exp_live)
+
+        one = dict(m, L=1)
+        for (l, p), olds in before.items():
+            lens1 = np.array([[T if exp_live[i, p] else 0] for i in range(N)], np.int32)
+            mini = [o.copy() for o in olds]                      # N*a pools of one old block each
+            _, _, st1 = oracle.kv_merge_inplace(one, T, N, a, 1, lens1, np.zeros((N, 1, 1), np.int32), mini)
+            assert st1 == 0
+            for w in range(N * a):
+                got = old_v[w][l, p].cpu().numpy().view(np.uint16)
+                assert np.array_equal(got, mini[w]), (l, p, w)
+
+        new_v = [p.view(L, NB * N, -1) for p in s.pools]        # [layer][new block][bytes]
+        for l in sum_layers:
+            after = 0
+            for i in range(N):
+                ids = live_old[i] * N + i
+                after += sum(int(v[l].view(torch.int64).view(NB * N, -1).index_select(0, ids).sum()) for v in new_v)
+            assert (after - sums_before[l]) % (1 << 64) == 0
+    finally:
+        del s
+        torch.cuda.empty_cache()

@@ -52,6 +52,16 @@ CONFIGS = {
 }
 
 
+# In-place merges of N instances of TP=a into one of TP=N*a (the paper's KV micro-benchmark setting: 4 x TP1 -> TP4
+# at 90 % KV-cache utilisation).  S sequences per instance; every instance has its own pool and block placement.
+MERGE_CONFIGS = {
+    "llama3_8b_merge_4x1to4": dict(model=_model(32, 4096, 32, 8, 128, 14336), dtype="bf16", N=4, a=1, S=48,
+                                   lens=("uniform", 512, 8192), utilisation=0.9),
+    "tiny_merge_2x1to2": dict(model=_model(2, 256, 4, 4, 64, 1024), dtype="fp16", N=2, a=1, S=4,
+                              lens=("uniform", 16, 256), utilisation=0.75),
+}
+
+
 def key(seed: int, purpose: str, *index: int) -> int:
     """128-bit generator key from (seed, purpose, index...)."""
     h = hashlib.blake2b(repr((int(seed), purpose, tuple(int(i) for i in index))).encode(), digest_size=16)
@@ -129,6 +139,25 @@ def draw_kv_state(cfg: dict, seed: int = DEFAULT_SEED, name: str = "", seq_lens=
         st["NB_dst"] = NB_dst
         st["dst_free_mask"] = mask
     return st
+
+
+def draw_merge_state(cfg: dict, seed: int = DEFAULT_SEED, name: str = "", T: int = BLOCK_TOKENS) -> dict:
+    """Tables of the N instances of a merge workload: seq_lens [N][S], src_bt [N][S][maxb] (-1 padded; each instance's
+    live blocks scattered over its own pool of NB blocks), NB, maxb, n_live (live blocks summed over instances)."""
+    N, S = cfg["N"], cfg["S"]
+    lens = np.stack([draw_seq_lens(cfg, seed, f"{name}/{i}") for i in range(N)])
+    nblk = (lens.astype(np.int64) + T - 1) // T
+    maxb = max(int(nblk.max()), 1)
+    NB = max(int(math.ceil(int(nblk.sum(axis=1).max()) / cfg.get("utilisation", 0.9))), 1)
+    bt = np.full((N, S, maxb), -1, dtype=np.int32)
+    for i in range(N):
+        ids = rng(seed, "merge_blocks", i, *name.encode()).permutation(NB).astype(np.int32)
+        k = 0
+        for s in range(S):
+            bt[i, s, :nblk[i, s]] = ids[k:k + nblk[i, s]]
+            k += int(nblk[i, s])
+    return dict(seq_lens=lens.astype(np.int32), src_bt=bt, NB=NB, maxb=maxb, n_live=int(nblk.sum()),
+                blocks_per_seq=nblk, T=T)
 
 
 def draw_kv_logical(cfg: dict, n_tokens: int, layers, seed: int = DEFAULT_SEED, dist: str = "normal") -> np.ndarray:
