@@ -267,3 +267,79 @@ def kv_merge_inplace(m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride
                                   new_bt.ctypes.data_as(C.POINTER(C.c_int32)),
                                   live.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(st))
     return new_bt, live, st.value
+
+
+
+# ---- Sec. 3.2, Improvement 1: padded partitions -----------------------------------------------------------------
+def pages_per_tensor(rows: int, cols: int, elem_bytes: int, TP: int, page_bytes: int = 2 << 20) -> float:
+    f = lib().oracle_pages_per_tensor
+    f.restype = C.c_double
+    return f(C.c_int64(rows), C.c_int64(cols), elem_bytes, TP, C.c_int64(page_bytes))
+
+
+def padded_pitch(partition_elems: int, page_elems: int) -> int:
+    f = lib().oracle_padded_pitch
+    f.restype = C.c_int64
+    return f(C.c_int64(partition_elems), C.c_int64(page_elems))
+
+
+def padded_partition_elems(m: dict, P: int, fused_qkv=True, fused_gate_up=True) -> dict:
+    """Elements of one partition of each buffer (before rounding up to pages)."""
+    hid, q, kv, f = m["hidden"], m["Hq"] * m["D"] // P * m["hidden"], m["Hkv"] * m["D"] // P * m["hidden"], \
+        m["I"] // P * m["hidden"]
+    out = {"o": q, "down": f}
+    if fused_qkv:
+        out["q"] = q + 2 * kv
+    else:
+        out.update(q=q, k=kv, v=kv)
+    if fused_gate_up:
+        out["gate"] = 2 * f
+    else:
+        out.update(gate=f, up=f)
+    return out
+
+
+def empty_padded_shards(m, TP, P, page_elems, fused_qkv=True, fused_gate_up=True, fill=0xA5A5):
+    """Flat uint16 buffers of P/TP padded partitions each, one dict per worker."""
+    n = P // TP
+    return [{name: np.full(n * padded_pitch(e, page_elems), fill, dtype=np.uint16)
+             for name, e in padded_partition_elems(m, P, fused_qkv, fused_gate_up).items()} for _ in range(TP)]
+
+
+def _padded_walk(logical, shards, m, TP, P, page_elems, fused_qkv, fused_gate_up, direction):
+    lg = _wstruct(logical)
+    mm = _model(m)
+    for r in range(TP):
+        sh = _wstruct(shards[r])
+        lib().oracle_weights_padded_walk(C.byref(mm), TP, r, P, C.c_int64(page_elems), int(fused_qkv),
+                                         int(fused_gate_up), C.byref(lg), C.byref(sh), direction)
+
+
+def weights_shard_padded(logical, m, TP, P, page_elems, fused_qkv=True, fused_gate_up=True, fill=0xA5A5):
+    shards = empty_padded_shards(m, TP, P, page_elems, fused_qkv, fused_gate_up, fill)
+    _padded_walk(logical, shards, m, TP, P, page_elems, fused_qkv, fused_gate_up, 0)
+    return shards
+
+
+def weights_reconstruct_padded(shards, m, TP, P, page_elems, fused_qkv=True, fused_gate_up=True):
+    logical = {n: np.zeros(s, dtype=np.uint16) for n, s in logical_shapes(m).items()}
+    _padded_walk(logical, shards, m, TP, P, page_elems, fused_qkv, fused_gate_up, 1)
+    return logical
+
+
+def weights_transform_any(src_shards, m, a, b, fused_qkv=True, fused_gate_up=True, src_pad=None, dst_pad=None,
+                          fill=0xA5A5):
+    """TP a->b on one layer's weights where either side may be padded: ``*_pad`` = (P, page_elems) or None for the
+    dense shards.  Reconstruct the logical tensors from the source form, shard them in the destination form."""
+    if src_pad:
+        logical = weights_reconstruct_padded(src_shards, m, a, src_pad[0], src_pad[1], fused_qkv, fused_gate_up)
+    else:
+        logical = weights_reconstruct(src_shards, m, a, fused_qkv, fused_gate_up)
+    if dst_pad:
+        return weights_shard_padded(logical, m, b, dst_pad[0], dst_pad[1], fused_qkv, fused_gate_up, fill)
+    out = empty_shards(m, b, fused_qkv, fused_gate_up, fill)
+    lg, mm = _wstruct(logical), _model(m)
+    for r in range(b):
+        sh = _wstruct(out[r])
+        lib().oracle_weights_shard(C.byref(mm), b, r, int(fused_qkv), int(fused_gate_up), C.byref(lg), C.byref(sh))
+    return out

@@ -36,6 +36,15 @@
  *     the header-centric layout that new block is, on the worker that retains it, exactly the retained segment of
  *     the old block: nothing of it moves.
  *
+ *   - Weight padding (Sec. 3.2, "Improvement 1", Eq. 2): padding is added at every potential partition boundary
+ *     so that each partition starts on an allocation-page boundary (2 MB in the paper, Table 2 counts such pages per
+ *     tensor).  With P = the largest TP degree the instance may take, a tensor is P partitions; a worker of TP = t
+ *     holds P/t consecutive partitions, each stored dense at a pitch rounded up to whole pages:
+ *     U' = [U_1, 0, U_2, 0, ...], D' = [D_1^T, 0, D_2^T, 0, ...]^T.  A partition of a tensor split by rows is its
+ *     rows; a partition of a tensor split by columns (o_proj, down_proj) is stored as its own dense
+ *     [hidden, columns/P] matrix (the paper's D_i).  A fused buffer pads after each partition's [q;k;v] or [gate;up].
+ *     The pad words themselves are never written here.
+ *
  * Elements are opaque 16-bit words (fp16 or bf16 makes no difference to movement).
  */
 #include <stdint.h>
@@ -419,4 +428,72 @@ void oracle_kv_merge_inplace(const oracle_model* m, int T, int N, int a, int NB,
     }
     for (int w = 0; w < N * a; ++w) free(old[w]);
     free(old);
+}
+
+
+/* ---- Sec. 3.2, Improvement 1: padded partitions ---- */
+
+/* Table 2: allocation pages one tensor of rows x cols elements of elem_bytes occupies when split TP ways. */
+double oracle_pages_per_tensor(int64_t rows, int64_t cols, int elem_bytes, int TP, int64_t page_bytes) {
+    return (double)rows * (double)cols * (double)elem_bytes / (double)TP / (double)page_bytes;
+}
+
+/* Elements from the start of one partition to the start of the next: the partition rounded up to whole pages. */
+int64_t oracle_padded_pitch(int64_t partition_elems, int64_t page_elems) {
+    return (partition_elems + page_elems - 1) / page_elems * page_elems;
+}
+
+/*
+ * Worker r (0-indexed) of TP holds partitions r*P/TP ... (r+1)*P/TP - 1 of every tensor, partition j of its own at
+ * element offset j*pitch of the buffer (pitch = the buffer's partition size rounded up to pages).
+ * Buffers: q,k,v,gate,up: partition = its rows, [rows/P, hidden]; o, down: partition = [hidden, cols/P] dense;
+ * fused_qkv: partition = [q_p; k_p; v_p] under the q pointer; fused_gate_up: [gate_p; up_p] under the gate pointer.
+ * dir = 0: logical -> shard, dir = 1: shard -> logical.
+ */
+static void padded_rows(uint16_t* logical, int64_t rows_total, int64_t cols, int P, int p, uint16_t* part, int dir) {
+    const int64_t rows_p = rows_total / P;
+    for (int64_t i = 0; i < rows_p; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            const int64_t lo = (p * rows_p + i) * cols + j;
+            if (dir == 0) part[i * cols + j] = logical[lo];
+            else logical[lo] = part[i * cols + j];
+        }
+}
+
+static void padded_cols(uint16_t* logical, int64_t rows, int64_t cols_total, int P, int p, uint16_t* part, int dir) {
+    const int64_t cols_p = cols_total / P;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols_p; ++j) {
+            const int64_t lo = i * cols_total + p * cols_p + j;
+            if (dir == 0) part[i * cols_p + j] = logical[lo];
+            else logical[lo] = part[i * cols_p + j];
+        }
+}
+
+void oracle_weights_padded_walk(const oracle_model* m, int TP, int r, int P, int64_t page_elems, int fused_qkv,
+                                int fused_gate_up, const oracle_weights* lg, const oracle_weights* sh, int dir) {
+    const int64_t hid = m->hidden, qrows = (int64_t)m->Hq * m->D, kvrows = (int64_t)m->Hkv * m->D, I = m->I;
+    const int n = P / TP;
+    const int64_t q_part = qrows / P * hid, kv_part = kvrows / P * hid, ffn_part = I / P * hid;
+    const int64_t pitch_q = oracle_padded_pitch(fused_qkv ? q_part + 2 * kv_part : q_part, page_elems);
+    const int64_t pitch_kv = oracle_padded_pitch(kv_part, page_elems);
+    const int64_t pitch_gate = oracle_padded_pitch(fused_gate_up ? 2 * ffn_part : ffn_part, page_elems);
+    const int64_t pitch_up = oracle_padded_pitch(ffn_part, page_elems);
+    const int64_t pitch_o = oracle_padded_pitch(q_part, page_elems);      /* [hidden, qrows/P] */
+    const int64_t pitch_down = oracle_padded_pitch(ffn_part, page_elems); /* [hidden, I/P] */
+    for (int j = 0; j < n; ++j) {
+        const int p = r * n + j; /* partition index among the P */
+        uint16_t* q_p = sh->q + j * pitch_q;
+        uint16_t* k_p = fused_qkv ? q_p + q_part : sh->k + j * pitch_kv;
+        uint16_t* v_p = fused_qkv ? k_p + kv_part : sh->v + j * pitch_kv;
+        uint16_t* gate_p = sh->gate + j * pitch_gate;
+        uint16_t* up_p = fused_gate_up ? gate_p + ffn_part : sh->up + j * pitch_up;
+        padded_rows(lg->q, qrows, hid, P, p, q_p, dir);
+        padded_rows(lg->k, kvrows, hid, P, p, k_p, dir);
+        padded_rows(lg->v, kvrows, hid, P, p, v_p, dir);
+        padded_rows(lg->gate, I, hid, P, p, gate_p, dir);
+        padded_rows(lg->up, I, hid, P, p, up_p, dir);
+        padded_cols(lg->o, hid, qrows, P, p, sh->o + j * pitch_o, dir);
+        padded_cols(lg->down, hid, I, P, p, sh->down + j * pitch_down, dir);
+    }
 }
