@@ -76,7 +76,27 @@ typedef struct {
     int32_t fused_qkv;     /* 1: worker buffer [q_r; k_r; v_r] (pointer in .q, .k/.v unused); 0: three buffers */
     int32_t fused_gate_up; /* 1: worker buffer [gate_r; up_r] (pointer in .gate, .up unused); 0: two buffers */
     int64_t kv_layer_stride_bytes; /* distance between layers inside a worker's pool; 0 = dense */
+    /* Weight padding (Sec. 3.2, "Improvement 1").  weight_pad_parts = P > 0: every weight buffer of a worker is P/tp
+     * partitions (P = the largest TP degree the instance may take; tp must divide P, P must divide the head counts
+     * and the FFN width), partition j starting at j * pitch, pitch = the partition's bytes rounded up to a multiple
+     * of weight_page_bytes (0 = 2 MiB, the allocation granularity the paper pads to).  A partition of q/k/v/gate/up
+     * is its rows; a partition of o_proj/down_proj is its own dense [hidden, columns/P] matrix (the paper's D_i); a
+     * fused buffer pads after each partition's [q;k;v] or [gate;up].  Pad bytes are never read or written.
+     * weight_pad_parts = 0: dense shards, no padding. */
+    int32_t weight_pad_parts;
+    int32_t reserved;
+    int64_t weight_page_bytes;
 } amoeba_layout;
+
+/* Padding arithmetic of one weight buffer of a layout (Sec. 3.2, Table 2 counts `pages` per tensor). */
+typedef struct {
+    int32_t partitions_per_worker; /* P/tp, or 1 without padding */
+    int32_t reserved;
+    int64_t partition_bytes;       /* bytes of one partition of this buffer */
+    int64_t pitch_bytes;           /* partition_bytes rounded up to whole pages (= partition_bytes without padding) */
+    int64_t page_bytes;
+    double pages;                  /* partition_bytes / page_bytes: fractional = the partition boundary is unaligned */
+} amoeba_pad_info;
 
 /* One worker's weight buffers for one layer (device pointers; unused slots NULL). */
 typedef struct {
@@ -88,6 +108,9 @@ typedef struct {
  * Errors: INVALID_ARG, UNSUPPORTED (same checks as amoeba_plan_create). */
 AMOEBA_API amoeba_status amoeba_layout_kv_pool_bytes(const amoeba_layout* layout, int64_t* bytes);
 AMOEBA_API amoeba_status amoeba_layout_weight_bytes(const amoeba_layout* layout, int32_t tensor, int64_t* bytes);
+/* Partition size, pitch and page count of buffer `tensor` (same numbering; a member of a fused buffer other than its
+ * first gives zeros).  Errors as above. */
+AMOEBA_API amoeba_status amoeba_layout_pad_info(const amoeba_layout* layout, int32_t tensor, amoeba_pad_info* out);
 
 typedef struct amoeba_plan amoeba_plan; /* opaque, host memory only */
 
@@ -274,7 +297,9 @@ AMOEBA_API amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_l
  * fixes which rows / columns each worker holds)
  *
  * src is a HOST array [a][num_layers] (worker-major) of device pointers, dst likewise [b][num_layers]; only layers
- * in [layer_begin, layer_end) are read.  A caller transforming a few layers per inference step (Sec. 3.3's
+ * in [layer_begin, layer_end) are read.  Either side may be padded (weight_pad_parts): padded -> padded moves whole
+ * partitions, dense <-> padded changes the pitch; pad bytes of the destination keep their values (zero them once at
+ * load time if a GEMM is to run over a whole padded buffer, Eq. 2).  A caller transforming a few layers per inference step (Sec. 3.3's
  * layer-by-layer order) passes successive ranges.
  */
 AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const amoeba_layer_weights* src,

@@ -50,7 +50,13 @@ class Model(C.Structure):
 class Layout(C.Structure):
     _fields_ = [("model", Model), ("tp", C.c_int32), ("block_tokens", C.c_int32), ("num_blocks", C.c_int32),
                 ("kv_order", C.c_int32), ("fused_qkv", C.c_int32), ("fused_gate_up", C.c_int32),
-                ("kv_layer_stride_bytes", C.c_int64)]
+                ("kv_layer_stride_bytes", C.c_int64), ("weight_pad_parts", C.c_int32), ("reserved", C.c_int32),
+                ("weight_page_bytes", C.c_int64)]
+
+
+class PadInfo(C.Structure):
+    _fields_ = [("partitions_per_worker", C.c_int32), ("reserved", C.c_int32), ("partition_bytes", C.c_int64),
+                ("pitch_bytes", C.c_int64), ("page_bytes", C.c_int64), ("pages", C.c_double)]
 
 
 class LayerWeights(C.Structure):
@@ -92,6 +98,7 @@ def _load():
         "amoeba_plan_destroy": (None, [VP]),
         "amoeba_layout_kv_pool_bytes": (I32, [P(Layout), P(I64)]),
         "amoeba_layout_weight_bytes": (I32, [P(Layout), I32, P(I64)]),
+        "amoeba_layout_pad_info": (I32, [P(Layout), I32, P(PadInfo)]),
         "amoeba_plan_bytes": (I32, [VP, I64, P(I64), P(I64)]),
         "amoeba_plan_kv_info": (I32, [VP, P(KvInfo)]),
         "amoeba_plan_num_weight_descs": (I32, [VP]),
@@ -152,11 +159,12 @@ class Plan:
 
 def make_layout(model: dict, tp: int, num_blocks: int, block_tokens: int = 16, fused_qkv: bool = True,
                 fused_gate_up: bool = True, elem_bytes: int = 2, kv_layer_stride_bytes: int = 0,
-                kv_order: int = 0) -> Layout:
-    """Layout from a shape dict with keys L, hidden, Hq, Hkv, D, I; kv_order KV_HEAD_MAJOR or KV_TOKEN_MAJOR."""
+                kv_order: int = 0, weight_pad_parts: int = 0, weight_page_bytes: int = 0) -> Layout:
+    """Layout from a shape dict with keys L, hidden, Hq, Hkv, D, I; kv_order KV_HEAD_MAJOR or KV_TOKEN_MAJOR;
+    weight_pad_parts > 0: padded weight partitions (page 0 = 2 MiB)."""
     m = Model(model["L"], model["hidden"], model["Hq"], model["Hkv"], model["D"], model["I"], elem_bytes)
     return Layout(m, tp, block_tokens, num_blocks, int(kv_order), int(fused_qkv), int(fused_gate_up),
-                  kv_layer_stride_bytes)
+                  kv_layer_stride_bytes, int(weight_pad_parts), 0, int(weight_page_bytes))
 
 
 def amoeba_status_string(status: int) -> str:
@@ -179,6 +187,15 @@ def amoeba_layout_weight_bytes(layout: Layout, tensor: int) -> int:
     out = C.c_int64()
     _check(_load().amoeba_layout_weight_bytes(C.byref(layout), tensor, C.byref(out)), "amoeba_layout_weight_bytes")
     return out.value
+
+
+def amoeba_layout_pad_info(layout: Layout, tensor: int) -> PadInfo:
+    out = PadInfo()
+    _check(_load().amoeba_layout_pad_info(C.byref(layout), tensor, C.byref(out)), "amoeba_layout_pad_info")
+    return out
+
+
+__all__ += ["PadInfo", "amoeba_layout_pad_info"]
 
 
 def amoeba_plan_destroy(plan: Plan) -> None:

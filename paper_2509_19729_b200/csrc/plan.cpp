@@ -32,7 +32,54 @@ static amoeba_status check_layout(const amoeba_layout& l) {
     // tp > num_kv_heads is not a re-layout of existing state and is not handled.
     if (m.num_q_heads % l.tp || m.num_kv_heads % l.tp || m.intermediate % l.tp) return AMOEBA_ERR_UNSUPPORTED;
     if (m.num_q_heads % m.num_kv_heads) return AMOEBA_ERR_UNSUPPORTED;
+    if (l.weight_pad_parts < 0 || l.weight_page_bytes < 0) return AMOEBA_ERR_INVALID_ARG;
+    if (l.weight_pad_parts > 0) {
+        const int P = l.weight_pad_parts;
+        if (P > 4 * AMOEBA_MAX_TP || P % l.tp || m.num_q_heads % P || m.num_kv_heads % P || m.intermediate % P)
+            return AMOEBA_ERR_UNSUPPORTED;
+        if (l.weight_page_bytes % 16) return AMOEBA_ERR_ALIGNMENT;
+    }
     return AMOEBA_OK;
+}
+
+// ---- how one layout stores the weights: every buffer is `parts` partitions, `per_worker` of them per worker, each
+// `block` bytes at a pitch of `pitch` bytes (dense shards: one partition per worker, parts = tp).
+constexpr int64_t kDefaultPageBytes = 2 << 20;
+enum { Q, K, V, O, GATE, UP, DOWN };
+
+struct WeightForm {
+    int parts, per_worker;
+    int64_t page;
+    int64_t block[kNumTensors], pitch[kNumTensors];  // per buffer (0 for a member folded into a fused buffer)
+    int buffer_of[kNumTensors];                      // buffer that holds the member
+    int64_t member_off[kNumTensors];                 // byte offset of the member inside a partition of its buffer
+};
+
+static WeightForm weight_form(const amoeba_layout& l) {
+    const amoeba_model& m = l.model;
+    WeightForm f{};
+    const bool padded = l.weight_pad_parts > 0;
+    f.parts = padded ? l.weight_pad_parts : l.tp;
+    f.per_worker = f.parts / l.tp;
+    f.page = padded ? (l.weight_page_bytes ? l.weight_page_bytes : kDefaultPageBytes) : 1;
+    const int64_t e = m.elem_bytes, hid = m.hidden;
+    const int64_t q = (int64_t)m.num_q_heads * m.head_dim / f.parts * hid * e;
+    const int64_t kv = (int64_t)m.num_kv_heads * m.head_dim / f.parts * hid * e;
+    const int64_t ffn = (int64_t)m.intermediate / f.parts * hid * e;
+    for (int t = 0; t < kNumTensors; ++t) f.buffer_of[t] = t;
+    f.block[Q] = q, f.block[K] = f.block[V] = kv, f.block[O] = q, f.block[GATE] = f.block[UP] = f.block[DOWN] = ffn;
+    if (l.fused_qkv) {
+        f.block[Q] = q + 2 * kv, f.block[K] = f.block[V] = 0;
+        f.buffer_of[K] = f.buffer_of[V] = Q;
+        f.member_off[K] = q, f.member_off[V] = q + kv;
+    }
+    if (l.fused_gate_up) {
+        f.block[GATE] = 2 * ffn, f.block[UP] = 0;
+        f.buffer_of[UP] = GATE;
+        f.member_off[UP] = ffn;
+    }
+    for (int t = 0; t < kNumTensors; ++t) f.pitch[t] = (f.block[t] + f.page - 1) / f.page * f.page;
+    return f;
 }
 
 // Largest divisor d of `total` with d <= cap and d % 16 == 0 (total % 16 == 0 is a precondition).
@@ -147,53 +194,64 @@ struct Range {
 };
 static Range part(int64_t total, int tp, int r) { return {total / tp * r, total / tp * (r + 1)}; }
 
-// Tensors partitioned by output rows: shard r holds rows part(rows, tp, r) of the logical [rows, cols] tensor.
-// `sec_src` / `sec_dst` are the byte offsets of this tensor's section inside a fused worker buffer.
-static void add_row_split(std::vector<amoeba_weight_desc>& out, int a, int b, int64_t rows, int64_t row_bytes,
-                          int src_tensor, int64_t sec_src, int dst_tensor, int64_t sec_dst) {
-    for (int i = 0; i < a; ++i)
-        for (int j = 0; j < b; ++j) {
-            const Range s = part(rows, a, i), d = part(rows, b, j);
+// Descriptors of one weight member between two forms.  The member has `units` rows (split_rows) or columns along
+// its partition axis; partition p of a form covers units [p*units/parts, (p+1)*units/parts) and lives in worker
+// p / per_worker at byte (p % per_worker) * pitch + member_off of the member's buffer.  Every intersection of a source
+// partition with a destination partition is one copy: contiguous for a row split (unit_bytes = bytes of one row),
+// `rows` strided runs for a column split (unit_bytes = bytes of one element), contiguous again when the common range
+// is a whole partition on both sides.
+static void add_member(std::vector<amoeba_weight_desc>& out, const WeightForm& fs, const WeightForm& fd, int member,
+                       int64_t units, int64_t unit_bytes, bool split_rows, int64_t rows) {
+    const int bs = fs.buffer_of[member], bd = fd.buffer_of[member];
+    for (int ps = 0; ps < fs.parts; ++ps)
+        for (int pd = 0; pd < fd.parts; ++pd) {
+            const Range s = part(units, fs.parts, ps), d = part(units, fd.parts, pd);
             const int64_t lo = std::max(s.lo, d.lo), hi = std::min(s.hi, d.hi);
             if (lo >= hi) continue;
             amoeba_weight_desc w{};
-            w.src_rank = i;
-            w.dst_rank = j;
-            w.src_tensor = src_tensor;
-            w.dst_tensor = dst_tensor;
-            w.src_off = sec_src + (lo - s.lo) * row_bytes;
-            w.dst_off = sec_dst + (lo - d.lo) * row_bytes;
-            w.row_bytes = (hi - lo) * row_bytes;  // consecutive rows are one contiguous run
-            w.n_rows = 1;
-            w.src_pitch = w.dst_pitch = w.row_bytes;
-            out.push_back(w);
-        }
-}
-
-// Tensors partitioned by input columns: shard r holds columns part(cols, tp, r) of the logical [rows, cols]
-// tensor as a dense [rows, cols/tp] buffer.
-static void add_col_split(std::vector<amoeba_weight_desc>& out, int a, int b, int64_t rows, int64_t cols, int64_t e,
-                          int tensor) {
-    for (int i = 0; i < a; ++i)
-        for (int j = 0; j < b; ++j) {
-            const Range s = part(cols, a, i), d = part(cols, b, j);
-            const int64_t lo = std::max(s.lo, d.lo), hi = std::min(s.hi, d.hi);
-            if (lo >= hi) continue;
-            amoeba_weight_desc w{};
-            w.src_rank = i;
-            w.dst_rank = j;
-            w.src_tensor = w.dst_tensor = tensor;
-            w.src_off = (lo - s.lo) * e;
-            w.dst_off = (lo - d.lo) * e;
-            w.row_bytes = (hi - lo) * e;
-            w.n_rows = (int32_t)rows;
-            w.src_pitch = (s.hi - s.lo) * e;
-            w.dst_pitch = (d.hi - d.lo) * e;
-            if (w.src_pitch == w.row_bytes && w.dst_pitch == w.row_bytes) {  // both dense: one run
-                w.row_bytes *= rows;
+            w.src_rank = ps / fs.per_worker;
+            w.dst_rank = pd / fd.per_worker;
+            w.src_tensor = bs;
+            w.dst_tensor = bd;
+            const int64_t sbase = (ps % fs.per_worker) * fs.pitch[bs] + fs.member_off[member];
+            const int64_t dbase = (pd % fd.per_worker) * fd.pitch[bd] + fd.member_off[member];
+            w.src_off = sbase + (lo - s.lo) * unit_bytes;
+            w.dst_off = dbase + (lo - d.lo) * unit_bytes;
+            w.row_bytes = (hi - lo) * unit_bytes;
+            if (split_rows) {  // consecutive rows are one contiguous run
                 w.n_rows = 1;
                 w.src_pitch = w.dst_pitch = w.row_bytes;
+            } else {
+                w.n_rows = (int32_t)rows;
+                w.src_pitch = (s.hi - s.lo) * unit_bytes;
+                w.dst_pitch = (d.hi - d.lo) * unit_bytes;
+                if (w.src_pitch == w.row_bytes && w.dst_pitch == w.row_bytes) {  // whole partition on both sides
+                    w.row_bytes *= rows;
+                    w.n_rows = 1;
+                    w.src_pitch = w.dst_pitch = w.row_bytes;
+                }
             }
+            // Fold an arithmetic progression of equal contiguous runs (partition after partition between the same
+            // two workers) into one 2-D descriptor.
+            if (!out.empty() && w.n_rows == 1) {
+                amoeba_weight_desc& p = out.back();
+                const bool same = p.src_rank == w.src_rank && p.dst_rank == w.dst_rank && p.src_tensor == w.src_tensor &&
+                                  p.dst_tensor == w.dst_tensor && p.row_bytes == w.row_bytes &&
+                                  (p.reserved & 255) == member + 1;
+                const bool foldable = (p.reserved & 256) != 0;
+                if (same && p.n_rows == 1 && w.src_off > p.src_off && w.dst_off > p.dst_off) {
+                    p.src_pitch = w.src_off - p.src_off;
+                    p.dst_pitch = w.dst_off - p.dst_off;
+                    p.n_rows = 2;
+                    continue;
+                }
+                if (same && p.n_rows > 1 && foldable && w.src_off == p.src_off + p.n_rows * p.src_pitch &&
+                    w.dst_off == p.dst_off + p.n_rows * p.dst_pitch) {
+                    ++p.n_rows;
+                    continue;
+                }
+            }
+            w.reserved = (member + 1) | (w.n_rows == 1 ? 256 : 0);  // building notes, cleared by the caller
             out.push_back(w);
         }
 }
@@ -250,19 +308,16 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
     const int64_t hid = m.hidden, qrows = (int64_t)m.num_q_heads * m.head_dim,
                   kvrows = (int64_t)m.num_kv_heads * m.head_dim, I = m.intermediate;
     const int64_t rb = hid * e;  // bytes of one [*, hidden] row
-    enum { Q, K, V, O, GATE, UP, DOWN };
     auto& w = p->wdescs;
-    // fused buffers: [q_r; k_r; v_r] and [gate_r; up_r], named by their first member
-    const int64_t k_sec_s = src->fused_qkv ? qrows / a * rb : 0, v_sec_s = src->fused_qkv ? (qrows + kvrows) / a * rb : 0;
-    const int64_t k_sec_d = dst->fused_qkv ? qrows / b * rb : 0, v_sec_d = dst->fused_qkv ? (qrows + kvrows) / b * rb : 0;
-    add_row_split(w, a, b, qrows, rb, Q, 0, Q, 0);
-    add_row_split(w, a, b, kvrows, rb, src->fused_qkv ? Q : K, k_sec_s, dst->fused_qkv ? Q : K, k_sec_d);
-    add_row_split(w, a, b, kvrows, rb, src->fused_qkv ? Q : V, v_sec_s, dst->fused_qkv ? Q : V, v_sec_d);
-    add_col_split(w, a, b, hid, qrows, e, O);
-    add_row_split(w, a, b, I, rb, GATE, 0, GATE, 0);
-    add_row_split(w, a, b, I, rb, src->fused_gate_up ? GATE : UP, src->fused_gate_up ? I / a * rb : 0,
-                  dst->fused_gate_up ? GATE : UP, dst->fused_gate_up ? I / b * rb : 0);
-    add_col_split(w, a, b, hid, I, e, DOWN);
+    const WeightForm fs = weight_form(*src), fd = weight_form(*dst);
+    add_member(w, fs, fd, Q, qrows, rb, true, 0);
+    add_member(w, fs, fd, K, kvrows, rb, true, 0);
+    add_member(w, fs, fd, V, kvrows, rb, true, 0);
+    add_member(w, fs, fd, O, qrows, e, false, hid);
+    add_member(w, fs, fd, GATE, I, rb, true, 0);
+    add_member(w, fs, fd, UP, I, rb, true, 0);
+    add_member(w, fs, fd, DOWN, I, e, false, hid);
+    for (auto& d : w) d.reserved = 0;
     if ((int)w.size() > kMaxWeightDescs) {
         delete p;
         return AMOEBA_ERR_UNSUPPORTED;
@@ -306,19 +361,24 @@ amoeba_status amoeba_layout_weight_bytes(const amoeba_layout* l, int32_t tensor,
     if (!l || !bytes || tensor < 0 || tensor >= kNumTensors) return AMOEBA_ERR_INVALID_ARG;
     const amoeba_status st = check_layout(*l);
     if (st != AMOEBA_OK) return st;
-    const amoeba_model& m = l->model;
-    const int64_t e = m.elem_bytes, hid = m.hidden, q = (int64_t)m.num_q_heads * m.head_dim / l->tp,
-                  kv = (int64_t)m.num_kv_heads * m.head_dim / l->tp, I = m.intermediate / l->tp;
-    int64_t rows = 0;  // rows of `hidden` elements each ([rows, hidden] or [hidden, rows]: same byte count)
-    switch (tensor) {
-        case 0: rows = l->fused_qkv ? q + 2 * kv : q; break;
-        case 1: case 2: rows = l->fused_qkv ? 0 : kv; break;
-        case 3: rows = q; break;
-        case 4: rows = l->fused_gate_up ? 2 * I : I; break;
-        case 5: rows = l->fused_gate_up ? 0 : I; break;
-        case 6: rows = I; break;
-    }
-    *bytes = rows * hid * e;
+    const WeightForm f = weight_form(*l);
+    // dense shards: the one partition; padded: per_worker partitions at the padded pitch
+    *bytes = f.block[tensor] ? (l->weight_pad_parts > 0 ? f.per_worker * f.pitch[tensor] : f.block[tensor]) : 0;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_layout_pad_info(const amoeba_layout* l, int32_t tensor, amoeba_pad_info* out) {
+    if (!l || !out || tensor < 0 || tensor >= kNumTensors) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_status st = check_layout(*l);
+    if (st != AMOEBA_OK) return st;
+    const WeightForm f = weight_form(*l);
+    const int64_t page = l->weight_pad_parts > 0 ? f.page : (l->weight_page_bytes ? l->weight_page_bytes : kDefaultPageBytes);
+    *out = amoeba_pad_info{};
+    out->partitions_per_worker = f.block[tensor] ? f.per_worker : 0;
+    out->partition_bytes = f.block[tensor];
+    out->pitch_bytes = f.pitch[tensor];
+    out->page_bytes = page;
+    out->pages = (double)f.block[tensor] / (double)page;
     return AMOEBA_OK;
 }
 

@@ -30,20 +30,21 @@ class Session:
 
     model: shape dict (L, hidden, Hq, Hkv, D, I); a, b: source / destination TP; NB_src / NB_dst: pool capacities;
     kv_layers: number of layers the KV pools hold (the first kv_layers layers; None = all); weights: allocate the
-    weight shards too.  Buffers are uint8 tensors; KV pools are one tensor per worker.
+    weight shards too; src_weight_pad / dst_weight_pad: (partitions P, page bytes) for padded weight buffers.  Buffers are uint8 tensors; KV pools are one tensor per worker.
     """
 
     def __init__(self, model: dict, a: int, b: int, NB_src: int, NB_dst: int, num_seqs: int, max_blocks_per_seq: int,
                  pairs_cap: int, kv_layers: Optional[int] = None, kv: bool = True, weights: bool = True,
                  fused_qkv: bool = True, fused_gate_up: bool = True, block_tokens: int = 16, device="cuda:0",
                  dst_fill: Optional[int] = 0xA5, src_kv_order: int = A.KV_HEAD_MAJOR,
-                 dst_kv_order: int = A.KV_HEAD_MAJOR):
+                 dst_kv_order: int = A.KV_HEAD_MAJOR, src_weight_pad=None, dst_weight_pad=None):
         self.model, self.a, self.b = model, a, b
         self.device = torch.device(device)
+        pad = lambda p: dict(weight_pad_parts=p[0], weight_page_bytes=p[1]) if p else {}  # (P, page bytes) or None
         self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up,
-                                        kv_order=src_kv_order)
+                                        kv_order=src_kv_order, **pad(src_weight_pad))
         self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up,
-                                        kv_order=dst_kv_order)
+                                        kv_order=dst_kv_order, **pad(dst_weight_pad))
         self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
         self.info = A.amoeba_plan_kv_info(self.plan)
         self.L = model["L"]

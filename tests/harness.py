@@ -16,11 +16,12 @@ class Case:
 
 def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_slack=0.25, dst_occupied=0.3, seed=0,
               fused_qkv=True, fused_gate_up=True, weights=True, kv=True, dtype="bf16", free_override=None,
-              src_bt_override=None, pairs_cap=None, src_order=0, dst_order=0):
+              src_bt_override=None, pairs_cap=None, src_order=0, dst_order=0, src_pad=None, dst_pad=None):
     """Seeded inputs + the oracle's expected outputs for one TP a->b transformation."""
     c = Case()
     c.model, c.a, c.b, c.T, c.fq, c.fg = model, a, b, T, fused_qkv, fused_gate_up
     c.src_order, c.dst_order = src_order, dst_order  # 0 header-centric, 1 token-first (same codes on both sides)
+    c.src_pad, c.dst_pad = src_pad, dst_pad          # (partitions P, page bytes) of padded weight buffers, or None
     cfg = dict(model=model, dtype=dtype, S=len(seq_lens), src_free=src_free, dst_form=dst_form, dst_slack=dst_slack,
                dst_occupied=dst_occupied)
     st = wl.draw_kv_state(cfg, seed=seed, name="case", seq_lens=np.maximum(np.asarray(seq_lens), 0), T=T)
@@ -62,6 +63,15 @@ def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_sl
         c.src_w, c.exp_dst_w = [], []
         for l in range(L):
             W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in oracle.logical_shapes(model).items()}
+            if src_pad or dst_pad:
+                opad = lambda pad: (pad[0], pad[1] // 2) if pad else None  # the oracle counts pages in elements
+                sa = (oracle.weights_shard_padded(W, model, a, *opad(src_pad), fused_qkv, fused_gate_up, fill=0x5A5A)
+                      if src_pad else oracle.weights_shard(W, model, a, fused_qkv, fused_gate_up))
+                c.src_w.append(sa)
+                c.exp_dst_w.append(oracle.weights_transform_any(sa, model, a, b, fused_qkv, fused_gate_up,
+                                                                src_pad=opad(src_pad), dst_pad=opad(dst_pad),
+                                                                fill=FILL16))
+                continue
             sa = oracle.weights_shard(W, model, a, fused_qkv, fused_gate_up)
             c.src_w.append(sa)
             c.exp_dst_w.append(oracle.weights_transform(sa, model, a, b, fused_qkv, fused_gate_up))
@@ -77,7 +87,8 @@ def run_case(c, copy_path=None, options=(), device="cuda:0", steps=1):
 
     s = Session(c.model, c.a, c.b, c.NB_src, c.NB_dst, len(c.seq_lens), c.maxb, c.pairs_cap, kv=c.kv,
                 weights=c.weights, fused_qkv=c.fq, fused_gate_up=c.fg, block_tokens=c.T, device=device,
-                src_kv_order=c.src_order, dst_kv_order=c.dst_order)
+                src_kv_order=c.src_order, dst_kv_order=c.dst_order, src_weight_pad=c.src_pad,
+                dst_weight_pad=c.dst_pad)
     if copy_path is not None:
         s.set_option(A.OPT_COPY_PATH, copy_path)
     for opt, val in options:

@@ -259,3 +259,23 @@ def test_token_first_full_transformation_with_weights_and_mask():
     lens = list(np.random.default_rng(4).integers(1, 400, size=60))
     c = make_case(GQA, 2, 4, lens, dst_form="mask", dst_occupied=0.3, src_free=0.3, seed=21, src_order=TF, dst_order=TF)
     check_case(c, run_case(c))
+
+
+# ---- padded weight partitions (Sec. 3.2, Improvement 1): every byte of every padded buffer, pads included
+PADM = dict(L=2, hidden=256, Hq=16, Hkv=8, D=32, I=768)
+PAD_CASES = [(1, 4, (4, 4096), (4, 4096)), (4, 1, (4, 4096), (4, 4096)), (2, 4, (8, 2048), (8, 2048)),
+             (1, 4, (4, 4096), None), (4, 2, None, (4, 4096)), (2, 4, (8, 8192), (4, 4096)), (2, 1, (2, 4096), (8, 1024)),
+             (1, 1, None, (8, 8192)), (8, 8, (8, 4096), None)]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("a,b,sp,dp", PAD_CASES)
+def test_padded_weight_partitions(path, a, b, sp, dp):
+    c = make_case(PADM, a, b, [20], kv=False, seed=a * 8 + b, src_pad=sp, dst_pad=dp)
+    check_case(c, run_case(c, path))
+
+
+@pytest.mark.parametrize("fq,fg", [(False, False), (True, False)])
+def test_padded_unfused_buffers_and_kv_together(fq, fg):
+    c = make_case(PADM, 2, 4, [40, 3], fused_qkv=fq, fused_gate_up=fg, seed=12, src_pad=(4, 4096), dst_pad=(4, 4096))
+    check_case(c, run_case(c))

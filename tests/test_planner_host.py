@@ -155,3 +155,87 @@ def test_unknown_kv_order_is_unsupported():
     with pytest.raises(A.AmoebaError) as e:
         A.amoeba_plan_create(A.make_layout(odd, 1, 8, kv_order=1), A.make_layout(odd, 2, 8, kv_order=1))
     assert e.value.status == A.ERR_ALIGNMENT
+
+
+# ---- padded weight partitions (Sec. 3.2, Improvement 1)
+PADM = dict(L=1, hidden=32, Hq=16, Hkv=8, D=8, I=192)  # every partition size is a multiple of 16 bytes down to P = 8
+PAD_CASES = [  # a, b, source (P, page bytes) or None, destination (P, page bytes) or None
+    (1, 4, (4, 2048), (4, 2048)), (4, 1, (4, 2048), (4, 2048)), (2, 4, (8, 1024), (8, 1024)), (1, 4, (4, 2048), None),
+    (4, 2, None, (4, 2048)), (2, 4, (8, 4096), (4, 2048)), (2, 1, (2, 2048), (8, 512)), (1, 1, None, (8, 4096)),
+    (8, 8, (8, 2048), None), (4, 4, (4, 2048), (4, 512)),
+]
+
+
+@pytest.mark.parametrize("fq,fg", [(True, True), (False, False)])
+@pytest.mark.parametrize("a,b,sp,dp", PAD_CASES)
+def test_padded_weight_descriptors_reproduce_oracle(oracle, a, b, sp, dp, fq, fg):
+    m = PADM
+    g = np.random.default_rng(a * 100 + b)
+    W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in oracle.logical_shapes(m).items()}
+    opad = lambda pad: (pad[0], pad[1] // 2) if pad else None   # the oracle counts pages in elements
+    src = oracle.weights_shard_padded(W, m, a, *opad(sp), fq, fg) if sp else oracle.weights_shard(W, m, a, fq, fg)
+    exp = oracle.weights_transform_any(src, m, a, b, fq, fg, src_pad=opad(sp), dst_pad=opad(dp), fill=0xA5A5)
+    lay = lambda tp, pad: A.make_layout(m, tp, 4, fused_qkv=fq, fused_gate_up=fg, weight_pad_parts=pad[0] if pad else 0,
+                                        weight_page_bytes=pad[1] if pad else 0)
+    plan = A.amoeba_plan_create(lay(a, sp), lay(b, dp))
+    as_bytes = lambda sh: [[sh_r[n].reshape(-1).view(np.uint8) if n in sh_r else None for n in A.TENSOR_NAMES]
+                           for sh_r in sh]
+    dst = [[np.full(e.size, 0xA5, np.uint8) if e is not None else None for e in r] for r in as_bytes(exp)]
+    counts = _apply_descs(plan, as_bytes(src), dst)
+    total = 0
+    for r in range(b):
+        for t, n in enumerate(A.TENSOR_NAMES):
+            if n in exp[r]:
+                assert A.amoeba_layout_weight_bytes(lay(b, dp), t) == exp[r][n].size * 2, (r, n)
+                assert np.array_equal(dst[r][t], exp[r][n].reshape(-1).view(np.uint8)), (r, n)
+                assert counts[r][t].max() == 1      # no byte written twice; pad bytes never written
+                total += int(counts[r][t].sum())
+            else:
+                assert A.amoeba_layout_weight_bytes(lay(b, dp), t) == 0
+    assert total == sum(x.size * 2 for x in W.values())  # every weight byte written exactly once
+    _, w = A.amoeba_plan_bytes(plan, 0)
+    assert w == 2 * total
+
+
+def test_padded_partitions_fold_into_few_descriptors():
+    """Padded -> padded moves whole partitions: per (source worker, destination worker, tensor) one 2-D descriptor whose
+    rows are the partitions, not one descriptor per partition."""
+    m = dict(L=1, hidden=64, Hq=32, Hkv=32, D=8, I=512)
+    lay = lambda tp: A.make_layout(m, tp, 4, weight_pad_parts=32, weight_page_bytes=4096)
+    plan = A.amoeba_plan_create(lay(1), lay(4))
+    n = A.amoeba_plan_num_weight_descs(plan)
+    assert n == 7 * 4
+    d = A.amoeba_plan_weight_desc(plan, 0)
+    assert d.n_rows == 8 and d.src_pitch == d.dst_pitch  # 8 partitions per destination worker, same pitch both sides
+
+
+def test_pad_info_reproduces_table2():
+    rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table2_pages.txt"))
+            if l.strip() and not l.startswith("#")]
+    for name, hidden, inter, experts, fused, p1, p4 in rows:
+        # an expert-parallel FFN tensor holds `experts` matrices: the page arithmetic sees hidden x (inter * experts)
+        I = int(inter) * int(experts) * int(fused)
+        m = dict(L=1, hidden=int(hidden), Hq=64, Hkv=64, D=int(hidden) // 64, I=I)
+        for tp, printed in ((1, p1), (4, p4)):
+            info = A.amoeba_layout_pad_info(A.make_layout(m, tp, 4, fused_gate_up=False, weight_pad_parts=tp), 6)
+            digits = len(printed.split(".")[1]) if "." in printed else 0
+            assert abs(info.pages - float(printed)) <= 0.5 * 10.0 ** -digits + 1e-9, (name, tp, info.pages)
+            assert info.page_bytes == 2 << 20 and info.partitions_per_worker == 1
+            assert info.pitch_bytes == -(-info.partition_bytes // info.page_bytes) * info.page_bytes
+    # Qwen2.5-32B at TP4: 33.75 pages per partition -> padded to 34; Llama-3.1-70B: 56, already aligned
+    qwen = A.make_layout(dict(L=1, hidden=5120, Hq=40, Hkv=8, D=128, I=27648), 1, 4, weight_pad_parts=4)
+    assert A.amoeba_layout_pad_info(qwen, 6).pitch_bytes == 34 * (2 << 20)
+    assert A.amoeba_layout_weight_bytes(qwen, 6) == 4 * 34 * (2 << 20)
+    llama = A.make_layout(dict(L=1, hidden=8192, Hq=64, Hkv=8, D=128, I=28672), 4, 4, weight_pad_parts=4)
+    assert A.amoeba_layout_pad_info(llama, 6).pitch_bytes == 56 * (2 << 20) == A.amoeba_layout_weight_bytes(llama, 6)
+
+
+def test_padded_layout_validation():
+    m = PADM
+    for kw, status in ((dict(weight_pad_parts=3), A.ERR_UNSUPPORTED),          # tp = 2 does not divide P = 3
+                       (dict(weight_pad_parts=16), A.ERR_UNSUPPORTED),         # P = 16 does not divide Hkv = 8
+                       (dict(weight_pad_parts=-1), A.ERR_INVALID_ARG),
+                       (dict(weight_pad_parts=4, weight_page_bytes=100), A.ERR_ALIGNMENT)):
+        with pytest.raises(A.AmoebaError) as e:
+            A.amoeba_plan_create(A.make_layout(m, 2, 4, **kw), A.make_layout(m, 2, 4))
+        assert e.value.status == status, kw
