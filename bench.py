@@ -217,7 +217,7 @@ KV_ORDERS = {"head": (0, 0), "token": (1, 1), "token2head": (1, 0), "head2token"
 
 
 def build_session(cfg_name: str, device, layers=None, kv=True, weights=True, seed=wl.DEFAULT_SEED, fill=True,
-                  kv_order="head"):
+                  kv_order="head", weight_pad=0):
     import torch
 
     from paper_2509_19729_b200.session import Session
@@ -231,7 +231,9 @@ def build_session(cfg_name: str, device, layers=None, kv=True, weights=True, see
     st = wl.draw_kv_state(cfg, seed=seed, name=cfg_name)
     s = Session(m, cfg["a"], cfg["b"], st["NB_src"], st["NB_dst"], cfg["S"], st["maxb"], st["n_live"],
                 kv_layers=kv_layers, kv=kv, weights=weights, device=device, dst_fill=None,
-                src_kv_order=KV_ORDERS[kv_order][0], dst_kv_order=KV_ORDERS[kv_order][1])
+                src_kv_order=KV_ORDERS[kv_order][0], dst_kv_order=KV_ORDERS[kv_order][1],
+                src_weight_pad=(weight_pad, 0) if weight_pad else None,
+                dst_weight_pad=(weight_pad, 0) if weight_pad else None)
     s.set_tables(st["seq_lens"], st["src_bt"], st.get("dst_free_list"), st.get("dst_free_mask"))
     if fill:
         for i, p in enumerate(s.src_pools):
@@ -368,12 +370,13 @@ def run_e2e(args, device, world):
     L_full = cfg["model"]["L"]
     # size the layer slice so that the pinned host buffers stay within the cap
     budget = min(int(args.e2e_gib * 2**30), host_free_bytes() // 3)
-    s1, st = build_session(args.config, device, layers=1, fill=False, kv_order=args.kv_order)
+    s1, st = build_session(args.config, device, layers=1, fill=False, kv_order=args.kv_order,
+                           weight_pad=args.weight_pad)
     per_layer = sum(p.numel() for p in s1.src_pools + s1.dst_pools + s1._wbufs)
     del s1
     torch.cuda.empty_cache()
     layers = int(max(1, min(L_full, budget // max(per_layer, 1))))
-    s, st = build_session(args.config, device, layers=layers, kv_order=args.kv_order)
+    s, st = build_session(args.config, device, layers=layers, kv_order=args.kv_order, weight_pad=args.weight_pad)
     kvl = s.kv_layers
     a = cfg["a"]
 
@@ -480,6 +483,8 @@ def main():
     ap.add_argument("--kv-order", default="head", choices=list(KV_ORDERS),
                     help="KV storage order: header-centric on both sides (default), token-first on both sides, or a "
                          "conversion between them")
+    ap.add_argument("--weight-pad", type=int, default=0,
+                    help="P > 0: both sides hold their weights as P padded partitions per tensor (2 MiB pages)")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -503,7 +508,8 @@ def main():
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     cfg = wl.CONFIGS[args.config]
-    s, st = build_session(args.config, device, layers=args.layers, kv_order=args.kv_order)
+    s, st = build_session(args.config, device, layers=args.layers, kv_order=args.kv_order,
+                          weight_pad=args.weight_pad)
     for opt, val in ((A.OPT_COPY_PATH, args.copy_path), (A.OPT_CHUNK_BYTES, args.chunk), (A.OPT_STAGES, args.stages),
                      (A.OPT_CTAS_PER_SM, args.ctas_per_sm)):
         if val:
@@ -567,7 +573,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']}", "layers": n_seq_layers[0], "kv_layers": n_seq_layers[1],
-                   "kv_order": args.kv_order, "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
+                   "kv_order": args.kv_order, "weight_pad_parts": args.weight_pad, "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
                    "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
                    "l2_policy": "no flush: every step streams far more than the 126 MB L2",
                    "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],

@@ -171,3 +171,33 @@ def test_full_size_inplace_merge(oracle):
     finally:
         del s
         torch.cuda.empty_cache()
+
+
+def test_full_size_padded_weights(oracle):
+    """Llama-3-8B-shaped weights held as 4 padded partitions per tensor (2 MiB pages) on both sides, TP 1 -> 4: two
+    layers compared whole with the oracle, pad bytes included (they keep the destination's fill)."""
+    import torch
+
+    import bench
+
+    name, P = "llama3_8b_1to4", 4
+    cfg = wl.CONFIGS[name]
+    m, a, b = cfg["model"], cfg["a"], cfg["b"]
+    s, st = bench.build_session(name, torch.device("cuda:0"), kv=False, weight_pad=P)
+    try:
+        s.status.zero_()
+        s.reshard_weights()
+        torch.cuda.synchronize()
+        assert int(s.status.item()) == 0
+        page_elems = (2 << 20) // 2
+        for l in (0, m["L"] - 1):
+            src_sh = [{n: t.cpu().numpy().view(np.uint16) for n, t in s.src_w[r][l].items()} for r in range(a)]
+            exp = oracle.weights_transform_any(src_sh, m, a, b, src_pad=(P, page_elems), dst_pad=(P, page_elems),
+                                               fill=0xA5A5)
+            for r in range(b):
+                for n, e in exp[r].items():
+                    got = s.dst_w[r][l][n].cpu().numpy().view(np.uint16)
+                    assert np.array_equal(got, e), (l, r, n)
+    finally:
+        del s
+        torch.cuda.empty_cache()
