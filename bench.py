@@ -485,6 +485,9 @@ def main():
                          "conversion between them")
     ap.add_argument("--weight-pad", type=int, default=0,
                     help="P > 0: both sides hold their weights as P padded partitions per tensor (2 MiB pages)")
+    ap.add_argument("--layers-per-call", type=int, default=0,
+                    help="k > 0: transform k layers per call (KV and weights), as when a few layers are transformed "
+                         "per inference step; 0 = all layers in one call")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -534,14 +537,19 @@ def main():
     t_begin, t_end = ev(), ev()
     torch.cuda.synchronize()
     t_begin.record(stream)
+    k = args.layers_per_call
+    kv_ranges = [(l, min(l + k, s.kv_layers)) for l in range(0, s.kv_layers, k)] if k else [(0, s.kv_layers)]
+    w_ranges = [(l, min(l + k, s.L)) for l in range(0, s.L, k)] if k else [(0, s.L)]
     for _ in range(args.steps):
         m = [ev() for _ in range(4)]
         m[0].record(stream)
         s.rewrite_block_tables()
         m[1].record(stream)
-        s.reshard_kv()
+        for lo, hi in kv_ranges:
+            s.reshard_kv(None, lo, hi)
         m[2].record(stream)
-        s.reshard_weights()
+        for lo, hi in w_ranges:
+            s.reshard_weights(None, lo, hi)
         m[3].record(stream)
         marks.append(m)
     t_end.record(stream)
@@ -573,7 +581,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']}", "layers": n_seq_layers[0], "kv_layers": n_seq_layers[1],
-                   "kv_order": args.kv_order, "weight_pad_parts": args.weight_pad, "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
+                   "layers_per_call": args.layers_per_call or "all", "kv_order": args.kv_order, "weight_pad_parts": args.weight_pad, "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
                    "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
                    "l2_policy": "no flush: every step streams far more than the 126 MB L2",
                    "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],

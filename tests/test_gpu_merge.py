@@ -171,3 +171,37 @@ def test_merge_host_detected_errors():
                                                        live, 0, 1, z)) == A.ERR_ALIGNMENT
     assert status_of(lambda: A.amoeba_merge_block_tables(plan, z, z, 2, 4, z, live.data_ptr() + 4, z)) == A.ERR_ALIGNMENT
     assert status_of(lambda: A.amoeba_merge_block_tables(plan, z, z, 2, 0, z, live, z)) == A.ERR_INVALID_ARG
+
+
+def test_merge_replayed_from_a_cuda_graph(oracle):
+    """The merge's two calls (a memset, the table kernel, the exchange kernel) recorded into a CUDA graph: one replay
+    gives the oracle's result, a second replay exchanges the live segments back where every instance holds the block."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    m, T, N, a, NB = GQA, 16, 2, 1, 11
+    lens, bt, pools = _instances(oracle, m, T, N, a, NB, [[100, 60], [150, 3]], seed=8)
+    exp_pools = [p.copy() for p in pools]
+    exp_bt, exp_live, exp_status = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, exp_pools)
+    dev = torch.device("cuda:0")
+    plan = A.amoeba_plan_create(A.make_layout(m, a, NB, block_tokens=T), A.make_layout(m, N * a, NB * N, block_tokens=T))
+    d_bt, d_lens = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+    d_new = torch.full(bt.shape, -9, dtype=torch.int32, device=dev)
+    d_live = torch.zeros(A.amoeba_merge_live_bytes(plan), dtype=torch.uint8, device=dev)
+    d_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    scratch = [torch.zeros(p.size * 2, dtype=torch.uint8, device=dev) for p in pools]
+    A.amoeba_merge_block_tables(plan, d_bt, d_lens, bt.shape[1], bt.shape[2], d_new, d_live, d_status)  # one-time set-up
+    A.amoeba_merge_kv_inplace(plan, scratch, d_live, 0, m["L"], d_status)
+    torch.cuda.synchronize()
+    d_pools = [torch.from_numpy(p.view(np.uint8).copy()).to(dev) for p in pools]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        A.amoeba_merge_block_tables(plan, d_bt, d_lens, bt.shape[1], bt.shape[2], d_new, d_live, d_status)
+        A.amoeba_merge_kv_inplace(plan, d_pools, d_live, 0, m["L"], d_status)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(d_status.item()) == exp_status == 0
+    assert np.array_equal(d_new.cpu().numpy(), exp_bt)
+    for g, e in zip(d_pools, exp_pools):
+        assert np.array_equal(g.cpu().numpy().view(np.uint16), e)

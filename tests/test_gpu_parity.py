@@ -279,3 +279,32 @@ def test_padded_weight_partitions(path, a, b, sp, dp):
 def test_padded_unfused_buffers_and_kv_together(fq, fg):
     c = make_case(PADM, 2, 4, [40, 3], fused_qkv=fq, fused_gate_up=fg, seed=12, src_pad=(4, 4096), dst_pad=(4, 4096))
     check_case(c, run_case(c))
+
+
+# ---- stream capture: the data calls only enqueue work, so a transformation can be recorded once and replayed
+@pytest.mark.parametrize("so,do", [(HC, HC), (TF, TF), (TF, HC)])
+def test_step_replayed_from_a_cuda_graph(so, do):
+    import torch
+
+    c = make_case(GQA, 2, 4, [300, 17, 64, 5], seed=31, src_order=so, dst_order=do)
+    s = run_case(c)          # one plain run first: one-time set-up (function attributes, entry points) happens here
+    check_case(c, s)
+
+    def wipe():
+        for t in s.dst_pools + s._wbufs[c.a:]:
+            t.fill_(0xA5)
+        s.dst_bt.fill_(-2)
+        s.pairs.fill_(-3)
+        s.num_pairs.zero_()
+        s.free_count.zero_()
+
+    wipe()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        s.status.zero_()
+        s.step()
+    for _ in range(2):       # replay twice, wiping the outputs in between
+        graph.replay()
+        torch.cuda.synchronize()
+        check_case(c, s)
+        wipe()
