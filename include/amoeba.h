@@ -306,6 +306,18 @@ AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
                                      const amoeba_layer_weights* dst, int32_t layer_begin, int32_t layer_end,
                                      int32_t* d_status, void* cuda_stream);
 
+/*
+ * amoeba_plan_weight_alias  (Sec. 3.2, Improvement 1: with padded partitions a scale-up needs no weight copy at all)
+ *
+ * When both layouts are padded with the same weight_pad_parts, page size and fused flags and the destination TP is a
+ * multiple of the source TP, the buffer `tensor` of destination worker dst_rank is, byte for byte (pads included),
+ * the range [*src_offset, *src_offset + *bytes) of the same buffer of source worker *src_rank: the worker that keeps
+ * those pages can use them where they are and release the others, instead of calling amoeba_reshard_weights.
+ * Host arithmetic only.  Errors: INVALID_ARG; UNSUPPORTED when the layouts do not allow it (a copy is needed).
+ */
+AMOEBA_API amoeba_status amoeba_plan_weight_alias(const amoeba_plan* plan, int32_t dst_rank, int32_t tensor,
+                                       int32_t* src_rank, int64_t* src_offset, int64_t* bytes);
+
 /* Number of kernels the library has launched in this process (for launch accounting in benchmarks). */
 AMOEBA_API int64_t amoeba_launch_count(void);
 

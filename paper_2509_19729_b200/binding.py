@@ -113,6 +113,7 @@ def _load():
         "amoeba_merge_bytes": (I32, [VP, I64, P(I64)]),
         "amoeba_merge_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, VP, VP]),
         "amoeba_merge_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
+        "amoeba_plan_weight_alias": (I32, [VP, I32, I32, P(I32), P(I64), P(I64)]),
         "amoeba_launch_count": (I64, []),
         "amoeba_status_string": (C.c_char_p, [I32]),
     }
@@ -328,6 +329,18 @@ def amoeba_merge_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int,
 
 
 __all__ += ["amoeba_merge_live_bytes", "amoeba_merge_bytes", "amoeba_merge_block_tables", "amoeba_merge_kv_inplace"]
+
+
+def amoeba_plan_weight_alias(plan: Plan, dst_rank: int, tensor: int):
+    """(source worker, byte offset, bytes) of the source buffer range that already is the destination worker's
+    buffer; raises AmoebaError(ERR_UNSUPPORTED) when the layouts need a copy."""
+    r, off, n = C.c_int32(), C.c_int64(), C.c_int64()
+    _check(_load().amoeba_plan_weight_alias(plan.handle, dst_rank, tensor, C.byref(r), C.byref(off), C.byref(n)),
+           "amoeba_plan_weight_alias")
+    return r.value, off.value, n.value
+
+
+__all__.append("amoeba_plan_weight_alias")
 
 
 def amoeba_launch_count() -> int:

@@ -483,6 +483,24 @@ amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_live_blocks,
     return AMOEBA_OK;
 }
 
+amoeba_status amoeba_plan_weight_alias(const amoeba_plan* plan, int32_t dst_rank, int32_t tensor, int32_t* src_rank,
+                                       int64_t* src_offset, int64_t* bytes) {
+    if (!plan || !src_rank || !src_offset || !bytes || tensor < 0 || tensor >= kNumTensors || dst_rank < 0 ||
+        dst_rank >= plan->dst.tp)
+        return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_layout &s = plan->src, &d = plan->dst;
+    if (s.weight_pad_parts <= 0 || s.weight_pad_parts != d.weight_pad_parts || s.fused_qkv != d.fused_qkv ||
+        s.fused_gate_up != d.fused_gate_up || d.tp % s.tp)
+        return AMOEBA_ERR_UNSUPPORTED;
+    const WeightForm fs = weight_form(s), fd = weight_form(d);
+    if (fs.page != fd.page) return AMOEBA_ERR_UNSUPPORTED;
+    const int first = dst_rank * fd.per_worker;  // first partition the destination worker holds
+    *src_rank = first / fs.per_worker;
+    *src_offset = (int64_t)(first % fs.per_worker) * fs.pitch[tensor];
+    *bytes = fd.block[tensor] ? (int64_t)fd.per_worker * fd.pitch[tensor] : 0;
+    return AMOEBA_OK;
+}
+
 int64_t amoeba_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* amoeba_status_string(amoeba_status s) {

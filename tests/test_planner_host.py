@@ -239,3 +239,33 @@ def test_padded_layout_validation():
         with pytest.raises(A.AmoebaError) as e:
             A.amoeba_plan_create(A.make_layout(m, 2, 4, **kw), A.make_layout(m, 2, 4))
         assert e.value.status == status, kw
+
+
+@pytest.mark.parametrize("fq,fg", [(True, True), (False, False)])
+@pytest.mark.parametrize("a,b,P", [(1, 4, 4), (2, 8, 8), (1, 2, 8), (4, 4, 8)])
+def test_padded_scale_up_is_an_alias_of_the_source_buffers(oracle, a, b, P, fq, fg):
+    """Sec. 3.2 Improvement 1: with padded partitions every destination shard already sits in a source buffer."""
+    m, page = PADM, 1024
+    g = np.random.default_rng(P)
+    W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in oracle.logical_shapes(m).items()}
+    src = oracle.weights_shard_padded(W, m, a, P, page // 2, fq, fg, fill=0)
+    dst = oracle.weights_shard_padded(W, m, b, P, page // 2, fq, fg, fill=0)
+    lay = lambda tp: A.make_layout(m, tp, 4, fused_qkv=fq, fused_gate_up=fg, weight_pad_parts=P, weight_page_bytes=page)
+    plan = A.amoeba_plan_create(lay(a), lay(b))
+    for j in range(b):
+        for t, n in enumerate(A.TENSOR_NAMES):
+            r, off, nbytes = A.amoeba_plan_weight_alias(plan, j, t)
+            if n not in dst[j]:
+                assert nbytes == 0
+                continue
+            assert nbytes == dst[j][n].size * 2 and off % page == 0
+            assert np.array_equal(src[r][n].view(np.uint8)[off:off + nbytes], dst[j][n].view(np.uint8))
+    for other in (A.make_layout(m, b, 4, fused_qkv=fq, fused_gate_up=fg),                                   # dense
+                  A.make_layout(m, b, 4, fused_qkv=fq, fused_gate_up=fg, weight_pad_parts=P, weight_page_bytes=512)):
+        with pytest.raises(A.AmoebaError) as e:
+            A.amoeba_plan_weight_alias(A.amoeba_plan_create(lay(a), other), 0, 0)
+        assert e.value.status == A.ERR_UNSUPPORTED
+    if a > 1:  # scale-down gathers partitions of several workers: a copy
+        with pytest.raises(A.AmoebaError) as e:
+            A.amoeba_plan_weight_alias(A.amoeba_plan_create(lay(b), lay(1)), 0, 0)
+        assert e.value.status == A.ERR_UNSUPPORTED or b == 1
