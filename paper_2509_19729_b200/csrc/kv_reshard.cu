@@ -52,25 +52,35 @@ __device__ __forceinline__ int64_t pool_offset(bool token_major, int32_t nb, int
                        : ((((int64_t)blk * heads + hl) * 2 + c) * T) * vec;
 }
 
+// Least significant digit of `rem` in a mixed-radix number; `rem` keeps the higher digits.
+__device__ __forceinline__ int32_t take_digit(uint32_t& rem, int32_t radix) {
+    if (radix == 1) return 0;
+    const uint32_t q = rem / (uint32_t)radix;
+    const int32_t d = (int32_t)(rem - q * (uint32_t)radix);
+    rem = q;
+    return d;
+}
+
 struct KvItems {
     const KvParams& p;
     int32_t n_pairs;
-    __device__ __forceinline__ int64_t items_per_pair() const {
-        return (int64_t)p.planes * p.head_units * p.row_groups * p.col_chunks;
+    __device__ __forceinline__ int32_t items_per_pair() const {
+        return p.planes * p.head_units * p.row_groups * p.col_chunks;
     }
     __device__ __forceinline__ int64_t count() const { return (int64_t)n_pairs * p.n_layers * items_per_pair(); }
     // n_rows == 0 marks a skipped pair.
     __device__ __forceinline__ Item operator()(int64_t w) const {
-        const int32_t col = (int32_t)(w % p.col_chunks);
-        int64_t t = w / p.col_chunks;
-        const int32_t rg = (int32_t)(t % p.row_groups);
-        t /= p.row_groups;
-        const int32_t hu = (int32_t)(t % p.head_units);
-        t /= p.head_units;
-        const int32_t c = (int32_t)(t % p.planes);
-        t /= p.planes;
-        const int32_t pair = (int32_t)(t % n_pairs);
-        const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
+        // Two 64-bit divisions (by the items of one pair, by the pair count); everything inside a pair is 32-bit,
+        // and a digit whose radix is 1 costs nothing.
+        const int32_t ipp = items_per_pair();
+        const int64_t lp = w / ipp;
+        uint32_t rem = (uint32_t)(w - lp * ipp);
+        const int32_t col = take_digit(rem, p.col_chunks);
+        const int32_t rg = take_digit(rem, p.row_groups);
+        const int32_t hu = take_digit(rem, p.head_units);
+        const int32_t c = (int32_t)rem;  // < planes
+        const int32_t pair = (int32_t)(lp % n_pairs);
+        const int32_t layer = p.layer_begin + (int32_t)(lp / n_pairs);
         const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
         Item it;
         it.src_map = it.dst_map = nullptr;
@@ -107,18 +117,19 @@ struct KvBoxItems {
     const KvParams& p;
     const KvMaps& maps;
     int32_t n_pairs;
-    __device__ __forceinline__ int64_t count() const {
-        return (int64_t)n_pairs * p.n_layers * p.runs_per_block * p.box_sub_runs * p.box_tok_groups;
+    __device__ __forceinline__ int32_t items_per_pair() const {
+        return p.runs_per_block * p.box_sub_runs * p.box_tok_groups;
     }
+    __device__ __forceinline__ int64_t count() const { return (int64_t)n_pairs * p.n_layers * items_per_pair(); }
     __device__ __forceinline__ Item operator()(int64_t w) const {
-        const int32_t tg = (int32_t)(w % p.box_tok_groups);
-        int64_t t = w / p.box_tok_groups;
-        const int32_t sub = (int32_t)(t % p.box_sub_runs);
-        t /= p.box_sub_runs;
-        const int32_t run = (int32_t)(t % p.runs_per_block);
-        t /= p.runs_per_block;
-        const int32_t pair = (int32_t)(t % n_pairs);
-        const int32_t layer = p.layer_begin + (int32_t)(t / n_pairs);
+        const int32_t ipp = items_per_pair();
+        const int64_t lp = w / ipp;
+        uint32_t rem = (uint32_t)(w - lp * ipp);
+        const int32_t tg = take_digit(rem, p.box_tok_groups);
+        const int32_t sub = take_digit(rem, p.box_sub_runs);
+        const int32_t run = (int32_t)rem;  // < runs_per_block
+        const int32_t pair = (int32_t)(lp % n_pairs);
+        const int32_t layer = p.layer_begin + (int32_t)(lp / n_pairs);
         const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
         Item it;
         it.src_map = it.dst_map = nullptr;
@@ -250,14 +261,14 @@ struct MergeItems {
         return (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
     }
     __device__ __forceinline__ Item operator()(int64_t w) const {
-        const int32_t chunk = (int32_t)(w % p.chunks_per_seg);
-        int64_t t = w / p.chunks_per_seg;
-        int32_t pr = (int32_t)(t % p.n_pairs);
-        t /= p.n_pairs;
-        const int32_t r = (int32_t)(t % p.a);
-        t /= p.a;
-        const int32_t blk = (int32_t)(t % p.nb);
-        const int32_t layer = p.layer_begin + (int32_t)(t / p.nb);
+        const int32_t ipb = p.a * p.n_pairs * p.chunks_per_seg;  // items of one (layer, block)
+        const int64_t lb = w / ipb;
+        uint32_t rem = (uint32_t)(w - lb * ipb);
+        const int32_t chunk = take_digit(rem, p.chunks_per_seg);
+        int32_t pr = take_digit(rem, p.n_pairs);
+        const int32_t r = (int32_t)rem;  // < a
+        const int32_t blk = (int32_t)(lb % p.nb);
+        const int32_t layer = p.layer_begin + (int32_t)(lb / p.nb);
         int32_t i = 0;  // pr-th pair (i, k) with i < k, in lexicographic order
         while (pr >= p.n_inst - 1 - i) {
             pr -= p.n_inst - 1 - i;
