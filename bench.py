@@ -591,10 +591,10 @@ def main():
         "phases_gbs": {"reshard_kv": kv_gbs, "reshard_weights": w_gbs},
         "pct_of_nominal_8TBs": {"reshard_kv": 100 * kv_gbs / NOMINAL_HBM_GBS,
                                 "reshard_weights": 100 * w_gbs / NOMINAL_HBM_GBS if w_gbs else None},
-        "roofline": {"kernel": "kv_reshard", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": "kv_reshard_pair" if not args.copy_path else "kv_reshard", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
                      "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": NCU_KV_TRAFFIC_RATIO * kv_bytes if traffic_known else None},
-        "roofline_weights": None if not w_gbs else {"kernel": "w_reshard", "bound": "hbm", "achieved": w_gbs,
+        "roofline_weights": None if not w_gbs else {"kernel": "w_reshard_pair" if not args.copy_path else "w_reshard", "bound": "hbm", "achieved": w_gbs,
                                                     "peak": peak, "unit": "GB/s", "frac": w_gbs / peak},
         "gpu_launches": int(launches), "clocks": clocks,
     }

@@ -246,6 +246,29 @@ def assign_blocks(seq_lens, T, src_bt, NB_src, NB_dst, free_list=None, free_mask
 
 
 
+def kv_split_inplace(m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride=None):
+    """The way back from ``kv_merge_inplace``: one instance of TP=N*a becomes N instances of TP=a in place.
+
+    seq_lens [N][S], bt [N][S][maxb]: the merged instance's table rows of the requests that go to instance i (ids over
+    NB*N blocks, each = i mod N); pools[i*a + r] = merged worker r*N+i, rewritten into worker r of instance i.
+    Returns (old_bt [N][S][maxb] with q -> q // N, live [N][NB], status)."""
+    sl = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    b = np.ascontiguousarray(bt, dtype=np.int32)
+    assert sl.ndim == 2 and b.ndim == 3 and sl.shape[0] == N and b.shape[:2] == sl.shape and len(pools) == N * a
+    S, maxb = b.shape[1], b.shape[2]
+    stride = pool_elems_per_layer(m, T, a, NB) if layer_stride is None else layer_stride
+    old_bt = np.empty_like(b)
+    live = np.empty((N, NB), dtype=np.uint8)
+    st = C.c_int32(status)
+    mm = _model(m)
+    lib().oracle_kv_split_inplace(C.byref(mm), T, N, a, NB, C.c_int64(stride), S,
+                                  sl.ctypes.data_as(C.POINTER(C.c_int32)), maxb,
+                                  b.ctypes.data_as(C.POINTER(C.c_int32)), _ptr_array(pools),
+                                  old_bt.ctypes.data_as(C.POINTER(C.c_int32)),
+                                  live.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(st))
+    return old_bt, live, st.value
+
+
 def kv_merge_inplace(m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride=None):
     """In-place merge of N instances of TP=a into one of TP=N*a (Sec. 3.1, Improvement 1).
 

@@ -497,3 +497,76 @@ void oracle_weights_padded_walk(const oracle_model* m, int TP, int r, int P, int
         padded_cols(lg->down, hid, I, P, p, sh->down + j * pitch_down, dir);
     }
 }
+
+
+/*
+ * The way back (Sec. 3.3, scale-down: "KV first", each new instance must hold all headers of its own requests),
+ * in place: one instance of TP = N*a becomes N instances of TP = a on the same workers' memory.  It undoes
+ * oracle_kv_merge_inplace and uses the same reading: merged worker r*N+i becomes worker r of instance i, and a block
+ * whose merged id is q = p*N+i belongs to instance i and becomes its block p (the N new-size slots p*N .. p*N+N-1 of
+ * that instance's pools).  The scheduler decides which request goes to which instance; a request may go to instance
+ * i only while its blocks have ids = i (mod N) - other blocks are first renumbered by an ordinary block-table
+ * rewrite with a free list of such ids.
+ *
+ * in : seq_lens[N][S], bt[N][S][maxb]: row block i = the merged instance's table rows of the requests that go to
+ *      instance i (ids over the merged pools of NB*N blocks); pools[i*a + r] = merged worker r*N+i,
+ *      [L][NB*N][Hkv/(N*a)][K/V][T][D].
+ * out: pools[i*a + r] = worker r of instance i, [L][NB][Hkv/a][K/V][T][D]; old_bt[N][S][maxb] (entry q -> q/N);
+ *      live[N][NB] = 1 for every block of instance i that now holds a request's data.
+ * Errors as in the merge; in addition an id q with q mod N != i is BAD_BLOCK_ID (entry -1, block not moved).
+ */
+void oracle_kv_split_inplace(const oracle_model* m, int T, int N, int a, int NB, int64_t layer_stride, int S,
+                             const int32_t* seq_lens, int maxb, const int32_t* bt, uint16_t* const* pools,
+                             int32_t* old_bt, uint8_t* live, int32_t* status) {
+    const int TPn = N * a, Ha = m->Hkv / a, Hn = m->Hkv / TPn;
+    const int64_t pool_elems = (int64_t)m->L * layer_stride;
+    for (int64_t k = 0; k < (int64_t)N * S * maxb; ++k) old_bt[k] = -1;
+    for (int64_t k = 0; k < (int64_t)N * NB; ++k) live[k] = 0;
+    for (int64_t k = 0; k < (int64_t)N * S; ++k)
+        if (seq_lens[k] < 0 || blocks_of(seq_lens[k], T) > maxb) {
+            if (*status == 0) *status = ORACLE_INVALID_ARG;
+            return;
+        }
+    uint16_t** old = (uint16_t**)malloc(sizeof(uint16_t*) * (size_t)(N * a));
+    for (int w = 0; w < N * a; ++w) {
+        old[w] = (uint16_t*)malloc((size_t)pool_elems * sizeof(uint16_t));
+        memcpy(old[w], pools[w], (size_t)pool_elems * sizeof(uint16_t));
+    }
+    for (int i = 0; i < N; ++i)
+        for (int s = 0; s < S; ++s)
+            for (int64_t j = 0; j < blocks_of(seq_lens[i * S + s], T); ++j) {
+                const int64_t e = ((int64_t)i * S + s) * maxb + j;
+                const int64_t q = bt[e];
+                if (q < 0 || q >= (int64_t)NB * N || q % N != i) {
+                    if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+                    continue;
+                }
+                const int64_t p = q / N;
+                old_bt[e] = (int32_t)p;
+                if (live[(int64_t)i * NB + p]) {
+                    if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+                    continue;
+                }
+                live[(int64_t)i * NB + p] = 1;
+                for (int l = 0; l < m->L; ++l)
+                    for (int header = 1; header <= m->Hkv; ++header) {
+                        /* before: merged worker wn, which lives in the memory of worker (wn-1)/N of instance (wn-1)%N */
+                        const int wn = oracle_worker_of_header(m->Hkv, TPn, header);
+                        /* after: worker wa of instance i */
+                        const int wa = oracle_worker_of_header(m->Hkv, a, header);
+                        int fa, fn, last;
+                        oracle_header_range(m->Hkv, TPn, wn, &fn, &last);
+                        oracle_header_range(m->Hkv, a, wa, &fa, &last);
+                        const uint16_t* sp = old[((wn - 1) % N) * a + (wn - 1) / N] + (int64_t)l * layer_stride;
+                        uint16_t* dp = pools[i * a + (wa - 1)] + (int64_t)l * layer_stride;
+                        for (int c = 0; c < 2; ++c)
+                            for (int tok = 0; tok < T; ++tok)
+                                for (int d = 0; d < m->D; ++d)
+                                    dp[pool_offset(ORACLE_HEADER_CENTRIC, NB, Ha, T, m->D, p, header - fa, c, tok, d)] =
+                                        sp[pool_offset(ORACLE_HEADER_CENTRIC, (int64_t)NB * N, Hn, T, m->D, q,
+                                                       header - fn, c, tok, d)];
+                    }
+            }
+    for (int w = 0; w < N * a; ++w) free(old[w]);
+    free(old);
+}

@@ -195,3 +195,88 @@ def test_merge_decode_attention_unchanged(oracle):
     assert st == 0
     back = oracle.kv_reconstruct(pools, m, T, N, NB * N, lens[1], new_bt[1])
     assert np.array_equal(attend(back, lens[1], q).view(np.uint32), ref.view(np.uint32))
+
+
+# ---------------- the way back: one instance of TP = N*a -> N instances of TP = a, in place ----------------
+def _merged_instance(oracle, m, T, N, a, NB, lens_per_group, seed=0):
+    """One instance at TP = N*a whose requests are already grouped by the instance they will go to: group i's blocks
+    have ids = i (mod N).  Returns lens [N][S], bt [N][S][maxb], the logical KV of each group, and the pools in the
+    order pools[i*a + r] = merged worker r*N+i."""
+    g = np.random.default_rng(seed)
+    S = max(len(l) for l in lens_per_group)
+    lens = np.zeros((N, S), np.int32)
+    for i, l in enumerate(lens_per_group):
+        lens[i, :len(l)] = l
+    nblk = (lens + T - 1) // T
+    maxb = max(int(nblk.max()), 1)
+    bt = np.full((N, S, maxb), -1, np.int32)
+    merged = [np.full(m["L"] * oracle.pool_elems_per_layer(m, T, N * a, NB * N), 0x2000 + w, np.uint16)
+              for w in range(N * a)]
+    KVs = []
+    for i in range(N):
+        ids = g.permutation(NB) * N + i
+        k = 0
+        for s in range(S):
+            bt[i, s, :nblk[i, s]] = ids[k:k + nblk[i, s]]
+            k += int(nblk[i, s])
+        G = int(nblk[i].sum()) * T
+        KV = g.integers(0, 65536, size=(m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+        KVs.append(KV)
+        part = oracle.kv_shard(KV, m, T, N * a, NB * N, lens[i], bt[i], fill=0)
+        where = oracle.kv_shard(np.full_like(KV, 1), m, T, N * a, NB * N, lens[i], bt[i], fill=0)  # 1 = written word
+        for w in range(N * a):
+            merged[w][where[w] != 0] = part[w][where[w] != 0]
+    pools = [None] * (N * a)
+    for w in range(N * a):
+        pools[(w % N) * a + (w // N)] = merged[w]
+    return lens, bt, KVs, pools
+
+
+@pytest.mark.parametrize("N,a", [(4, 1), (2, 1), (2, 2)])
+def test_split_gives_every_instance_all_headers_of_its_requests(oracle, N, a):
+    m, T, NB = MHA8, 4, 7
+    lens, bt, KVs, pools = _merged_instance(oracle, m, T, N, a, NB, [[5, 9], [16], [3, 3, 3], [7]][:N], seed=N + a)
+    old_bt, live, st = oracle.kv_split_inplace(m, T, N, a, NB, lens, bt, pools)
+    assert st == 0
+    for i in range(N):
+        assert np.array_equal(old_bt[i][bt[i] >= 0], bt[i][bt[i] >= 0] // N)
+        back = oracle.kv_reconstruct(pools[i * a:(i + 1) * a], m, T, a, NB, lens[i], old_bt[i])
+        assert np.array_equal(back, KVs[i])
+        assert np.array_equal(np.flatnonzero(live[i]), np.sort(old_bt[i][old_bt[i] >= 0]))
+
+
+@pytest.mark.parametrize("N,a", [(4, 1), (2, 2)])
+def test_split_undoes_merge_and_merge_undoes_split(oracle, N, a):
+    m, T, NB = MHA8, 4, 9
+    lens, bt, KVs, pools = _instances(oracle, m, T, N, a, NB, [[5, 9, 1], [16], [3, 3, 3], [0, 7]][:N], seed=21)
+    first = [p.copy() for p in pools]
+    new_bt, live_m, st = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, pools)
+    assert st == 0
+    old_bt, live_s, st = oracle.kv_split_inplace(m, T, N, a, NB, lens, new_bt, pools)
+    assert st == 0 and np.array_equal(old_bt, bt) and np.array_equal(live_s, live_m)
+    per_block = (m["Hkv"] // a) * 2 * T * m["D"]
+    for i in range(N):
+        for r in range(a):
+            now = pools[i * a + r].reshape(m["L"], NB, per_block)
+            was = first[i * a + r].reshape(m["L"], NB, per_block)
+            assert np.array_equal(now[:, live_m[i] != 0], was[:, live_m[i] != 0])  # every live block is back, whole
+
+
+def test_split_rejects_blocks_of_the_wrong_residue(oracle):
+    m, T, N, a, NB = MHA8, 4, 2, 1, 5
+    lens, bt, KVs, pools = _merged_instance(oracle, m, T, N, a, NB, [[8], [4, 4]], seed=3)
+    before = [p.copy() for p in pools]
+    bad = bt.copy()
+    good = int(bad[0, 0, 1])
+    bad[0, 0, 0] = int(bad[0, 0, 0]) + 1           # an id = 1 (mod 2) in the rows of instance 0
+    bad[1, 1, 0] = NB * N                          # out of range
+    old_bt, live, st = oracle.kv_split_inplace(m, T, N, a, NB, lens, bad, pools)
+    assert st == oracle.BAD_BLOCK_ID
+    assert old_bt[0, 0, 0] == -1 and old_bt[1, 1, 0] == -1 and old_bt[0, 0, 1] == good // N
+    assert live[0].sum() == 1 and live[1].sum() == 1
+    neg = lens.copy()
+    neg[0, 0] = -1
+    pools2 = [p.copy() for p in before]
+    old_bt, live, st = oracle.kv_split_inplace(m, T, N, a, NB, neg, bt, pools2)
+    assert st == oracle.INVALID_ARG and np.all(old_bt == -1) and not live.any()
+    assert all(np.array_equal(p, q) for p, q in zip(pools2, before))
