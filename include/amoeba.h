@@ -288,6 +288,28 @@ AMOEBA_API amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, cons
                                         uint8_t* d_live, int32_t* d_status, void* cuda_stream);
 AMOEBA_API amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
                                       int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
+/*
+ * amoeba_split_block_tables  (the way back: Sec. 3.3's scale-down, where the KV cache is transformed first so that
+ * every new instance holds all headers of its own requests; in place, with the same plan as the merge)
+ *
+ * One instance of TP = N*a becomes N instances of TP = a on the same memory.  d_merged_bt int32
+ * [N][num_seqs][max_blocks_per_seq], d_seq_lens int32 [N][num_seqs]: row block i = the merged instance's table rows
+ * of the requests that go to instance i.  A block with merged id q = p*N+i can only go to instance i and becomes its
+ * block p; blocks with other ids are first renumbered by the caller with amoeba_rewrite_block_tables /
+ * amoeba_reshard_kv inside the merged pools, using a free list of ids = i (mod N).  Writes d_inst_bt (q -> q/N, -1
+ * past each sequence's blocks) and d_live as amoeba_merge_block_tables does; an id outside [0, NB*N) or with q mod N
+ * != i is BAD_BLOCK_ID (entry -1, block not moved).
+ *
+ * amoeba_split_kv_inplace: same arguments as amoeba_merge_kv_inplace, with the live marks of
+ * amoeba_split_block_tables; pools[i*a + r] is merged worker r*N+i before and worker r of instance i after.  Where
+ * both blocks of a pair are live the two segments are exchanged exactly as in the merge; where one is live the
+ * direction is the opposite one: the live block of instance i fetches its headers from the other worker.
+ */
+AMOEBA_API amoeba_status amoeba_split_block_tables(const amoeba_plan* plan, const int32_t* d_merged_bt, const int32_t* d_seq_lens,
+                                        int32_t num_seqs, int32_t max_blocks_per_seq, int32_t* d_inst_bt,
+                                        uint8_t* d_live, int32_t* d_status, void* cuda_stream);
+AMOEBA_API amoeba_status amoeba_split_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                      int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
 /* Bytes read + written by amoeba_merge_kv_inplace when n_live_blocks old blocks (summed over the instances) are
  * live, over all layers: 2 * (N-1)/N of their size. */
 AMOEBA_API amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_live_blocks, int64_t* kv_bytes_rw);

@@ -112,7 +112,9 @@ def _load():
         "amoeba_merge_live_bytes": (I32, [VP, P(I64)]),
         "amoeba_merge_bytes": (I32, [VP, I64, P(I64)]),
         "amoeba_merge_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, VP, VP]),
+        "amoeba_split_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, VP, VP]),
         "amoeba_merge_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
+        "amoeba_split_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
         "amoeba_plan_weight_alias": (I32, [VP, I32, I32, P(I32), P(I64), P(I64)]),
         "amoeba_launch_count": (I64, []),
         "amoeba_status_string": (C.c_char_p, [I32]),
@@ -318,6 +320,16 @@ def amoeba_merge_block_tables(plan: Plan, src_bt, seq_lens, num_seqs: int, max_b
            "amoeba_merge_block_tables")
 
 
+def amoeba_split_block_tables(plan: Plan, merged_bt, seq_lens, num_seqs: int, max_blocks_per_seq: int, inst_bt, live,
+                              status, stream=None) -> None:
+    _check(_load().amoeba_split_block_tables(plan.handle, _ptr(merged_bt), _ptr(seq_lens), num_seqs,
+                                             max_blocks_per_seq, _ptr(inst_bt), _ptr(live), _ptr(status),
+                                             _stream(stream)), "amoeba_split_block_tables")
+
+
+__all__.append("amoeba_split_block_tables")
+
+
 def amoeba_merge_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int, layer_end: int, status,
                             stream=None) -> None:
     """pools: N*a tensors or addresses, pools[i*a + r] = worker r of instance i."""
@@ -328,7 +340,17 @@ def amoeba_merge_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int,
                                            _stream(stream)), "amoeba_merge_kv_inplace")
 
 
-__all__ += ["amoeba_merge_live_bytes", "amoeba_merge_bytes", "amoeba_merge_block_tables", "amoeba_merge_kv_inplace"]
+def amoeba_split_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int, layer_end: int, status,
+                            stream=None) -> None:
+    """pools: N*a tensors or addresses, pools[i*a + r] = merged worker r*N+i, afterwards worker r of instance i."""
+    if len(pools) != plan.dst.tp:
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_split_kv_inplace (need N*a pools)")
+    pp = (C.c_void_p * len(pools))(*[_ptr(x) for x in pools])
+    _check(_load().amoeba_split_kv_inplace(plan.handle, pp, _ptr(live), layer_begin, layer_end, _ptr(status),
+                                           _stream(stream)), "amoeba_split_kv_inplace")
+
+
+__all__ += ["amoeba_split_kv_inplace", "amoeba_merge_live_bytes", "amoeba_merge_bytes", "amoeba_merge_block_tables", "amoeba_merge_kv_inplace"]
 
 
 def amoeba_plan_weight_alias(plan: Plan, dst_rank: int, tensor: int):

@@ -219,6 +219,9 @@ extern "C" amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
 // (a few KB), the live bytes are zeroed by a memset that precedes the launch on the stream.
 namespace amoeba {
 
+// split == false: instance tables -> merged table (p -> p*N+i).  split == true: the way back, merged table rows of
+// the requests that go to instance i -> that instance's table (q -> q/N; q must be = i mod N).
+template <bool split>
 __global__ void __launch_bounds__(256) merge_tables(const int32_t* __restrict__ src_bt,
                                                     const int32_t* __restrict__ seq_lens, int32_t n_inst,
                                                     int32_t num_seqs, int32_t block_tokens,
@@ -246,9 +249,12 @@ __global__ void __launch_bounds__(256) merge_tables(const int32_t* __restrict__ 
         for (int32_t i = col0 + lane; i < min(col0 + kSegment, max_blocks_per_seq); i += 32) {
             int32_t out = -1;
             if (i < nblk) {
-                const int32_t p = src_bt[row * max_blocks_per_seq + i];
-                if (p >= 0 && p < nb) {
-                    out = p * n_inst + inst;
+                const int32_t id = src_bt[row * max_blocks_per_seq + i];
+                const bool ok = split ? (id >= 0 && id < (int64_t)nb * n_inst && id % n_inst == inst)
+                                      : (id >= 0 && id < nb);
+                if (ok) {
+                    const int32_t p = split ? id / n_inst : id;  // block of the instance's own pool
+                    out = split ? p : p * n_inst + inst;
                     const int64_t idx = (int64_t)inst * nb + p;  // byte of the live array
                     const uint32_t bit = 1u << (8 * (idx & 3));
                     if (atomicOr(live_words + (idx >> 2), bit) & bit) bad = true;  // named twice by this instance
@@ -264,10 +270,9 @@ __global__ void __launch_bounds__(256) merge_tables(const int32_t* __restrict__ 
 
 }  // namespace amoeba
 
-extern "C" amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
-                                                   const int32_t* d_seq_lens, int32_t num_seqs,
-                                                   int32_t max_blocks_per_seq, int32_t* d_dst_bt, uint8_t* d_live,
-                                                   int32_t* d_status, void* cuda_stream) {
+static amoeba_status merge_or_split_tables(bool split, const amoeba_plan* plan, const int32_t* d_src_bt,
+                                           const int32_t* d_seq_lens, int32_t num_seqs, int32_t max_blocks_per_seq,
+                                           int32_t* d_dst_bt, uint8_t* d_live, int32_t* d_status, void* cuda_stream) {
     if (!plan || num_seqs < 0 || max_blocks_per_seq <= 0 || !d_live || !d_status) return AMOEBA_ERR_INVALID_ARG;
     if (num_seqs > 0 && (!d_src_bt || !d_seq_lens || !d_dst_bt)) return AMOEBA_ERR_INVALID_ARG;
     const int n = merge_instances(plan);
@@ -283,12 +288,28 @@ extern "C" amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, cons
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
     const int64_t units = (int64_t)n * num_seqs * ((max_blocks_per_seq + kSegment - 1) / kSegment);
     const int grid = (int)std::min<int64_t>((units + 7) / 8, (int64_t)dev.sms * 4);
-    merge_tables<<<grid, 256, 0, stream>>>(d_src_bt, d_seq_lens, n, num_seqs, plan->src.block_tokens,
-                                           max_blocks_per_seq, plan->src.num_blocks, d_dst_bt,
-                                           reinterpret_cast<uint32_t*>(d_live), d_status);
+    auto kernel = split ? merge_tables<true> : merge_tables<false>;
+    kernel<<<grid, 256, 0, stream>>>(d_src_bt, d_seq_lens, n, num_seqs, plan->src.block_tokens, max_blocks_per_seq,
+                                     plan->src.num_blocks, d_dst_bt, reinterpret_cast<uint32_t*>(d_live), d_status);
     if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();
     return AMOEBA_OK;
+}
+
+extern "C" amoeba_status amoeba_merge_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
+                                                   const int32_t* d_seq_lens, int32_t num_seqs,
+                                                   int32_t max_blocks_per_seq, int32_t* d_dst_bt, uint8_t* d_live,
+                                                   int32_t* d_status, void* cuda_stream) {
+    return merge_or_split_tables(false, plan, d_src_bt, d_seq_lens, num_seqs, max_blocks_per_seq, d_dst_bt, d_live,
+                                 d_status, cuda_stream);
+}
+
+extern "C" amoeba_status amoeba_split_block_tables(const amoeba_plan* plan, const int32_t* d_merged_bt,
+                                                   const int32_t* d_seq_lens, int32_t num_seqs,
+                                                   int32_t max_blocks_per_seq, int32_t* d_inst_bt, uint8_t* d_live,
+                                                   int32_t* d_status, void* cuda_stream) {
+    return merge_or_split_tables(true, plan, d_merged_bt, d_seq_lens, num_seqs, max_blocks_per_seq, d_inst_bt, d_live,
+                                 d_status, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------------------------------------

@@ -253,6 +253,7 @@ struct MergeParams {
     const uint8_t* live;  // [N][nb]
     int64_t layer_stride, block_bytes, seg_bytes, chunk_bytes;
     int32_t n_inst, a, nb, layer_begin, n_layers, chunks_per_seg, n_pairs;
+    int32_t split;  // 0: merge (a live block sends its segments away), 1: the way back (a live block gathers them)
 };
 
 struct MergeItems {
@@ -294,9 +295,11 @@ struct MergeItems {
             it.dst = B;
             it.dst_pitch = A - B;
         } else {
+            // merge: the live block's segment leaves for the other worker; split: the live block fetches its segment
+            const bool a_to_b = (live_i != 0) != (p.split != 0);
             it.n_rows = 1;
-            it.src = live_i ? A : B;
-            it.dst = live_i ? B : A;
+            it.src = a_to_b ? A : B;
+            it.dst = a_to_b ? B : A;
         }
         return it;
     }
@@ -481,9 +484,8 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     return AMOEBA_OK;
 }
 
-extern "C" amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
-                                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status,
-                                                 void* cuda_stream) {
+static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                       int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream) {
     if (!plan || !pools || !d_live || !d_status) return AMOEBA_ERR_INVALID_ARG;
     const amoeba_model& m = plan->src.model;
     if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
@@ -519,6 +521,7 @@ extern "C" amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* 
     p.layer_begin = layer_begin;
     p.n_layers = layer_end - layer_begin;
     p.n_pairs = n * (n - 1) / 2;
+    p.split = split ? 1 : 0;
 
     DeviceInfo dev;
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
@@ -536,4 +539,16 @@ extern "C" amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* 
     if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();
     return AMOEBA_OK;
+}
+
+extern "C" amoeba_status amoeba_merge_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status,
+                                                 void* cuda_stream) {
+    return merge_or_split_kv(false, plan, pools, d_live, layer_begin, layer_end, d_status, cuda_stream);
+}
+
+extern "C" amoeba_status amoeba_split_kv_inplace(const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
+                                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status,
+                                                 void* cuda_stream) {
+    return merge_or_split_kv(true, plan, pools, d_live, layer_begin, layer_end, d_status, cuda_stream);
 }

@@ -205,3 +205,79 @@ def test_merge_replayed_from_a_cuda_graph(oracle):
     assert np.array_equal(d_new.cpu().numpy(), exp_bt)
     for g, e in zip(d_pools, exp_pools):
         assert np.array_equal(g.cpu().numpy().view(np.uint16), e)
+
+
+# ---- the way back: one instance of TP = N*a -> N instances of TP = a, in place
+def _run_split(m, T, N, a, NB, lens, bt, pools):
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    dev = torch.device("cuda:0")
+    plan = A.amoeba_plan_create(A.make_layout(m, a, NB, block_tokens=T), A.make_layout(m, N * a, NB * N, block_tokens=T))
+    d_pools = [torch.from_numpy(p.view(np.uint8).copy()).to(dev) for p in pools]
+    d_bt, d_lens = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+    d_old = torch.full(bt.shape, -9, dtype=torch.int32, device=dev)
+    d_live = torch.full((A.amoeba_merge_live_bytes(plan),), 7, dtype=torch.uint8, device=dev)
+    d_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    A.amoeba_split_block_tables(plan, d_bt, d_lens, bt.shape[1], bt.shape[2], d_old, d_live, d_status)
+    A.amoeba_split_kv_inplace(plan, d_pools, d_live, 0, m["L"], d_status)
+    torch.cuda.synchronize()
+    return ([p.cpu().numpy().view(np.uint16) for p in d_pools], d_old.cpu().numpy(),
+            d_live.cpu().numpy()[:N * NB].reshape(N, NB), int(d_status.item()))
+
+
+def _scribble_free_blocks(m, T, N, a, NB, merged_bt, pools, seed=99):
+    """Overwrite every merged-size block no table names (the merge leaves stale copies there, a running instance would
+    have reused them): a split that moved a segment the wrong way would now fetch garbage."""
+    g = np.random.default_rng(seed)
+    used = np.zeros(NB * N, bool)
+    used[merged_bt[merged_bt >= 0]] = True
+    per = (m["Hkv"] // (N * a)) * 2 * T * m["D"]
+    for p in pools:
+        v = p.reshape(m["L"], NB * N, per)
+        v[:, ~used] = g.integers(0, 65536, size=(m["L"], int((~used).sum()), per), dtype=np.uint16)
+
+
+@pytest.mark.parametrize("N,a", [(2, 1), (4, 1), (2, 2), (4, 2)])
+def test_split_matches_oracle(oracle, N, a):
+    """Start from the oracle's merged state (so block ids have the residue of their instance), split on the GPU."""
+    m, T, NB = MHA8, 4, 23
+    lens, bt, pools = _instances(oracle, m, T, N, a, NB, LENS[:N], seed=N * 8 + a)
+    merged_bt, _, st = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, pools)   # pools are now the merged instance
+    assert st == 0
+    _scribble_free_blocks(m, T, N, a, NB, merged_bt, pools)
+    exp_pools = [p.copy() for p in pools]
+    exp_bt, exp_live, exp_status = oracle.kv_split_inplace(m, T, N, a, NB, lens, merged_bt, exp_pools)
+    got_pools, got_bt, got_live, got_status = _run_split(m, T, N, a, NB, lens, merged_bt, pools)
+    assert got_status == exp_status == 0
+    assert np.array_equal(got_bt, exp_bt) and np.array_equal(got_bt, bt)
+    assert np.array_equal(got_live, exp_live)
+    for w, (g, e) in enumerate(zip(got_pools, exp_pools)):
+        assert np.array_equal(g, e), w
+
+
+def test_split_device_detected_errors(oracle):
+    m, T, N, a, NB = MHA8, 4, 2, 1, 9
+    lens, bt, pools = _instances(oracle, m, T, N, a, NB, [[8, 4, 20], [5, 9]], seed=2)
+    merged_bt, _, _ = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, pools)
+    _scribble_free_blocks(m, T, N, a, NB, merged_bt, pools)
+    bad = merged_bt.copy()
+    bad[0, 0, 0] += 1            # residue of the other instance
+    bad[1, 1, 0] = NB * N        # out of range
+    bad[0, 2, 1] = -1            # hole inside a sequence
+    exp_pools = [p.copy() for p in pools]
+    exp_bt, exp_live, exp_status = oracle.kv_split_inplace(m, T, N, a, NB, lens, bad, exp_pools)
+    got_pools, got_bt, got_live, got_status = _run_split(m, T, N, a, NB, lens, bad, pools)
+    assert got_status == exp_status == 5
+    assert np.array_equal(got_bt, exp_bt) and np.array_equal(got_live, exp_live)
+    for g, e in zip(got_pools, exp_pools):
+        assert np.array_equal(g, e)
+    neg = lens.copy()
+    neg[1, 0] = -2
+    exp_pools = [p.copy() for p in pools]
+    exp_bt, exp_live, exp_status = oracle.kv_split_inplace(m, T, N, a, NB, neg, merged_bt, exp_pools)
+    got_pools, got_bt, got_live, got_status = _run_split(m, T, N, a, NB, neg, merged_bt, pools)
+    assert got_status == exp_status == 1 and np.array_equal(got_bt, exp_bt) and not got_live.any()
+    for g, e in zip(got_pools, exp_pools):
+        assert np.array_equal(g, e)
