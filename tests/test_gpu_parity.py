@@ -308,3 +308,120 @@ def test_step_replayed_from_a_cuda_graph(so, do):
         torch.cuda.synchronize()
         check_case(c, s)
         wipe()
+
+
+# ---- out-of-place merge of N instances into one (distinct request sets, one shared destination free list)
+def test_out_of_place_merge_of_instances_by_composition():
+    """N instances of TP = a become one instance of TP = N*a in fresh pools: one table rewrite and one KV call per
+    instance, each taking the part of the shared free list the earlier instances left (the caller knows the block counts
+    from the sequence lengths).  Expected: the oracle's a -> N*a transformation of each instance into the same pools."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    m, T, N, a = GQA, 16, 3, 2
+    b = 4  # destination TP (the three instances need not fill a multiple of their own TP)
+    dev = torch.device("cuda:0")
+    g = np.random.default_rng(17)
+    lens_all = [[100, 17, 300], [64], [5, 5, 5, 200]]
+    NB_src, need = 40, sum(sum((l + T - 1) // T for l in ls) for ls in lens_all)
+    NB_dst = need + 9
+    free = g.permutation(NB_dst).astype(np.int32)
+    exp_pools = [np.full(m["L"] * O.pool_elems_per_layer(m, T, b, NB_dst), 0xA5A5, np.uint16) for _ in range(b)]
+    d_dst = [torch.full((p.size * 2,), 0xA5, dtype=torch.uint8, device=dev) for p in exp_pools]
+    d_free = torch.from_numpy(free).to(dev)
+    d_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    plan = A.amoeba_plan_create(A.make_layout(m, a, NB_src, T), A.make_layout(m, b, NB_dst, T))
+    consumed, keep = 0, []
+    for i, ls in enumerate(lens_all):
+        lens = np.array(ls, np.int32)
+        nblk = (lens + T - 1) // T
+        maxb = int(nblk.max())
+        bt = np.full((len(ls), maxb), -1, np.int32)
+        ids = g.permutation(NB_src)
+        k = 0
+        for s, n in enumerate(nblk):
+            bt[s, :n] = ids[k:k + n]
+            k += int(n)
+        KV = g.integers(0, 65536, size=(m["L"], int(nblk.sum()) * T, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+        src = O.kv_shard(KV, m, T, a, NB_src, lens, bt)
+        # expected: this instance's blocks take the next ids of the shared list
+        exp_bt, exp_pairs, n_pairs, left, st = O.assign_blocks(lens, T, bt, NB_src, NB_dst, free_list=free[consumed:])
+        assert st == 0
+        O.kv_transform(m, T, lens, a, NB_src, bt, src, b, NB_dst, exp_bt, exp_pools)
+        # device: the same with the free list advanced by what the earlier instances took
+        d_src = [torch.from_numpy(p.view(np.uint8)).to(dev) for p in src]
+        d_bt, d_lens = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+        d_new = torch.empty_like(d_bt)
+        d_pairs = torch.empty((n_pairs, 2), dtype=torch.int32, device=dev)
+        d_n, d_left = torch.zeros(1, dtype=torch.int32, device=dev), torch.zeros(1, dtype=torch.int32, device=dev)
+        ws_bytes = A.amoeba_rewrite_workspace_bytes(plan, len(ls), NB_dst - consumed)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        A.amoeba_rewrite_block_tables(plan, d_bt, d_lens, len(ls), maxb, d_free[consumed:], None, NB_dst - consumed,
+                                      d_new, d_pairs, n_pairs, d_n, d_left, d_status, ws, ws_bytes)
+        A.amoeba_reshard_kv(plan, d_src, d_dst, d_pairs, d_n, n_pairs, 0, m["L"], d_status)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_new.cpu().numpy(), exp_bt) and int(d_left.item()) == left
+        keep.append((d_src, d_bt, d_lens, d_new, d_pairs, ws))
+        consumed += n_pairs
+    assert int(d_status.item()) == 0
+    for r in range(b):
+        assert np.array_equal(d_dst[r].cpu().numpy().view(np.uint16), exp_pools[r]), r
+
+
+def test_writes_stay_inside_the_buffers():
+    """Every destination buffer sits between guard regions inside one allocation; after a whole transformation (KV in
+    both storage orders, weights) the guards still hold their pattern."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    m, T, a, b, NB_s, NB_d = GQA, 16, 2, 4, 12, 15
+    dev = torch.device("cuda:0")
+    GUARD = 4096
+    for order in (0, 1):
+        src_l = A.make_layout(m, a, NB_s, T, kv_order=order)
+        dst_l = A.make_layout(m, b, NB_d, T, kv_order=order)
+        plan = A.amoeba_plan_create(src_l, dst_l)
+        pool_bytes = A.amoeba_layout_kv_pool_bytes(dst_l)
+        w_sizes = [A.amoeba_layout_weight_bytes(dst_l, t) for t in range(7)]
+        per_rank = [pool_bytes] + [s for s in w_sizes if s] * m["L"]
+        total = sum(GUARD + (s + 255) // 256 * 256 for s in per_rank) * b + GUARD
+        arena = torch.full((total,), 0xC3, dtype=torch.uint8, device=dev)
+        off, dst_pools, dst_w, spans = GUARD, [], [], []
+        for r in range(b):
+            dst_pools.append(arena[off:off + pool_bytes])
+            spans.append((off, pool_bytes))
+            off += (pool_bytes + 255) // 256 * 256 + GUARD
+            layers = []
+            for l in range(m["L"]):
+                d = {}
+                for t, s in enumerate(w_sizes):
+                    if s:
+                        d[A.TENSOR_NAMES[t]] = arena[off:off + s]
+                        spans.append((off, s))
+                        off += (s + 255) // 256 * 256 + GUARD
+                layers.append(d)
+            dst_w.append(layers)
+        g = torch.Generator(device=dev).manual_seed(5)
+        src_pools = [torch.randint(0, 256, (A.amoeba_layout_kv_pool_bytes(src_l),), dtype=torch.uint8, device=dev,
+                                   generator=g) for _ in range(a)]
+        src_w = [[{A.TENSOR_NAMES[t]: torch.randint(0, 256, (A.amoeba_layout_weight_bytes(src_l, t),), dtype=torch.uint8,
+                                                    device=dev, generator=g)
+                   for t in range(7) if A.amoeba_layout_weight_bytes(src_l, t)} for _ in range(m["L"])] for _ in range(a)]
+        pairs = torch.tensor([[i, NB_d - 1 - i] for i in range(NB_s)], dtype=torch.int32, device=dev)
+        n = torch.tensor([NB_s], dtype=torch.int32, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        for path in PATHS:
+            A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, path)
+            A.amoeba_reshard_kv(plan, src_pools, dst_pools, pairs, n, NB_s, 0, m["L"], status)
+            A.amoeba_reshard_weights(plan, src_w, dst_w, 0, m["L"], status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        inside = torch.zeros(total, dtype=torch.bool, device=dev)
+        for o, s in spans:
+            inside[o:o + s] = True
+        assert bool((arena[~inside] == 0xC3).all())
+        assert not bool((arena[inside] == 0xC3).all())  # and the buffers themselves were written
