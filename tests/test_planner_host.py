@@ -269,3 +269,45 @@ def test_padded_scale_up_is_an_alias_of_the_source_buffers(oracle, a, b, P, fq, 
         with pytest.raises(A.AmoebaError) as e:
             A.amoeba_plan_weight_alias(A.amoeba_plan_create(lay(b), lay(1)), 0, 0)
         assert e.value.status == A.ERR_UNSUPPORTED or b == 1
+
+
+def test_random_layout_pairs_reproduce_oracle(oracle):
+    """Seeded random shapes, TP degrees, fused / unfused buffers and dense / padded forms on either side: the planner's
+    descriptors, applied as plain byte copies, give the oracle's destination buffers and write no byte twice."""
+    g = np.random.default_rng(20250919)
+    done = 0
+    while done < 40:
+        Hkv = int(g.choice([4, 8, 12, 16, 24]))
+        m = dict(L=1, hidden=int(g.choice([16, 24, 40])), Hq=Hkv * int(g.choice([1, 2])), Hkv=Hkv,
+                 D=int(g.choice([8, 16])), I=Hkv * int(g.choice([8, 24])))
+        divs = [d for d in (1, 2, 3, 4, 6, 8, 12) if Hkv % d == 0]
+        a, b = int(g.choice(divs)), int(g.choice(divs))
+        fq, fg = bool(g.integers(2)), bool(g.integers(2))
+
+        def pick_pad(tp):
+            if g.integers(3) == 0:
+                return None
+            P = int(g.choice([d for d in divs if d % tp == 0]))
+            return (P, int(g.choice([64, 256, 1024])))
+
+        sp, dp = pick_pad(a), pick_pad(b)
+        W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in oracle.logical_shapes(m).items()}
+        opad = lambda pad: (pad[0], pad[1] // 2) if pad else None
+        src = oracle.weights_shard_padded(W, m, a, *opad(sp), fq, fg) if sp else oracle.weights_shard(W, m, a, fq, fg)
+        exp = oracle.weights_transform_any(src, m, a, b, fq, fg, src_pad=opad(sp), dst_pad=opad(dp), fill=0xA5A5)
+        lay = lambda tp, pad: A.make_layout(m, tp, 4, fused_qkv=fq, fused_gate_up=fg,
+                                            weight_pad_parts=pad[0] if pad else 0, weight_page_bytes=pad[1] if pad else 0)
+        try:
+            plan = A.amoeba_plan_create(lay(a, sp), lay(b, dp))
+        except A.AmoebaError as e:  # more descriptors than one launch carries: refused, not mis-planned
+            assert e.status == A.ERR_UNSUPPORTED, (m, a, b, sp, dp)
+            continue
+        as_bytes = lambda sh: [[r[n].reshape(-1).view(np.uint8) if n in r else None for n in A.TENSOR_NAMES] for r in sh]
+        dst = [[np.full(e.size, 0xA5, np.uint8) if e is not None else None for e in r] for r in as_bytes(exp)]
+        counts = _apply_descs(plan, as_bytes(src), dst)
+        for r in range(b):
+            for t, n in enumerate(A.TENSOR_NAMES):
+                if n in exp[r]:
+                    assert np.array_equal(dst[r][t], exp[r][n].reshape(-1).view(np.uint8)), (m, a, b, sp, dp, fq, fg, r, n)
+                    assert counts[r][t].max() == 1
+        done += 1
