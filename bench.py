@@ -121,7 +121,7 @@ def barrier(world: int):
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(cfg_name: str, kv_layers=2, n_seqs=None, w_layers=4, threads=1):
+def oracle_sample(cfg_name: str, kv_layers=4, n_seqs=None, w_layers=4, threads=1):
     """A bounded sample of the workload for the CPU oracle: the first n_seqs sequences (None = all) over kv_layers
     layers of KV, and w_layers layers of weights; values are uniform 16-bit words (the movement does not depend on
     them).  Returns a closure that runs one oracle a->b pass and the bytes it moves."""

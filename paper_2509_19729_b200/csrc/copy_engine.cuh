@@ -3,8 +3,8 @@
 // A work item is a small 2-D copy: n_rows runs of row_bytes bytes, run i read at src + i*src_pitch and written at
 // dst + i*dst_pitch (n_rows == 1 is a plain contiguous chunk).  All addresses, pitches and row_bytes are
 // multiples of 16 bytes.  Three ways to move items:
-//   * cta_copy_item      every thread of the CTA moves 16-byte vectors, all loads of an unrolled batch issued
-//                        before the first store, streaming cache hints;
+//   * warp_copy_item     a warp moves an item with 16-byte vector loads / stores, all loads of an unrolled batch
+//                        issued before the first store, streaming cache hints;
 //   * warp_bulk_ring     each warp drives its own ring of shared-memory stages with the bulk-copy engine (TMA, 1-D
 //                        cp.async.bulk, no multicast): global -> shared completes on an mbarrier, shared -> global is
 //                        tracked by the issuing thread's bulk groups; loads lead stores by a fixed lag;
@@ -70,24 +70,25 @@ __device__ __forceinline__ void copy_vecs(const uint4* __restrict__ s, uint4* __
     }
 }
 
-// All threads of the CTA call this with the same item.
+// All lanes of a warp call this with the same item: the warp alone moves it, UNROLL 16-byte loads in flight per lane
+// before the first store.  Rows shorter than 512 bytes are dealt to the lanes vector by vector across rows.
 template <int UNROLL>
-__device__ __forceinline__ void cta_copy_item(const Item& it) {
+__device__ __forceinline__ void warp_copy_item(const Item& it) {
+    const int lane = threadIdx.x & 31;
     if (it.n_rows == 1 || (it.src_pitch == it.row_bytes && it.dst_pitch == it.row_bytes)) {
         copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src), reinterpret_cast<uint4*>(it.dst),
-                          (it.n_rows * it.row_bytes) >> 4, threadIdx.x, blockDim.x);
-    } else if (it.row_bytes >= 512) {  // one warp per row, lanes along the row
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-        for (int r = warp; r < it.n_rows; r += nwarps)
+                          (it.n_rows * it.row_bytes) >> 4, lane, 32);
+    } else if (it.row_bytes >= 512) {
+        for (int r = 0; r < it.n_rows; ++r)
             copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch),
                               reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch), it.row_bytes >> 4, lane, 32);
-    } else {  // short rows: the vectors of all rows are dealt to the threads of the CTA
+    } else {
         const int vpr = it.row_bytes >> 4, n = it.n_rows * vpr;
-        for (int base = 0; base < n; base += blockDim.x * UNROLL) {
+        for (int base = 0; base < n; base += 32 * UNROLL) {
             uint4 v[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                const int i = base + u * blockDim.x + threadIdx.x;
+                const int i = base + u * 32 + lane;
                 if (i < n) {
                     const int r = i / vpr, c = i - r * vpr;
                     v[u] = ld_stream(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch) + c);
@@ -95,7 +96,7 @@ __device__ __forceinline__ void cta_copy_item(const Item& it) {
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                const int i = base + u * blockDim.x + threadIdx.x;
+                const int i = base + u * 32 + lane;
                 if (i < n) {
                     const int r = i / vpr, c = i - r * vpr;
                     st_stream(reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch) + c, v[u]);

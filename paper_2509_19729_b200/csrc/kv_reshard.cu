@@ -177,13 +177,15 @@ __device__ __forceinline__ int32_t clamp_pairs(const KvParams& p) {
     return n < 0 ? 0 : (n > p.pairs_cap ? p.pairs_cap : n);
 }
 
-template <int UNROLL>
-__global__ void __launch_bounds__(256) kv_reshard_ldst(const __grid_constant__ KvParams p) {
+// Vector load/store path: one work item per warp at a time, warps strided over the items.
+template <int UNROLL, int CTAS_PER_SM>
+__global__ void __launch_bounds__(256, CTAS_PER_SM) kv_reshard_ldst(const __grid_constant__ KvParams p) {
     const KvItems items{p, clamp_pairs(p)};
     const int64_t n = items.count();
-    for (int64_t w = blockIdx.x; w < n; w += gridDim.x) {
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < n; w += n_warps) {
         const Item it = items(w);
-        if (it.n_rows) cta_copy_item<UNROLL>(it);
+        if (it.n_rows) warp_copy_item<UNROLL>(it);
     }
 }
 
@@ -443,9 +445,12 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
                                          : (int64_t)g.planes * g.head_units * g.row_groups * g.col_chunks;
     const int64_t max_items = (int64_t)pairs_cap * p.n_layers * items_per_pair;
     if (path == 1) {
-        const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 16;
-        const int grid = (int)std::min<int64_t>(max_items, (int64_t)dev.sms * per_sm);
-        kv_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
+        // loads in flight per lane x resident CTAs: 8 x 2, 6 x 3 or 4 x 4 and more
+        const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : kLdstCtasPerSm;
+        const int grid = (int)std::min<int64_t>((max_items + 7) / 8, (int64_t)dev.sms * per_sm);
+        if (per_sm <= 2) kv_reshard_ldst<8, 2><<<grid, 256, 0, stream>>>(p);
+        else if (per_sm == 3) kv_reshard_ldst<6, 3><<<grid, 256, 0, stream>>>(p);
+        else kv_reshard_ldst<4, 4><<<grid, 256, 0, stream>>>(p);
         e = cudaGetLastError();
     } else if (boxes) {
         KvMaps maps;  // encoded per call: the pool addresses are arguments of this call

@@ -16,6 +16,7 @@ struct KernelDefaults {
 };
 constexpr KernelDefaults kKvDefaults{3, 4, 2, 5, 4};
 constexpr KernelDefaults kWDefaults{3, 4, 2, 5, 4};
+constexpr int kLdstCtasPerSm = 6;  // vector load/store kernels: resident CTAs per SM (and loads in flight per lane)
 
 struct DeviceInfo {
     int sms = 0;

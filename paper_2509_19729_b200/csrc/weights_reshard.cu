@@ -48,11 +48,13 @@ struct WItems {
     }
 };
 
-template <int UNROLL>
-__global__ void __launch_bounds__(256) w_reshard_ldst(const __grid_constant__ WParams p) {
+template <int UNROLL, int CTAS_PER_SM>
+__global__ void __launch_bounds__(256, CTAS_PER_SM) w_reshard_ldst(const __grid_constant__ WParams p) {
     const WItems items{p};
     const int64_t n = items.count();
-    for (int64_t w = blockIdx.x; w < n; w += gridDim.x) cta_copy_item<UNROLL>(items(w));
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < n; w += n_warps)
+        warp_copy_item<UNROLL>(items(w));
 }
 
 __global__ void __launch_bounds__(1024) w_reshard_bulk(const __grid_constant__ WParams p, const RingShape rs,
@@ -137,9 +139,11 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
         const int64_t n_items = (int64_t)p.items_per_layer * nl;
         cudaError_t e;
         if (path == 1) {
-            const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 16;
-            const int grid = (int)std::min<int64_t>(n_items, (int64_t)dev.sms * per_sm);
-            w_reshard_ldst<4><<<grid, 256, 0, stream>>>(p);
+            const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : kLdstCtasPerSm;
+            const int grid = (int)std::min<int64_t>((n_items + 7) / 8, (int64_t)dev.sms * per_sm);
+            if (per_sm <= 2) w_reshard_ldst<8, 2><<<grid, 256, 0, stream>>>(p);
+            else if (per_sm == 3) w_reshard_ldst<6, 3><<<grid, 256, 0, stream>>>(p);
+            else w_reshard_ldst<4, 4><<<grid, 256, 0, stream>>>(p);
             e = cudaGetLastError();
         } else {
             const BulkShape bs = bulk_shape(dev, opt, kWDefaults, path, stage_bytes);
