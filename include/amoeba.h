@@ -165,6 +165,10 @@ enum {
     AMOEBA_OPT_L2_HINT = 6,     /* 1 = none, 2 = loads evict-first, 3 = stores evict-first, 4 = both */
     AMOEBA_OPT_TENSOR_MAPS = 7, /* KV, bulk-copy paths, token-first sides: 1 = one bulk copy per token row,
                                    2 = one tiled (tensor-map) copy per work item */
+    AMOEBA_OPT_MAX_CTAS = 8,    /* cap on the persistent grid of the copy kernels (0 = none).  One CTA occupies one SM,
+                                   so a cap below the SM count leaves SMs to kernels running on other streams - the
+                                   paper launches its migration "when enough free SMs are available" (Sec. 3.1,
+                                   Improvement 2) */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };

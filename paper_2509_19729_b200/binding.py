@@ -12,7 +12,7 @@ from . import build as _build
 
 __all__ = [
     "AmoebaError", "Model", "Layout", "LayerWeights", "KvInfo", "WeightDesc", "Plan", "STATUS_NAMES", "TENSOR_NAMES",
-    "OPT_COPY_PATH", "OPT_CTAS_PER_SM", "OPT_CHUNK_BYTES", "OPT_STAGES", "OPT_LAG", "OPT_WARPS", "OPT_L2_HINT", "OPT_TENSOR_MAPS",
+    "OPT_COPY_PATH", "OPT_CTAS_PER_SM", "OPT_CHUNK_BYTES", "OPT_STAGES", "OPT_LAG", "OPT_WARPS", "OPT_L2_HINT", "OPT_TENSOR_MAPS", "OPT_MAX_CTAS",
     "OPT_WEIGHTS_ONLY", "OPT_KV_ONLY", "COPY_PATH_LDST", "COPY_PATH_BULK", "COPY_PATH_PAIR",
     "amoeba_plan_create", "amoeba_plan_destroy", "amoeba_layout_kv_pool_bytes", "amoeba_layout_weight_bytes", "amoeba_plan_bytes", "amoeba_plan_kv_info",
     "amoeba_plan_num_weight_descs", "amoeba_plan_weight_desc", "amoeba_plan_set_option",
@@ -28,7 +28,7 @@ BUILTIN_SCRATCH_BYTES = 1 << 20
 __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
             "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "BUILTIN_SCRATCH_BYTES",
             "amoeba_rewrite_block_tables_builtin_scratch"]
-OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS = range(8)
+OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS, OPT_MAX_CTAS = range(9)
 OPT_WEIGHTS_ONLY, OPT_KV_ONLY = 16, 32  # add to an option id to set one kernel only
 COPY_PATH_LDST, COPY_PATH_BULK, COPY_PATH_PAIR = 1, 2, 3
 KV_HEAD_MAJOR, KV_TOKEN_MAJOR = 0, 1  # [block][header][K/V][token][dim] / [K/V][block][token][header][dim]

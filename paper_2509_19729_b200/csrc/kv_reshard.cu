@@ -447,7 +447,7 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     if (path == 1) {
         // loads in flight per lane x resident CTAs: 8 x 2, 6 x 3 or 4 x 4 and more
         const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : kLdstCtasPerSm;
-        const int grid = (int)std::min<int64_t>((max_items + 7) / 8, (int64_t)dev.sms * per_sm);
+        const int grid = (int)std::min<int64_t>((max_items + 7) / 8, grid_cap(opt, (int64_t)dev.sms * per_sm));
         if (per_sm <= 2) kv_reshard_ldst<8, 2><<<grid, 256, 0, stream>>>(p);
         else if (per_sm == 3) kv_reshard_ldst<6, 3><<<grid, 256, 0, stream>>>(p);
         else kv_reshard_ldst<4, 4><<<grid, 256, 0, stream>>>(p);
@@ -467,7 +467,7 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
                     return AMOEBA_ERR_CUDA;
         const int stage_bytes = (int)((bx.item_bytes + 127) / 128 * 128);  // tiled copies want 128-byte aligned stages
         const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, stage_bytes);
-        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
         auto kernel = path == 3 ? kv_reshard_pair_box : kv_reshard_bulk_box;
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
         if (e == cudaSuccess) {
@@ -476,7 +476,7 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
         }
     } else {
         const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)g.item_bytes);
-        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+        const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
         auto kernel = path == 3 ? kv_reshard_pair : kv_reshard_bulk;
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
         if (e == cudaSuccess) {
@@ -534,7 +534,7 @@ static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void
     const int path = opt.copy_path == 2 ? 2 : 3;  // a swap needs a staged copy: the rings only
     const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)(2 * p.chunk_bytes));
     const int64_t n_items = (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
-    const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+    const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
     auto kernel = path == 3 ? kv_merge_pair : kv_merge_bulk;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
     if (e == cudaSuccess) {

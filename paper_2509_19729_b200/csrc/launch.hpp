@@ -33,6 +33,11 @@ inline bool device_info(DeviceInfo* out) {
     return out->sms > 0;
 }
 
+// Persistent grid size: the default (a multiple of the SM count), or the caller's cap when it leaves SMs to other work.
+inline int64_t grid_cap(const KernelOpts& opt, int64_t grid) {
+    return opt.max_ctas > 0 ? std::min<int64_t>(grid, opt.max_ctas) : grid;
+}
+
 constexpr int kBarrierBytes = 1024;  // head of dynamic shared memory: up to 128 mbarriers
 
 struct BulkShape {

@@ -449,6 +449,10 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
                 if (value > 4) return AMOEBA_ERR_INVALID_ARG;
                 k->hint = (int)value;
                 break;
+            case AMOEBA_OPT_MAX_CTAS:
+                if (value > (1 << 20)) return AMOEBA_ERR_INVALID_ARG;
+                k->max_ctas = (int)value;
+                break;
             case AMOEBA_OPT_TENSOR_MAPS:
                 if (value > 2) return AMOEBA_ERR_INVALID_ARG;
                 k->tensor_maps = (int)value;

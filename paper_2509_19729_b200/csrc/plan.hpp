@@ -50,6 +50,7 @@ struct KernelOpts {
     int lag = 0;          // loads ahead of stores (path 2) / stores kept in flight (path 3)
     int warps = 0;        // rings per CTA
     int hint = 0;         // 1 + bit mask: bit 0 loads evict-first, bit 1 stores evict-first (0 = default)
+    int max_ctas = 0;     // cap on the persistent grid (0 = none): leaves SMs free for kernels that run beside the copy
     int tensor_maps = 0;  // KV only: 1 = row copies on token-first sides, 2 = tensor-map boxes (0 = default)
 };
 

@@ -140,14 +140,14 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
         cudaError_t e;
         if (path == 1) {
             const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : kLdstCtasPerSm;
-            const int grid = (int)std::min<int64_t>((n_items + 7) / 8, (int64_t)dev.sms * per_sm);
+            const int grid = (int)std::min<int64_t>((n_items + 7) / 8, grid_cap(opt, (int64_t)dev.sms * per_sm));
             if (per_sm <= 2) w_reshard_ldst<8, 2><<<grid, 256, 0, stream>>>(p);
             else if (per_sm == 3) w_reshard_ldst<6, 3><<<grid, 256, 0, stream>>>(p);
             else w_reshard_ldst<4, 4><<<grid, 256, 0, stream>>>(p);
             e = cudaGetLastError();
         } else {
             const BulkShape bs = bulk_shape(dev, opt, kWDefaults, path, stage_bytes);
-            const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, (int64_t)dev.sms * bs.ctas_per_sm);
+            const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
             auto kernel = path == 3 ? w_reshard_pair : w_reshard_bulk;
             e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
             if (e == cudaSuccess) {

@@ -425,3 +425,12 @@ def test_writes_stay_inside_the_buffers():
             inside[o:o + s] = True
         assert bool((arena[~inside] == 0xC3).all())
         assert not bool((arena[inside] == 0xC3).all())  # and the buffers themselves were written
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("cap", [1, 7, 100000])
+def test_grid_cap_leaves_results_unchanged(path, cap):
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 2, 4, [300, 17, 64, 5], seed=41)
+    check_case(c, run_case(c, path, options=[(A.OPT_MAX_CTAS, cap)]))
