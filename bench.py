@@ -485,6 +485,8 @@ def main():
                          "conversion between them")
     ap.add_argument("--weight-pad", type=int, default=0,
                     help="P > 0: both sides hold their weights as P padded partitions per tensor (2 MiB pages)")
+    ap.add_argument("--opt", action="append", default=[], metavar="NAME=VALUE",
+                    help="any plan option by name (e.g. WARPS=6, LAG=3, L2_HINT=1, TENSOR_MAPS=1), repeatable")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the copy kernels' persistent grid (0 = all SMs)")
     ap.add_argument("--layers-per-call", type=int, default=0,
                     help="k > 0: transform k layers per call (KV and weights), as when a few layers are transformed "
@@ -518,6 +520,9 @@ def main():
                      (A.OPT_CTAS_PER_SM, args.ctas_per_sm), (A.OPT_MAX_CTAS, args.max_ctas)):
         if val:
             s.set_option(opt, val)
+    for item in args.opt:
+        name, val = item.split("=")
+        s.set_option(getattr(A, "OPT_" + name.upper()), int(val))
     kv_bytes, w_bytes = s.bytes_rw(st["n_live"])
     stream = torch.cuda.current_stream()
 
@@ -574,7 +579,7 @@ def main():
     peak, peak_kind = peaks()
     traffic_known = (NCU_KV_TRAFFIC_RATIO is not None and args.config == NCU_KV_TRAFFIC_CONFIG
                      and args.kv_order == "head"
-                     and not (args.copy_path or args.chunk or args.stages or args.ctas_per_sm or args.max_ctas))
+                     and not (args.copy_path or args.chunk or args.stages or args.ctas_per_sm or args.max_ctas or args.opt))
     kv_gbs = kv_bytes / (kv_ms / 1e3) / 1e9
     w_gbs = w_bytes / (w_ms / 1e3) / 1e9 if w_bytes else None
     out = {
@@ -585,7 +590,7 @@ def main():
                    "layers_per_call": args.layers_per_call or "all", "kv_order": args.kv_order, "weight_pad_parts": args.weight_pad, "sequences": cfg["S"], "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS,
                    "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
                    "l2_policy": "no flush: every step streams far more than the 126 MB L2",
-                   "max_ctas": args.max_ctas or "all SMs", "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],
+                   "max_ctas": args.max_ctas or "all SMs", "options": args.opt, "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],
                    "chunk_bytes": n_seq_layers[2]},
         "phases_ms": {"rewrite_block_tables": bt_ms, "reshard_kv": kv_ms, "reshard_weights": w_ms,
                       "reshard_kv_min": min(phase[1]), "reshard_weights_min": min(phase[2])},
