@@ -167,7 +167,7 @@ enum {
                                    2 = one tiled (tensor-map) copy per work item */
     AMOEBA_OPT_MAX_CTAS = 8,    /* cap on the persistent grid of the copy kernels (0 = none).  One CTA occupies one SM,
                                    so a cap below the SM count leaves SMs to kernels running on other streams - the
-                                   paper launches its migration "when enough free SMs are available" (Sec. 3.1,
+                                   paper starts its migration on a side stream once enough SMs are free (Sec. 3.1,
                                    Improvement 2) */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32

@@ -22,14 +22,14 @@
  *     [in,out] algebra FFN = f(I x U) x D.  Weights are stored [out,in] row-major here, so the paper's columns
  *     of U are rows of up/gate (contiguous) and the paper's rows of D are columns of down (strided).
  *     Attention projections follow the same rule by heads: q/k/v like U, o_proj like D.
- *   - Destination block bookkeeping (Sec. 3.1: each worker "prepares reserved pages" for incoming KV): the
+ *   - Destination block bookkeeping (Sec. 3.1: every worker sets pages aside for the KV it will receive): the
  *     paper gives no order; the reading used here is sequences in index order, logical blocks in order, each
  *     taking the next id of the ordered free list (list order, or ascending id when a mask is given).
  *
  *   - In-place migration (Sec. 3.1, "Improvement 1"; the scenario of Sec. 3.1's example, N x TP1 -> TP N, here
  *     N x TP a -> TP N*a): every worker keeps its memory.  A worker retains, for the requests of its own instance, the
  *     headers the target TP assigns to it, sends the other headers to their workers, and the room they leave is
- *     reused "through block reshaping": an old block of Hkv/a headers becomes N new blocks of Hkv/(N*a) headers.
+ *     reused by reshaping blocks: an old block of Hkv/a headers becomes N new blocks of Hkv/(N*a) headers.
  *     The paper names no block numbering; the reading used here: the worker r of instance i becomes worker r*N+i of
  *     the merged instance (so that, with a = 1, W_i keeps header group i as in the paper's example), and block p of
  *     instance i becomes block p*N+i of the merged instance (on every worker: the block table stays shared).  With
