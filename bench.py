@@ -266,6 +266,90 @@ def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED
     return s, st
 
 
+def build_merge_copy_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, kv_order="head"):
+    """The same merge workload done out of place: N source instances, one fresh set of destination pools."""
+    import torch
+
+    from paper_2509_19729_b200.session import MergeCopySession
+
+    cfg = wl.MERGE_CONFIGS[cfg_name]
+    m = dict(cfg["model"])
+    if layers is not None:
+        m["L"] = layers
+    st = wl.draw_merge_state(cfg, seed=seed, name=cfg_name)
+    NB_dst = st["n_live"] + max(st["n_live"] // 64, 1)
+    free = wl.rng(seed, "merge_dst_blocks", *cfg_name.encode()).permutation(NB_dst).astype(np.int32)
+    s = MergeCopySession(m, cfg["N"], cfg["a"], st["NB"], NB_dst, st["seq_lens"], st["src_bt"], free, device=device,
+                         src_kv_order=KV_ORDERS[kv_order][0], dst_kv_order=KV_ORDERS[kv_order][1])
+    k = 0
+    for inst in s.src_pools:
+        for p in inst:
+            wl.hash_fill_(p, seed, 400 + k)
+            k += 1
+    for p in s.dst_pools:
+        p.fill_(0xA5)
+    torch.cuda.synchronize()
+    return s, st
+
+
+def run_merge_copy(args, rank, world, local):
+    """Out-of-place variant of the merge workload (what the merge costs without in-place block reshaping)."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    cfg = wl.MERGE_CONFIGS[args.config]
+    s, st = build_merge_copy_session(args.config, device, layers=args.layers, kv_order=args.kv_order)
+    nbytes = s.bytes_rw()
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        s.status.zero_()
+        s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = A.amoeba_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for _ in range(args.steps):
+        s.step()
+    t1.record(stream)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    barrier(world)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0
+    sec = t0.elapsed_time(t1) / 1e3 / args.steps
+    sec_all, bytes_all = aggregate(world, sec, nbytes, device)
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    N, a = cfg["N"], cfg["a"]
+    gbs = bytes_all / sec_all / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{N}x{a}->{N * a} out of place", "kv_order": args.kv_order,
+                   "layers": s.kv_layers, "sequences_per_instance": cfg["S"], "live_blocks": st["n_live"],
+                   "kv_bytes_rw": nbytes, "weight_bytes_rw": 0,
+                   "source_pool_bytes": sum(p.numel() for inst in s.src_pools for p in inst),
+                   "extra_kv_memory_bytes": sum(p.numel() for p in s.dst_pools),
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
+        "roofline": {"kernel": "kv_reshard_pair" if args.kv_order == "head" else "kv_reshard_pair_box", "bound": "hbm",
+                     "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": None,
+    }))
+
+
 def run_merge(args, rank, world, local):
     """In-place merge workload: one step = merged block tables + the in-place KV exchange of all layers.  (A second
     step over the same tables exchanges the same segments back: every step moves the same bytes.)"""
@@ -485,6 +569,8 @@ def main():
                          "conversion between them")
     ap.add_argument("--weight-pad", type=int, default=0,
                     help="P > 0: both sides hold their weights as P padded partitions per tensor (2 MiB pages)")
+    ap.add_argument("--merge-mode", default="inplace", choices=["inplace", "outofplace"],
+                    help="merge workloads: exchange segments in place (default) or copy every instance into fresh pools")
     ap.add_argument("--opt", action="append", default=[], metavar="NAME=VALUE",
                     help="any plan option by name (e.g. WARPS=6, LAG=3, L2_HINT=1, TENSOR_MAPS=1), repeatable")
     ap.add_argument("--max-ctas", type=int, default=0, help="cap on the copy kernels' persistent grid (0 = all SMs)")
@@ -504,7 +590,7 @@ def main():
         return
 
     if args.config in wl.MERGE_CONFIGS:
-        run_merge(args, rank, world, local)
+        (run_merge if args.merge_mode == "inplace" else run_merge_copy)(args, rank, world, local)
         return
 
     import torch

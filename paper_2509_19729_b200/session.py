@@ -188,3 +188,63 @@ class MergeSession:
     def bytes_rw(self, n_live: int) -> int:
         """Bytes read + written by one merge with n_live live old blocks (summed over instances), held layers."""
         return A.amoeba_merge_bytes(self.plan, n_live) * self.kv_layers // self.L
+
+
+
+class MergeCopySession:
+    """N instances of TP=a become one instance of TP=N*a in FRESH pools (out of place): one table rewrite and one KV
+    call per instance, each given the part of the shared destination free list the earlier instances left.  This is
+    what a merge costs without in-place block reshaping (and the only way with token-first pools); it needs a second
+    set of pools.  seq_lens [N][S] and src_bt [N][S][maxb] are host arrays (the block counts that advance the free list
+    are computed from the lengths on the host)."""
+
+    def __init__(self, model: dict, N: int, a: int, NB_src: int, NB_dst: int, seq_lens, src_bt, free_list,
+                 kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0",
+                 src_kv_order: int = A.KV_HEAD_MAJOR, dst_kv_order: int = A.KV_HEAD_MAJOR):
+        self.model, self.N, self.a = model, N, a
+        self.device = dev = torch.device(device)
+        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, kv_order=src_kv_order)
+        self.dst_layout = A.make_layout(model, N * a, NB_dst, block_tokens, kv_order=dst_kv_order)
+        self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
+        self.L = model["L"]
+        self.kv_layers = self.L if kv_layers is None else kv_layers
+        lens = torch.as_tensor(seq_lens, dtype=torch.int32)
+        bt = torch.as_tensor(src_bt, dtype=torch.int32)
+        self.num_seqs, self.maxb = int(bt.shape[1]), int(bt.shape[2])
+        i32 = dict(dtype=torch.int32, device=dev)
+        counts = [int(((lens[i].long() + block_tokens - 1) // block_tokens).sum()) for i in range(N)]
+        self.counts, self.offsets = counts, [sum(counts[:i]) for i in range(N)]
+        self.free_list = torch.as_tensor(free_list, dtype=torch.int32).to(dev)
+        assert self.free_list.numel() >= sum(counts)
+        self.seq_lens, self.src_bt = lens.to(dev), bt.to(dev)
+        self.dst_bt = torch.full(tuple(bt.shape), -2, **i32)
+        self.pairs = [torch.full((max(c, 1), 2), -3, **i32) for c in counts]
+        self.num_pairs = torch.zeros(N, **i32)
+        self.free_count = torch.zeros(N, **i32)
+        self.status = torch.zeros(1, **i32)
+        self.ws_bytes = A.amoeba_rewrite_workspace_bytes(self.plan, self.num_seqs, self.free_list.numel())
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        src_per_layer = A.amoeba_layout_kv_pool_bytes(self.src_layout) // self.L
+        dst_per_layer = A.amoeba_layout_kv_pool_bytes(self.dst_layout) // self.L
+        self.src_pools = [[torch.empty(src_per_layer * self.kv_layers, dtype=torch.uint8, device=dev) for _ in range(a)]
+                          for _ in range(N)]
+        self.dst_pools = [torch.empty(dst_per_layer * self.kv_layers, dtype=torch.uint8, device=dev)
+                          for _ in range(N * a)]
+
+    def step(self, stream=None) -> None:
+        n_free = self.free_list.numel()
+        for i in range(self.N):
+            off = self.offsets[i]
+            A.amoeba_rewrite_block_tables(self.plan, self.src_bt[i], self.seq_lens[i], self.num_seqs, self.maxb,
+                                          self.free_list[off:], None, n_free - off, self.dst_bt[i], self.pairs[i],
+                                          self.counts[i], self.num_pairs[i:i + 1], self.free_count[i:i + 1],
+                                          self.status, self.workspace, self.ws_bytes, stream)
+            A.amoeba_reshard_kv(self.plan, self.src_pools[i], self.dst_pools, self.pairs[i], self.num_pairs[i:i + 1],
+                                self.counts[i], 0, self.kv_layers, self.status, stream)
+
+    def set_option(self, option: int, value: int) -> None:
+        A.amoeba_plan_set_option(self.plan, option, value)
+
+    def bytes_rw(self) -> int:
+        kv, _ = A.amoeba_plan_bytes(self.plan, sum(self.counts))
+        return kv * self.kv_layers // self.L

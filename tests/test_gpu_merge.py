@@ -281,3 +281,36 @@ def test_split_device_detected_errors(oracle):
     assert got_status == exp_status == 1 and np.array_equal(got_bt, exp_bt) and not got_live.any()
     for g, e in zip(got_pools, exp_pools):
         assert np.array_equal(g, e)
+
+
+@pytest.mark.parametrize("order", ["head", "token"])
+def test_out_of_place_merge_session_matches_oracle(oracle, order):
+    """The benchmark's out-of-place merge plumbing on the tiny merge workload: every destination pool equals the
+    oracle's a -> N*a transformation of each instance with the free list advanced by the earlier instances."""
+    import torch
+
+    import bench
+    import workloads as wl
+
+    name = "tiny_merge_2x1to2"
+    cfg = wl.MERGE_CONFIGS[name]
+    m, N, a, T = cfg["model"], cfg["N"], cfg["a"], wl.BLOCK_TOKENS
+    so, do = bench.KV_ORDERS[order]
+    s, st = bench.build_merge_copy_session(name, torch.device("cuda:0"), kv_order=order)
+    s.status.zero_()
+    s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    NB_dst = s.dst_layout.num_blocks
+    free = s.free_list.cpu().numpy()
+    exp = [np.full(m["L"] * oracle.pool_elems_per_layer(m, T, N * a, NB_dst), 0xA5A5, np.uint16) for _ in range(N * a)]
+    for i in range(N):
+        src = [p.cpu().numpy().view(np.uint16) for p in s.src_pools[i]]
+        exp_bt, _, n, _, status = oracle.assign_blocks(st["seq_lens"][i], T, st["src_bt"][i], st["NB"], NB_dst,
+                                                       free_list=free[s.offsets[i]:])
+        assert status == 0 and n == s.counts[i]
+        assert np.array_equal(s.dst_bt[i].cpu().numpy(), exp_bt)
+        oracle.kv_transform(m, T, st["seq_lens"][i], a, st["NB"], st["src_bt"][i], src, N * a, NB_dst, exp_bt, exp,
+                            src_order=so, dst_order=do)
+    for w in range(N * a):
+        assert np.array_equal(s.dst_pools[w].cpu().numpy().view(np.uint16), exp[w]), w
