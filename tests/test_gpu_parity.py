@@ -434,3 +434,28 @@ def test_grid_cap_leaves_results_unchanged(path, cap):
 
     c = make_case(GQA, 2, 4, [300, 17, 64, 5], seed=41)
     check_case(c, run_case(c, path, options=[(A.OPT_MAX_CTAS, cap)]))
+
+
+def test_random_shapes_orders_and_options():
+    """Seeded random small cases: block sizes from 1 token, head dims from 8, any divisor pair of TP degrees, either
+    storage order on either side, every copy path, odd chunk sizes."""
+    import paper_2509_19729_b200 as A
+
+    g = np.random.default_rng(2509)
+    for trial in range(48):
+        Hkv = int(g.choice([1, 2, 4, 6, 8, 12]))
+        D = int(g.choice([8, 16, 40, 64, 128]))
+        T = int(g.choice([1, 3, 8, 16, 32]))
+        divs = [d for d in (1, 2, 3, 4, 6, 8, 12) if Hkv % d == 0]
+        a, b = int(g.choice(divs)), int(g.choice(divs))
+        m = dict(L=int(g.integers(1, 4)), hidden=64, Hq=Hkv * int(g.choice([1, 2])), Hkv=Hkv, D=D, I=Hkv * 16)
+        so, do = int(g.integers(2)), int(g.integers(2))
+        path, tm = VARIANTS[int(g.integers(len(VARIANTS)))]
+        chunk = int(g.choice([16, 48, 256, 4096, 8192, 65536]))
+        lens = [int(x) for x in g.integers(0, 6 * T, size=int(g.integers(1, 7)))]
+        c = make_case(m, a, b, lens, T=T, weights=bool(g.integers(2)), seed=trial, src_order=so, dst_order=do)
+        try:
+            check_case(c, run_case(c, path, options=_opts(tm, [(A.OPT_CHUNK_BYTES, chunk)])))
+        except Exception as e:
+            raise AssertionError(f"trial {trial}: m={m} T={T} {a}->{b} orders {so}{do} path {path} tm {tm} chunk {chunk} "
+                                 f"lens {lens}: {e}") from e
