@@ -59,7 +59,8 @@ enum {
     AMOEBA_KV_HEAD_MAJOR = 0, /* [block][header][K/V][token][dim] */
     AMOEBA_KV_TOKEN_MAJOR = 1 /* [K/V][block][token][header][dim] */
 };
-enum { AMOEBA_MAX_TP = 32 }; /* and at most 22 intersecting (source worker, destination worker) pairs */
+enum { AMOEBA_MAX_TP = 32 }; /* and at most 36 intersecting (source worker, destination worker) pairs: 256 weight
+                                descriptors per layer; nested degrees up to 32 -> 1 and 1 -> 32 fit */
 
 /* Transformer shape.  elem_bytes is the size of one weight / KV element (2: fp16 or bf16). */
 typedef struct {

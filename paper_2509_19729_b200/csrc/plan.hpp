@@ -8,8 +8,9 @@
 namespace amoeba {
 
 constexpr int kNumTensors = 7;  // q,k,v,o,gate,up,down
-constexpr int kMaxWeightDescs = 160;
-constexpr int kMaxWeightPtrs = 2048;  // per launch: layers * (a + b) * kNumTensors pointers
+constexpr int kMaxWeightDescs = 256;
+constexpr int kMaxWeightPtrs = 1536;  // per launch: layers * (a + b) * kNumTensors pointers
+// (descriptors and pointers travel in kernel parameter space: 256 * 72 + 1536 * 8 bytes, under the 32 KiB limit)
 constexpr int64_t kDefaultKvChunk = 8192;   // upper bound of one KV copy work item
 constexpr int64_t kDefaultWChunk = 8192;    // upper bound of one weight copy work item
 

@@ -459,3 +459,13 @@ def test_random_shapes_orders_and_options():
         except Exception as e:
             raise AssertionError(f"trial {trial}: m={m} T={T} {a}->{b} orders {so}{do} path {path} tm {tm} chunk {chunk} "
                                  f"lens {lens}: {e}") from e
+
+
+@pytest.mark.parametrize("a,b", [(32, 1), (1, 32), (32, 32), (16, 32)])
+def test_largest_tp_degrees(a, b):
+    """The largest worker counts the library accepts: 32 pools on a side, one header per worker."""
+    wide = dict(L=2, hidden=128, Hq=32, Hkv=32, D=16, I=512)
+    c = make_case(wide, a, b, [70, 9, 33], T=8, seed=a + b)
+    check_case(c, run_case(c))
+    c = make_case(wide, a, b, [70, 9], T=8, weights=False, seed=a + b, src_order=TF, dst_order=HC)
+    check_case(c, run_case(c))
