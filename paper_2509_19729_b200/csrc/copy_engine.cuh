@@ -6,7 +6,7 @@
 //   * warp_copy_item     a warp moves an item with 16-byte vector loads / stores, all loads of an unrolled batch
 //                        issued before the first store, streaming cache hints;
 //   * warp_bulk_ring     each warp drives its own ring of shared-memory stages with the bulk-copy engine (TMA, 1-D
-//                        cp.async.bulk, no multicast): global -> shared completes on an mbarrier, shared -> global is
+//                        cp.async.bulk, one CTA, no cluster): global -> shared completes on an mbarrier, shared -> global is
 //                        tracked by the issuing thread's bulk groups; loads lead stores by a fixed lag;
 //   * pair_bulk_ring     a producer warp and a consumer warp share one ring: the producer only issues loads (waits
 //                        on "empty" barriers), the consumer only issues stores (waits on "full" barriers), so the
