@@ -326,7 +326,9 @@ AMOEBA_API amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_l
  * src is a HOST array [a][num_layers] (worker-major) of device pointers, dst likewise [b][num_layers]; only layers
  * in [layer_begin, layer_end) are read.  Either side may be padded (weight_pad_parts): padded -> padded moves whole
  * partitions, dense <-> padded changes the pitch; pad bytes of the destination keep their values (zero them once at
- * load time if a GEMM is to run over a whole padded buffer, Eq. 2).  A caller transforming a few layers per inference step (Sec. 3.3's
+ * load time if a GEMM is to run over a whole padded buffer, Eq. 2).  A destination worker whose seven pointers are all
+ * NULL in a layer is left out: its shard is not produced (a worker that only needs its own new shard, as each worker
+ * of a merge does, passes the others as NULL).  Any other NULL pointer a descriptor needs is INVALID_ARG.  A caller transforming a few layers per inference step (Sec. 3.3's
  * layer-by-layer order) passes successive ranges.
  */
 AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const amoeba_layer_weights* src,

@@ -42,6 +42,13 @@ struct WItems {
         it.dst_pitch = d.dst_pitch;
         const char* s = static_cast<const char*>(p.ptrs[(layer * p.src_tp) * kNumTensors + d.src_slot]);
         char* t = static_cast<char*>(p.ptrs[p.dst_base + (layer * p.dst_tp) * kNumTensors + d.dst_slot]);
+        if (!t) {  // this destination worker's buffers were not given: its shard is not produced by this call
+            it.n_rows = 0;
+            it.row_bytes = 0;
+            it.src = nullptr;
+            it.dst = nullptr;
+            return it;
+        }
         it.src = s + d.src_off + r0 * d.src_pitch + off;
         it.dst = t + d.dst_off + r0 * d.dst_pitch + off;
         return it;
@@ -98,11 +105,20 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
     const int L = plan->src.model.num_layers, a = plan->src.tp, b = plan->dst.tp;
     if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
     const int n_descs = (int)plan->wdev.size();
-    // every buffer a descriptor names must be present and aligned, for every requested layer
+    // Every buffer a descriptor names must be present and aligned, for every requested layer - except that a
+    // destination worker may be left out of a layer altogether (all seven pointers NULL): its shard is then not produced.
+    auto left_out = [&](int rank, int l) {
+        void* const* sl = slots(&dst[(size_t)rank * L + l]);
+        for (int t = 0; t < kNumTensors; ++t)
+            if (sl[t]) return false;
+        return true;
+    };
     for (int l = layer_begin; l < layer_end; ++l)
         for (const WDescDev& d : plan->wdev) {
+            const int dst_rank = d.dst_slot / kNumTensors;
+            const void* t = slots(&dst[(size_t)dst_rank * L + l])[d.dst_slot % kNumTensors];
+            if (!t && left_out(dst_rank, l)) continue;
             const void* s = slots(&src[(size_t)(d.src_slot / kNumTensors) * L + l])[d.src_slot % kNumTensors];
-            const void* t = slots(&dst[(size_t)(d.dst_slot / kNumTensors) * L + l])[d.dst_slot % kNumTensors];
             if (!s || !t) return AMOEBA_ERR_INVALID_ARG;
             if (reinterpret_cast<uintptr_t>(s) % 16 || reinterpret_cast<uintptr_t>(t) % 16) return AMOEBA_ERR_ALIGNMENT;
         }

@@ -469,3 +469,43 @@ def test_largest_tp_degrees(a, b):
     check_case(c, run_case(c))
     c = make_case(wide, a, b, [70, 9], T=8, weights=False, seed=a + b, src_order=TF, dst_order=HC)
     check_case(c, run_case(c))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_weights_for_a_subset_of_destination_workers(path):
+    """Each worker of a merge only needs its own new shard: destination workers passed as all-NULL are left out, the
+    others get exactly what a full call gives them; a half-given worker is an error."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    m, a, b = dict(GQA, L=2), 1, 4
+    dev = torch.device("cuda:0")
+    g = np.random.default_rng(77)
+    plan = A.amoeba_plan_create(A.make_layout(m, a, 4), A.make_layout(m, b, 4))
+    A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, path)
+    src, exp = [], []
+    for l in range(m["L"]):
+        W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in O.logical_shapes(m).items()}
+        sa = O.weights_shard(W, m, a)
+        src.append(sa)
+        exp.append(O.weights_transform(sa, m, a, b))
+    d_src = [[{n: torch.from_numpy(x.reshape(-1).view(np.uint8)).to(dev) for n, x in src[l][0].items()}
+              for l in range(m["L"])]]
+    keep = (1, 3)  # the destination workers this call produces
+    d_dst = [[({n: torch.full((x.size * 2,), 0xA5, dtype=torch.uint8, device=dev) for n, x in exp[l][r].items()}
+               if r in keep else {}) for l in range(m["L"])] for r in range(b)]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    A.amoeba_reshard_weights(plan, d_src, d_dst, 0, m["L"], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for r in keep:
+        for l in range(m["L"]):
+            for n, e in exp[l][r].items():
+                assert np.array_equal(d_dst[r][l][n].cpu().numpy().view(np.uint16), e.reshape(-1)), (r, l, n)
+    half = [[dict(d) for d in row] for row in d_dst]
+    del half[1][0]["o"]
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_reshard_weights(plan, d_src, half, 0, m["L"], status)
+    assert e.value.status == A.ERR_INVALID_ARG
