@@ -128,16 +128,18 @@ def kv_reconstruct(pools, m, T, TP, NB, seq_lens, bt, layer_stride=None, order=H
 
 
 def kv_transform(m, T, seq_lens, a, NB_src, src_bt, src_pools, b, NB_dst, dst_bt, dst_pools,
-                 src_order=HEADER_CENTRIC, dst_order=HEADER_CENTRIC):
+                 src_order=HEADER_CENTRIC, dst_order=HEADER_CENTRIC, src_layer_stride=None, dst_layer_stride=None):
     """TP a->b on the KV pools: writes the live blocks of ``dst_pools`` in place (reconstruct, then shard)."""
     sl, slp = _i32(seq_lens)
     sbt, sbtp = _i32(src_bt)
     dbt, dbtp = _i32(dst_bt)
     assert sbt.shape == dbt.shape
     mm = _model(m)
+    ss = pool_elems_per_layer(m, T, a, NB_src) if src_layer_stride is None else src_layer_stride  # in elements
+    ds = pool_elems_per_layer(m, T, b, NB_dst) if dst_layer_stride is None else dst_layer_stride
     rc = lib().oracle_kv_transform(C.byref(mm), T, len(sl), slp, sbt.shape[1], a, NB_src, src_order,
-                                   C.c_int64(pool_elems_per_layer(m, T, a, NB_src)), sbtp, _ptr_array(src_pools), b,
-                                   NB_dst, dst_order, C.c_int64(pool_elems_per_layer(m, T, b, NB_dst)), dbtp,
+                                   C.c_int64(ss), sbtp, _ptr_array(src_pools), b,
+                                   NB_dst, dst_order, C.c_int64(ds), dbtp,
                                    _ptr_array(dst_pools))
     assert rc == 0
 

@@ -509,3 +509,48 @@ def test_weights_for_a_subset_of_destination_workers(path):
     with pytest.raises(A.AmoebaError) as e:
         A.amoeba_reshard_weights(plan, d_src, half, 0, m["L"], status)
     assert e.value.status == A.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("path,tm", VARIANTS)
+@pytest.mark.parametrize("so,do", [(HC, HC)] + ORDERS)
+def test_layers_further_apart_than_their_size(path, tm, so, do):
+    """kv_layer_stride_bytes larger than a layer on both sides: the gaps between layers keep their bytes."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    m, T, a, b, NB_s, NB_d = dict(GQA, L=3), 16, 2, 4, 9, 11
+    lens = np.array([40, 7, 64], np.int32)
+    nblk = (lens + T - 1) // T
+    g = np.random.default_rng(so * 2 + do)
+    bt = np.full((3, int(nblk.max())), -1, np.int32)
+    ids, k = g.permutation(NB_s), 0
+    for s, n in enumerate(nblk):
+        bt[s, :n] = ids[k:k + n]
+        k += int(n)
+    s_stride = O.pool_elems_per_layer(m, T, a, NB_s) + 2048   # elements
+    d_stride = O.pool_elems_per_layer(m, T, b, NB_d) + 512
+    KV = g.integers(0, 65536, size=(m["L"], int(nblk.sum()) * T, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    src = O.kv_shard(KV, m, T, a, NB_s, lens, bt, fill=0x5A5A, layer_stride=s_stride, order=so)
+    free = g.permutation(NB_d).astype(np.int32)
+    exp_bt, exp_pairs, n, _, st = O.assign_blocks(lens, T, bt, NB_s, NB_d, free_list=free)
+    exp = [np.full(m["L"] * d_stride, 0xA5A5, np.uint16) for _ in range(b)]
+    O.kv_transform(m, T, lens, a, NB_s, bt, src, b, NB_d, exp_bt, exp, src_order=so, dst_order=do,
+                   src_layer_stride=s_stride, dst_layer_stride=d_stride)
+    dev = torch.device("cuda:0")
+    plan = A.amoeba_plan_create(A.make_layout(m, a, NB_s, T, kv_order=so, kv_layer_stride_bytes=2 * s_stride),
+                                A.make_layout(m, b, NB_d, T, kv_order=do, kv_layer_stride_bytes=2 * d_stride))
+    for o, v in [(A.OPT_COPY_PATH, path)] + _opts(tm):
+        A.amoeba_plan_set_option(plan, o, v)
+    assert A.amoeba_layout_kv_pool_bytes(plan.dst) == 2 * d_stride * m["L"]
+    d_src = [torch.from_numpy(p.view(np.uint8)).to(dev) for p in src]
+    d_dst = [torch.full((p.size * 2,), 0xA5, dtype=torch.uint8, device=dev) for p in exp]
+    d_pairs = torch.from_numpy(exp_pairs).to(dev)
+    d_n = torch.tensor([n], dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    A.amoeba_reshard_kv(plan, d_src, d_dst, d_pairs, d_n, n, 0, m["L"], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for r in range(b):
+        assert np.array_equal(d_dst[r].cpu().numpy().view(np.uint16), exp[r]), r
