@@ -554,3 +554,12 @@ def test_layers_further_apart_than_their_size(path, tm, so, do):
     assert int(status.item()) == 0
     for r in range(b):
         assert np.array_equal(d_dst[r].cpu().numpy().view(np.uint16), exp[r]), r
+
+
+@pytest.mark.parametrize("hint", [1, 2, 3, 4])
+@pytest.mark.parametrize("so,do", [(HC, HC), (TF, TF), (TF, HC), (HC, TF)])
+def test_l2_hints_on_bulk_and_tiled_copies(hint, so, do):
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 2, 4, [100, 3, 48], seed=hint, src_order=so, dst_order=do)
+    check_case(c, run_case(c, PAIR, options=[(A.OPT_L2_HINT, hint)]))
