@@ -336,6 +336,23 @@ AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
                                      int32_t* d_status, void* cuda_stream);
 
 /*
+ * amoeba_compact_weights_inplace  (Sec. 3.2, base solution "partial swap": the part of a shard a worker keeps is moved
+ * to the start of the layer's weight space so that the rest can be released; the paper does it with a blocking copy)
+ *
+ * The plan's source layout is the instance before (TP = a), its destination layout the instance after (TP = N*a);
+ * both dense (no padding), same fused flags.  bufs is a HOST array [a][num_layers] of the a workers' buffers;
+ * keep[r] in [0, N) (host array) says which N-th of its shards worker r keeps: it becomes worker r*N + keep[r] of the
+ * new partition.  After the call the first bytes of every buffer hold exactly that worker's dense TP = N*a shard
+ * (the same bytes amoeba_reshard_weights writes for that worker); the bytes behind it are unspecified leftovers.
+ * No second buffer is used; 1/N of the weights is read and written.  The moves are ordered on the stream so that no
+ * byte is overwritten before it has been moved (a few launches per call, not one).  Errors: INVALID_ARG (null pointers,
+ * keep out of range, layers), UNSUPPORTED (padded layouts, different fused flags, TP not a multiple), ALIGNMENT, CUDA.
+ */
+AMOEBA_API amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
+                                             const int32_t* keep, int32_t layer_begin, int32_t layer_end,
+                                             int32_t* d_status, void* cuda_stream);
+
+/*
  * amoeba_plan_weight_alias  (Sec. 3.2, Improvement 1: with padded partitions a scale-up needs no weight copy at all)
  *
  * When both layouts are padded with the same weight_pad_parts, page size and fused flags and the destination TP is a

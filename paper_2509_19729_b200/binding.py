@@ -115,6 +115,7 @@ def _load():
         "amoeba_split_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, VP, VP]),
         "amoeba_merge_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
         "amoeba_split_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
+        "amoeba_compact_weights_inplace": (I32, [VP, P(LayerWeights), P(I32), I32, I32, VP, VP]),
         "amoeba_plan_weight_alias": (I32, [VP, I32, I32, P(I32), P(I64), P(I64)]),
         "amoeba_launch_count": (I64, []),
         "amoeba_status_string": (C.c_char_p, [I32]),
@@ -351,6 +352,22 @@ def amoeba_split_kv_inplace(plan: Plan, pools: Sequence, live, layer_begin: int,
 
 
 __all__ += ["amoeba_split_kv_inplace", "amoeba_merge_live_bytes", "amoeba_merge_bytes", "amoeba_merge_block_tables", "amoeba_merge_kv_inplace"]
+
+
+def amoeba_compact_weights_inplace(plan: Plan, bufs, keep: Sequence[int], layer_begin: int, layer_end: int, status,
+                                   stream=None) -> None:
+    """``bufs``: ``pack_weights`` array or [rank][layer] list of dicts of the TP=a workers' buffers; ``keep[r]``: which
+    N-th of its shards worker r keeps (it becomes worker r*N + keep[r] of TP = N*a)."""
+    if not isinstance(bufs, C.Array):
+        bufs = pack_weights(bufs)
+    if len(bufs) != plan.src.tp * plan.src.model.num_layers or len(keep) != plan.src.tp:
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_compact_weights_inplace (need [tp][num_layers] buffers, tp keeps)")
+    k = (C.c_int32 * len(keep))(*[int(x) for x in keep])
+    _check(_load().amoeba_compact_weights_inplace(plan.handle, bufs, k, layer_begin, layer_end, _ptr(status),
+                                                  _stream(stream)), "amoeba_compact_weights_inplace")
+
+
+__all__.append("amoeba_compact_weights_inplace")
 
 
 def amoeba_plan_weight_alias(plan: Plan, dst_rank: int, tensor: int):

@@ -89,6 +89,32 @@ static int64_t chunk_of(int64_t total, int64_t cap) {
     return 16;
 }
 
+// One public descriptor in kernel form: long rows are cut into column chunks of at most `cap` bytes, short rows are
+// grouped so that a work item is at most `cap` bytes.  *item counts the work items so far.
+WDescDev chunk_desc(const amoeba_weight_desc& d, int64_t cap, int64_t* item) {
+    WDescDev w{};
+    w.src_off = d.src_off;
+    w.dst_off = d.dst_off;
+    w.src_pitch = d.src_pitch;
+    w.dst_pitch = d.dst_pitch;
+    w.row_bytes = d.row_bytes;
+    w.n_rows = d.n_rows;
+    w.src_slot = d.src_rank * kNumTensors + d.src_tensor;
+    w.dst_slot = d.dst_rank * kNumTensors + d.dst_tensor;
+    if (d.row_bytes > cap) {
+        w.rows_per_item = 1;
+        w.col_chunks = (int32_t)((d.row_bytes + cap - 1) / cap);
+        w.chunk_bytes = (int32_t)cap;
+    } else {
+        w.rows_per_item = (int32_t)std::min<int64_t>(std::max<int64_t>(1, cap / d.row_bytes), d.n_rows);
+        w.col_chunks = 1;
+        w.chunk_bytes = (int32_t)d.row_bytes;
+    }
+    w.item_begin = (int32_t)*item;
+    *item += (int64_t)((d.n_rows + w.rows_per_item - 1) / w.rows_per_item) * w.col_chunks;
+    return w;
+}
+
 amoeba_status finalize_chunks(amoeba_plan* p) {
     const int64_t kv_cap = p->opt.kv.chunk_bytes > 0 ? p->opt.kv.chunk_bytes : kDefaultKvChunk;
     const int64_t cap = p->opt.w.chunk_bytes > 0 ? p->opt.w.chunk_bytes : kDefaultWChunk;
@@ -152,28 +178,8 @@ amoeba_status finalize_chunks(amoeba_plan* p) {
     p->wdev.clear();
     int64_t item = 0;
     for (const amoeba_weight_desc& d : p->wdescs) {
-        WDescDev w{};
-        w.src_off = d.src_off;
-        w.dst_off = d.dst_off;
-        w.src_pitch = d.src_pitch;
-        w.dst_pitch = d.dst_pitch;
-        w.row_bytes = d.row_bytes;
-        w.n_rows = d.n_rows;
-        w.src_slot = d.src_rank * kNumTensors + d.src_tensor;
-        w.dst_slot = d.dst_rank * kNumTensors + d.dst_tensor;
-        if (d.row_bytes > cap) {
-            w.rows_per_item = 1;
-            w.col_chunks = (int32_t)((d.row_bytes + cap - 1) / cap);
-            w.chunk_bytes = (int32_t)cap;
-        } else {
-            w.rows_per_item = (int32_t)std::min<int64_t>(std::max<int64_t>(1, cap / d.row_bytes), d.n_rows);
-            w.col_chunks = 1;
-            w.chunk_bytes = (int32_t)d.row_bytes;
-        }
-        w.item_begin = (int32_t)item;
-        item += (int64_t)((d.n_rows + w.rows_per_item - 1) / w.rows_per_item) * w.col_chunks;
+        p->wdev.push_back(chunk_desc(d, cap, &item));
         if (item > INT32_MAX) return AMOEBA_ERR_UNSUPPORTED;
-        p->wdev.push_back(w);
     }
     p->items_per_layer = (int32_t)item;
     return AMOEBA_OK;

@@ -103,6 +103,8 @@ struct amoeba_plan {
 namespace amoeba {
 // Number of instances N if the plan describes an in-place merge of N instances (see amoeba.h), else 0.
 int merge_instances(const amoeba_plan* p);
+// One public weight descriptor in kernel form; *item is the running count of work items.
+WDescDev chunk_desc(const amoeba_weight_desc& d, int64_t cap, int64_t* item);
 // Re-derives chunk sizes and the per-descriptor work-item split from plan->opt.
 amoeba_status finalize_chunks(amoeba_plan* p);
 void count_launch(int n = 1);

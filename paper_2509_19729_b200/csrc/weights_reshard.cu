@@ -93,53 +93,30 @@ __global__ void __launch_bounds__(1024) w_reshard_pair(const __grid_constant__ W
 
 static void* const* slots(const amoeba_layer_weights* w) { return reinterpret_cast<void* const*>(w); }
 
-}  // namespace amoeba
-
-using namespace amoeba;
-
-extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const amoeba_layer_weights* src,
-                                                const amoeba_layer_weights* dst, int32_t layer_begin,
-                                                int32_t layer_end, int32_t* d_status, void* cuda_stream) {
-    static_assert(sizeof(amoeba_layer_weights) == kNumTensors * sizeof(void*), "slot view of the weight struct");
-    if (!plan || !src || !dst || !d_status) return AMOEBA_ERR_INVALID_ARG;
-    const int L = plan->src.model.num_layers, a = plan->src.tp, b = plan->dst.tp;
-    if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
-    const int n_descs = (int)plan->wdev.size();
-    // Every buffer a descriptor names must be present and aligned, for every requested layer - except that a
-    // destination worker may be left out of a layer altogether (all seven pointers NULL): its shard is then not produced.
-    auto left_out = [&](int rank, int l) {
-        void* const* sl = slots(&dst[(size_t)rank * L + l]);
-        for (int t = 0; t < kNumTensors; ++t)
-            if (sl[t]) return false;
-        return true;
-    };
-    for (int l = layer_begin; l < layer_end; ++l)
-        for (const WDescDev& d : plan->wdev) {
-            const int dst_rank = d.dst_slot / kNumTensors;
-            const void* t = slots(&dst[(size_t)dst_rank * L + l])[d.dst_slot % kNumTensors];
-            if (!t && left_out(dst_rank, l)) continue;
-            const void* s = slots(&src[(size_t)(d.src_slot / kNumTensors) * L + l])[d.src_slot % kNumTensors];
-            if (!s || !t) return AMOEBA_ERR_INVALID_ARG;
-            if (reinterpret_cast<uintptr_t>(s) % 16 || reinterpret_cast<uintptr_t>(t) % 16) return AMOEBA_ERR_ALIGNMENT;
-        }
-    if (layer_begin == layer_end || n_descs == 0) return AMOEBA_OK;
-
+// Launches the copy kernel over `descs` (per-layer descriptors in kernel form, `items_per_layer` work items) for the
+// layers [layer_begin, layer_end): src is [src_tp][L], dst is [dst_tp][L] (worker-major host arrays of device pointers).
+static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDescDev>& descs, int32_t items_per_layer,
+                                  const amoeba_layer_weights* src, int src_tp, const amoeba_layer_weights* dst,
+                                  int dst_tp, int L, int layer_begin, int layer_end, int32_t* d_status,
+                                  cudaStream_t stream) {
+    const int n_descs = (int)descs.size();
+    if (layer_begin == layer_end || n_descs == 0 || items_per_layer == 0) return AMOEBA_OK;
     DeviceInfo dev;
     if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const KernelOpts& opt = plan->opt.w;
     const int path = opt.copy_path ? opt.copy_path : kWDefaults.copy_path;
     int stage_bytes = 16;
-    for (const WDescDev& d : plan->wdev)
+    for (const WDescDev& d : descs)
         stage_bytes = std::max<int64_t>(stage_bytes, (int64_t)d.rows_per_item * d.chunk_bytes);
+    const int a = src_tp, b = dst_tp;
     const int layers_per_launch = std::max(1, kMaxWeightPtrs / ((a + b) * kNumTensors));
 
     WParams p;  // large: filled per launch
     p.n_descs = n_descs;
-    p.items_per_layer = plan->items_per_layer;
+    p.items_per_layer = items_per_layer;
     p.src_tp = a;
     p.dst_tp = b;
-    for (int i = 0; i < n_descs; ++i) p.descs[i] = plan->wdev[i];
+    for (int i = 0; i < n_descs; ++i) p.descs[i] = descs[i];
     for (int l0 = layer_begin; l0 < layer_end; l0 += layers_per_launch) {
         const int nl = std::min(layers_per_launch, layer_end - l0);
         p.n_layers = nl;
@@ -163,7 +140,8 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
             e = cudaGetLastError();
         } else {
             const BulkShape bs = bulk_shape(dev, opt, kWDefaults, path, stage_bytes);
-            const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
+            const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings,
+                                                    grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
             auto kernel = path == 3 ? w_reshard_pair : w_reshard_bulk;
             e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
             if (e == cudaSuccess) {
@@ -173,6 +151,151 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
         }
         if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
         count_launch();
+    }
+    return AMOEBA_OK;
+}
+
+}  // namespace amoeba
+
+using namespace amoeba;
+
+extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const amoeba_layer_weights* src,
+                                                const amoeba_layer_weights* dst, int32_t layer_begin,
+                                                int32_t layer_end, int32_t* d_status, void* cuda_stream) {
+    static_assert(sizeof(amoeba_layer_weights) == kNumTensors * sizeof(void*), "slot view of the weight struct");
+    if (!plan || !src || !dst || !d_status) return AMOEBA_ERR_INVALID_ARG;
+    const int L = plan->src.model.num_layers, a = plan->src.tp, b = plan->dst.tp;
+    if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    // Every buffer a descriptor names must be present and aligned, for every requested layer - except that a
+    // destination worker may be left out of a layer altogether (all seven pointers NULL): its shard is then not produced.
+    auto left_out = [&](int rank, int l) {
+        void* const* sl = slots(&dst[(size_t)rank * L + l]);
+        for (int t = 0; t < kNumTensors; ++t)
+            if (sl[t]) return false;
+        return true;
+    };
+    for (int l = layer_begin; l < layer_end; ++l)
+        for (const WDescDev& d : plan->wdev) {
+            const int dst_rank = d.dst_slot / kNumTensors;
+            const void* t = slots(&dst[(size_t)dst_rank * L + l])[d.dst_slot % kNumTensors];
+            if (!t && left_out(dst_rank, l)) continue;
+            const void* s = slots(&src[(size_t)(d.src_slot / kNumTensors) * L + l])[d.src_slot % kNumTensors];
+            if (!s || !t) return AMOEBA_ERR_INVALID_ARG;
+            if (reinterpret_cast<uintptr_t>(s) % 16 || reinterpret_cast<uintptr_t>(t) % 16) return AMOEBA_ERR_ALIGNMENT;
+        }
+    return launch_descs(plan, plan->wdev, plan->items_per_layer, src, a, dst, b, L, layer_begin, layer_end, d_status,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Partial swap (Sec. 3.2, base solution): a worker of TP = a that becomes a worker of TP = N*a keeps one N-th of
+// every shard and moves it to the front of the buffer it is in, so that the rest can be released.  In place, hence
+// ordered: a phase only writes bytes whose old content an earlier phase has already moved (or that are not kept).
+//   rows (q, k, v, gate, up): one contiguous move per member; inside a fused buffer q moves first, then k, then v
+//     (the new k section may lie where the kept q rows were);
+//   columns (o_proj, down_proj): row j of the kept column range moves from j*w + keep*w/N to j*w/N; rows are done in
+//     waves [0,1), [1,N), [N,N^2), ...: the destination of wave [m, N*m) ends at byte m*w, where its sources begin.
+// Phases are separate launches on the stream; within a phase all copies are disjoint.
+extern "C" amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
+                                                        const int32_t* keep, int32_t layer_begin, int32_t layer_end,
+                                                        int32_t* d_status, void* cuda_stream) {
+    if (!plan || !bufs || !keep || !d_status) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_layout &sl = plan->src, &dl = plan->dst;
+    const amoeba_model& m = sl.model;
+    const int L = m.num_layers, a = sl.tp, b = dl.tp;
+    if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    if (b % a || sl.weight_pad_parts || dl.weight_pad_parts || sl.fused_qkv != dl.fused_qkv ||
+        sl.fused_gate_up != dl.fused_gate_up)
+        return AMOEBA_ERR_UNSUPPORTED;
+    const int N = b / a;
+    for (int r = 0; r < a; ++r)
+        if (keep[r] < 0 || keep[r] >= N) return AMOEBA_ERR_INVALID_ARG;
+    if (N == 1) return AMOEBA_OK;
+
+    enum { Q, K, V, O, GATE, UP, DOWN };
+    const int64_t e = m.elem_bytes, hid = m.hidden, rb = hid * e;
+    const int64_t rows_of[kNumTensors] = {(int64_t)m.num_q_heads * m.head_dim, (int64_t)m.num_kv_heads * m.head_dim,
+                                          (int64_t)m.num_kv_heads * m.head_dim, 0, m.intermediate, m.intermediate, 0};
+    // buffer and section offset (in rows of the old / the new shard) of every row-split member
+    int buffer_of[kNumTensors] = {Q, K, V, O, GATE, UP, DOWN};
+    int64_t sec_old[kNumTensors] = {0}, sec_new[kNumTensors] = {0};
+    if (sl.fused_qkv) {
+        buffer_of[K] = buffer_of[V] = Q;
+        sec_old[K] = rows_of[Q] / a, sec_old[V] = (rows_of[Q] + rows_of[K]) / a;
+        sec_new[K] = rows_of[Q] / b, sec_new[V] = (rows_of[Q] + rows_of[K]) / b;
+    }
+    if (sl.fused_gate_up) {
+        buffer_of[UP] = GATE;
+        sec_old[UP] = rows_of[GATE] / a, sec_new[UP] = rows_of[GATE] / b;
+    }
+    // every buffer that is touched must be there and aligned
+    for (int l = layer_begin; l < layer_end; ++l)
+        for (int r = 0; r < a; ++r)
+            for (int t = 0; t < kNumTensors; ++t) {
+                const void* ptr = slots(&bufs[(size_t)r * L + l])[buffer_of[t]];
+                if (!ptr) return AMOEBA_ERR_INVALID_ARG;
+                if (reinterpret_cast<uintptr_t>(ptr) % 16) return AMOEBA_ERR_ALIGNMENT;
+            }
+
+    std::vector<std::vector<amoeba_weight_desc>> phases;
+    auto phase = [&](size_t i) -> std::vector<amoeba_weight_desc>& {
+        if (phases.size() <= i) phases.resize(i + 1);
+        return phases[i];
+    };
+    const int chains[2][3] = {{Q, K, V}, {GATE, UP, -1}};
+    for (const auto& chain : chains)
+        for (int step = 0; step < 3 && chain[step] >= 0; ++step) {
+            const int t = chain[step];
+            for (int r = 0; r < a; ++r) {
+                amoeba_weight_desc d{};
+                d.src_rank = d.dst_rank = r;
+                d.src_tensor = d.dst_tensor = buffer_of[t];
+                d.row_bytes = rows_of[t] / b * rb;
+                d.src_off = (sec_old[t] + keep[r] * (rows_of[t] / b)) * rb;
+                d.dst_off = sec_new[t] * rb;
+                d.n_rows = 1;
+                d.src_pitch = d.dst_pitch = d.row_bytes;
+                if (d.src_off != d.dst_off) phase(step).push_back(d);
+            }
+        }
+    const int col_tensors[2] = {O, DOWN};
+    const int64_t cols_of[2] = {(int64_t)m.num_q_heads * m.head_dim, m.intermediate};
+    for (int c = 0; c < 2; ++c) {
+        const int64_t w_old = cols_of[c] / a * e, w_new = cols_of[c] / b * e;
+        int64_t lo = 0, hi = 1;
+        for (size_t wave = 0; lo < hid; ++wave) {
+            for (int r = 0; r < a; ++r) {
+                if (keep[r] == 0 && lo == 0) continue;  // row 0 of the first column range is already in place
+                amoeba_weight_desc d{};
+                d.src_rank = d.dst_rank = r;
+                d.src_tensor = d.dst_tensor = col_tensors[c];
+                d.row_bytes = w_new;
+                d.n_rows = (int32_t)(std::min(hi, hid) - lo);
+                d.src_off = lo * w_old + keep[r] * w_new;
+                d.dst_off = lo * w_new;
+                d.src_pitch = w_old;
+                d.dst_pitch = w_new;
+                phase(wave).push_back(d);
+            }
+            lo = hi;
+            hi *= N;
+        }
+    }
+
+    const int64_t cap = plan->opt.w.chunk_bytes > 0 ? plan->opt.w.chunk_bytes : kDefaultWChunk;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (const auto& ph : phases) {
+        std::vector<WDescDev> descs;
+        int64_t items = 0;
+        for (const amoeba_weight_desc& d : ph) {
+            if (d.row_bytes % 16 || d.src_off % 16 || d.dst_off % 16 || d.src_pitch % 16 || d.dst_pitch % 16)
+                return AMOEBA_ERR_ALIGNMENT;
+            descs.push_back(chunk_desc(d, cap, &items));
+            if (items > INT32_MAX || (int)descs.size() > kMaxWeightDescs) return AMOEBA_ERR_UNSUPPORTED;
+        }
+        const amoeba_status st = launch_descs(plan, descs, (int32_t)items, bufs, a, bufs, a, L, layer_begin, layer_end,
+                                              d_status, stream);
+        if (st != AMOEBA_OK) return st;
     }
     return AMOEBA_OK;
 }

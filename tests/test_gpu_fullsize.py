@@ -201,3 +201,35 @@ def test_full_size_padded_weights(oracle):
     finally:
         del s
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name,keep", [("llama3_8b_1to4", [2]), ("llama3_8b_2to8", [3, 0])])
+def test_full_size_weight_compaction_in_place(name, keep, oracle):
+    """Partial swap at the Llama-3-8B shape (4096 rows: 7 or 13 ordered waves for the column tensors, thousands of
+    concurrent work items per wave): the front of every source buffer becomes the kept worker's dense shard."""
+    import torch
+
+    import bench
+    import paper_2509_19729_b200 as A
+
+    cfg = wl.CONFIGS[name]
+    m, a, b = dict(cfg["model"]), cfg["a"], cfg["b"]
+    N = b // a
+    s, st = bench.build_session(name, torch.device("cuda:0"), layers=3, kv=False)
+    try:
+        m["L"] = 3
+        before = {l: [{n: t.cpu().numpy().view(np.uint16).reshape(oracle.shard_shapes(m, a)[n]).copy()
+                       for n, t in s.src_w[r][l].items()} for r in range(a)] for l in (0, 2)}
+        s.status.zero_()
+        A.amoeba_compact_weights_inplace(s.plan, s._src_w_packed, keep, 0, 3, s.status)
+        torch.cuda.synchronize()
+        assert int(s.status.item()) == 0
+        for l in (0, 2):
+            exp = oracle.weights_transform(before[l], m, a, b)
+            for r in range(a):
+                for n, e in exp[r * N + keep[r]].items():
+                    got = s.src_w[r][l][n].cpu().numpy().view(np.uint16)[:e.size]
+                    assert np.array_equal(got, e.reshape(-1)), (l, r, n)
+    finally:
+        del s
+        torch.cuda.empty_cache()

@@ -563,3 +563,74 @@ def test_l2_hints_on_bulk_and_tiled_copies(hint, so, do):
 
     c = make_case(GQA, 2, 4, [100, 3, 48], seed=hint, src_order=so, dst_order=do)
     check_case(c, run_case(c, PAIR, options=[(A.OPT_L2_HINT, hint)]))
+
+
+# ---- partial swap (Sec. 3.2, base solution): the kept N-th of every shard moves to the front of its buffer, in place
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("fq,fg", [(True, True), (False, False)])
+@pytest.mark.parametrize("a,b,keep", [(1, 2, [1]), (1, 4, [2]), (1, 4, [0]), (2, 4, [1, 0]), (2, 8, [3, 1]), (4, 8, [1, 0, 1, 1]),
+                                      (1, 8, [7])])
+def test_weights_compacted_in_place(path, fq, fg, a, b, keep):
+    """After the call the front of worker r's buffers is the dense TP = b shard of worker r*N + keep[r], byte for byte
+    what the oracle's a -> b transformation gives that worker."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    m = dict(L=2, hidden=96, Hq=16, Hkv=8, D=16, I=320)   # 96 rows: the waves of the column tensors end raggedly
+    N = b // a
+    dev = torch.device("cuda:0")
+    g = np.random.default_rng(a * 31 + b + sum(keep))
+    plan = A.amoeba_plan_create(A.make_layout(m, a, 4, fused_qkv=fq, fused_gate_up=fg),
+                                A.make_layout(m, b, 4, fused_qkv=fq, fused_gate_up=fg))
+    A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, path)
+    A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, 1024)
+    bufs, exp = [[None] * m["L"] for _ in range(a)], []
+    for l in range(m["L"]):
+        W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in O.logical_shapes(m).items()}
+        sa = O.weights_shard(W, m, a, fq, fg)
+        exp.append(O.weights_transform(sa, m, a, b, fq, fg))
+        for r in range(a):
+            bufs[r][l] = {n: torch.from_numpy(x.reshape(-1).view(np.uint8).copy()).to(dev) for n, x in sa[r].items()}
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    A.amoeba_compact_weights_inplace(plan, bufs, keep, 0, m["L"], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for r in range(a):
+        w = r * N + keep[r]
+        for l in range(m["L"]):
+            for n, e in exp[l][w].items():
+                got = bufs[r][l][n].cpu().numpy().view(np.uint16)[:e.size]
+                assert np.array_equal(got, e.reshape(-1)), (r, l, n)
+
+
+def test_weights_compaction_host_errors():
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    m = dict(L=1, hidden=64, Hq=8, Hkv=8, D=16, I=128)
+    dev = torch.device("cuda:0")
+    z = torch.zeros(1, dtype=torch.int32, device=dev)
+    buf = lambda lay: [[{A.TENSOR_NAMES[t]: torch.zeros(A.amoeba_layout_weight_bytes(lay, t), dtype=torch.uint8, device=dev)
+                         for t in range(7) if A.amoeba_layout_weight_bytes(lay, t)}] for _ in range(lay.tp)]
+
+    def status_of(fn):
+        with pytest.raises(A.AmoebaError) as e:
+            fn()
+        return e.value.status
+
+    src = A.make_layout(m, 2, 4)
+    plan = A.amoeba_plan_create(src, A.make_layout(m, 4, 4))
+    assert status_of(lambda: A.amoeba_compact_weights_inplace(plan, buf(src), [0, 2], 0, 1, z)) == A.ERR_INVALID_ARG
+    assert status_of(lambda: A.amoeba_compact_weights_inplace(plan, buf(src), [0, 1], 0, 2, z)) == A.ERR_INVALID_ARG
+    half = buf(src)
+    del half[1][0]["down"]
+    assert status_of(lambda: A.amoeba_compact_weights_inplace(plan, half, [0, 1], 0, 1, z)) == A.ERR_INVALID_ARG
+    for dst in (A.make_layout(m, 2, 4, weight_pad_parts=4), A.make_layout(m, 4, 4, fused_qkv=False)):
+        p2 = A.amoeba_plan_create(src, dst)
+        assert status_of(lambda: A.amoeba_compact_weights_inplace(p2, buf(src), [0, 0], 0, 1, z)) == A.ERR_UNSUPPORTED
+    p3 = A.amoeba_plan_create(A.make_layout(m, 4, 4), A.make_layout(m, 2, 4))  # scale-down is not a compaction
+    assert status_of(lambda: A.amoeba_compact_weights_inplace(p3, buf(A.make_layout(m, 4, 4)), [0] * 4, 0, 1, z)) \
+        == A.ERR_UNSUPPORTED
