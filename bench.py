@@ -272,11 +272,14 @@ def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED
     if layers is not None:
         m["L"] = layers
     st = wl.draw_merge_state(cfg, seed=seed, name=cfg_name)
-    s = MergeSession(m, cfg["N"], cfg["a"], st["NB"], cfg["S"], st["maxb"], device=device)
+    s = MergeSession(m, cfg["N"], cfg["a"], st["NB"], cfg["S"], st["maxb"], device=device,
+                     weights=bool(cfg.get("weights")))
     s.set_tables(st["seq_lens"], st["src_bt"])
     if fill:
         for i, p in enumerate(s.pools):
             wl.hash_fill_(p, seed, 300 + i)
+        for i, p in enumerate(s._wbufs):
+            wl.hash_fill_(p[:p.numel() // 8 * 8], seed, 500 + i)
     torch.cuda.synchronize()
     return s, st
 
@@ -380,7 +383,8 @@ def run_merge(args, rank, world, local):
                      (A.OPT_CTAS_PER_SM, args.ctas_per_sm)):
         if val:
             s.set_option(opt, val)
-    nbytes = s.bytes_rw(st["n_live"])
+    w_bytes = s.weight_bytes_rw()
+    nbytes = s.bytes_rw(st["n_live"]) + w_bytes
     stream = torch.cuda.current_stream()
     ev = lambda: torch.cuda.Event(enable_timing=True)
     for _ in range(args.warmup):
@@ -398,7 +402,10 @@ def run_merge(args, rank, world, local):
     torch.cuda.synchronize()
     t_begin.record(stream)
     for _ in range(args.steps):
-        m3 = [ev() for _ in range(3)]
+        m3 = [ev() for _ in range(4)]
+        m3[3].record(stream)
+        if s.inst_w:
+            s.compact_weights()
         m3[0].record(stream)
         s.merge_block_tables()
         m3[1].record(stream)
@@ -415,12 +422,13 @@ def run_merge(args, rank, world, local):
     sec = t_begin.elapsed_time(t_end) / 1e3 / args.steps
     bt_ms = statistics.mean(m3[0].elapsed_time(m3[1]) for m3 in marks)
     kv_ms = statistics.mean(m3[1].elapsed_time(m3[2]) for m3 in marks)
+    w_ms = statistics.mean(m3[3].elapsed_time(m3[0]) for m3 in marks)
     sec_all, bytes_all = aggregate(world, sec, nbytes, device)
     pool_bytes = sum(p.numel() for p in s.pools)
     if rank != 0:
         return
     peak, peak_kind = peaks()
-    kv_gbs = nbytes / (kv_ms / 1e3) / 1e9
+    kv_gbs = (nbytes - w_bytes) / (kv_ms / 1e3) / 1e9
     N, a = cfg["N"], cfg["a"]
     out = {
         "metric": METRIC, "value": bytes_all / sec_all / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -428,10 +436,10 @@ def run_merge(args, rank, world, local):
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.config, "tp": f"{N}x{a}->{N * a} in place", "layers": s.kv_layers,
                    "sequences_per_instance": cfg["S"], "live_blocks": st["n_live"], "pool_blocks": st["NB"],
-                   "block_tokens": wl.BLOCK_TOKENS, "kv_bytes_rw": nbytes, "weight_bytes_rw": 0,
-                   "pool_bytes": pool_bytes, "extra_kv_memory_bytes": 0,
+                   "block_tokens": wl.BLOCK_TOKENS, "kv_bytes_rw": nbytes - w_bytes, "weight_bytes_rw": w_bytes,
+                   "pool_bytes": pool_bytes, "extra_kv_memory_bytes": 0, "extra_weight_memory_bytes": 0,
                    "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
-        "phases_ms": {"merge_block_tables": bt_ms, "merge_kv_inplace": kv_ms},
+        "phases_ms": {"compact_weights_inplace": w_ms, "merge_block_tables": bt_ms, "merge_kv_inplace": kv_ms},
         "phases_gbs": {"merge_kv_inplace": kv_gbs},
         "roofline": {"kernel": "kv_merge_pair", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
                      "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None},

@@ -147,7 +147,7 @@ class MergeSession:
     after it.  kv_layers: layers the pools hold (None = all)."""
 
     def __init__(self, model: dict, N: int, a: int, NB: int, num_seqs: int, max_blocks_per_seq: int,
-                 kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0"):
+                 kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0", weights: bool = False):
         self.model, self.N, self.a, self.NB = model, N, a, NB
         self.device = torch.device(device)
         self.src_layout = A.make_layout(model, a, NB, block_tokens)
@@ -165,10 +165,38 @@ class MergeSession:
         per_layer = A.amoeba_layout_kv_pool_bytes(self.src_layout) // self.L
         self.pools = [torch.empty(per_layer * self.kv_layers, dtype=torch.uint8, device=self.device)
                       for _ in range(N * a)]
+        # weights: every instance holds the whole model as dense TP=a shards; instance i's worker r keeps sub-shard i
+        self.inst_w, self._inst_w_packed, self._wbufs = [], [], []
+        if weights:
+            sizes = [A.amoeba_layout_weight_bytes(self.src_layout, t) for t in range(len(A.TENSOR_NAMES))]
+            used = [(n, sz) for n, sz in zip(A.TENSOR_NAMES, sizes) if sz]
+            for _ in range(N):
+                shards = []
+                for _ in range(a):
+                    buf = torch.empty(_carved_bytes([sz for _, sz in used]) * self.L, dtype=torch.uint8,
+                                      device=self.device)
+                    views = _carve(buf, [sz for _, sz in used] * self.L)
+                    self._wbufs.append(buf)
+                    shards.append([{n: views[l * len(used) + j] for j, (n, _) in enumerate(used)}
+                                   for l in range(self.L)])
+                self.inst_w.append(shards)
+                self._inst_w_packed.append(A.pack_weights(shards))
 
     def set_tables(self, seq_lens, src_bt) -> None:
         self.seq_lens.copy_(torch.as_tensor(seq_lens, dtype=torch.int32))
         self.src_bt.copy_(torch.as_tensor(src_bt, dtype=torch.int32))
+
+    def compact_weights(self, stream=None) -> None:
+        """Every worker of every instance moves the part of its weight shards it keeps to the front, in place."""
+        for i, packed in enumerate(self._inst_w_packed):
+            A.amoeba_compact_weights_inplace(self.plan, packed, [i] * self.a, 0, self.L, self.status, stream)
+
+    def weight_bytes_rw(self) -> int:
+        """Bytes read + written by compact_weights: 1/N of every instance's weights, both ways."""
+        if not self.inst_w:
+            return 0
+        _, w = A.amoeba_plan_bytes(self.plan, 0)
+        return w  # N instances x (1/N of one model copy) x 2
 
     def merge_block_tables(self, stream=None) -> None:
         A.amoeba_merge_block_tables(self.plan, self.src_bt, self.seq_lens, self.num_seqs, self.maxb, self.dst_bt,
@@ -179,6 +207,9 @@ class MergeSession:
                                   self.kv_layers if layer_end is None else layer_end, self.status, stream)
 
     def step(self, stream=None) -> None:
+        """Weights first, then the KV cache: the order the paper gives for raising the TP degree (Sec. 3.3)."""
+        if self.inst_w:
+            self.compact_weights(stream)
         self.merge_block_tables(stream)
         self.merge_kv(stream)
 

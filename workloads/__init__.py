@@ -59,7 +59,7 @@ MERGE_CONFIGS = {
                                    lens=("uniform", 512, 8192), utilisation=0.9),
     # the same at 20 sequences per instance, so that a second set of pools (the out-of-place merge) also fits one GPU
     "llama3_8b_merge_4x1to4_s20": dict(model=_model(32, 4096, 32, 8, 128, 14336), dtype="bf16", N=4, a=1, S=20,
-                                       lens=("uniform", 512, 8192), utilisation=0.9),
+                                       lens=("uniform", 512, 8192), utilisation=0.9, weights=True),
     "tiny_merge_2x1to2": dict(model=_model(2, 256, 4, 4, 64, 1024), dtype="fp16", N=2, a=1, S=4,
                               lens=("uniform", 16, 256), utilisation=0.75),
 }
