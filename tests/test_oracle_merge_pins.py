@@ -280,3 +280,44 @@ def test_split_rejects_blocks_of_the_wrong_residue(oracle):
     old_bt, live, st = oracle.kv_split_inplace(m, T, N, a, NB, neg, bt, pools2)
     assert st == oracle.INVALID_ARG and np.all(old_bt == -1) and not live.any()
     assert all(np.array_equal(p, q) for p, q in zip(pools2, before))
+
+
+# ---------------- layer stride of the in-place merge and split ----------------
+@pytest.mark.parametrize("N,a", [(4, 1), (2, 2)])
+def test_inplace_merge_and_split_with_a_layer_stride(oracle, N, a):
+    """Pools whose layers are `stride` elements apart: layer l of the result sits at l*stride and equals layer l of
+    the dense result; the words between layers keep their values; and the split brings every live block back."""
+    m, T, NB = dict(MHA8, L=3), 4, 7
+    lens, bt, KVs, dense_pools = _instances(oracle, m, T, N, a, NB, [[5, 9, 1], [16], [3, 3, 3], [0, 7]][:N], seed=31)
+    dense = oracle.pool_elems_per_layer(m, T, a, NB)
+    stride = dense + 56
+    strided = []
+    for w, p in enumerate(dense_pools):
+        q = np.full(m["L"] * stride, 0x7000 + w, np.uint16)
+        q.reshape(m["L"], stride)[:, :dense] = p.reshape(m["L"], dense)
+        strided.append(q)
+    first = [q.copy() for q in strided]
+    bt_d, live_d, st = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, dense_pools)
+    assert st == 0
+    bt_s, live_s, st = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, strided, layer_stride=stride)
+    assert st == 0 and np.array_equal(bt_s, bt_d) and np.array_equal(live_s, live_d)
+    for w in range(N * a):
+        v = strided[w].reshape(m["L"], stride)
+        assert np.array_equal(v[:, :dense], dense_pools[w].reshape(m["L"], dense))
+        assert np.all(v[:, dense:] == 0x7000 + w)
+    # every instance's logical KV can be read back from the strided merged pools through the independent reconstruct
+    merged = _merged_order(strided, N, a)
+    for i in range(N):
+        back = oracle.kv_reconstruct(merged, m, T, N * a, NB * N, lens[i], bt_s[i], layer_stride=stride)
+        assert np.array_equal(back, KVs[i])
+    old_bt, _, st = oracle.kv_split_inplace(m, T, N, a, NB, lens, bt_s, strided, layer_stride=stride)
+    assert st == 0 and np.array_equal(old_bt, bt)
+    per_block = (m["Hkv"] // a) * 2 * T * m["D"]
+    for i in range(N):
+        for r in range(a):
+            now = strided[i * a + r].reshape(m["L"], stride)
+            was = first[i * a + r].reshape(m["L"], stride)
+            live = live_d[i] != 0
+            assert np.array_equal(now[:, :dense].reshape(m["L"], NB, per_block)[:, live],
+                                  was[:, :dense].reshape(m["L"], NB, per_block)[:, live])
+            assert np.array_equal(now[:, dense:], was[:, dense:])

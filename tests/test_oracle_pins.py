@@ -513,3 +513,70 @@ def test_decode_attention_from_token_first_strides(oracle):
         K1, V1 = (np.ascontiguousarray(a_tf[c].reshape(-1, m["D"])[:n]) for c in (0, 1))
         K2, V2 = (np.ascontiguousarray(a_hc[:, c].reshape(-1, m["D"])[:n]) for c in (0, 1))
         assert np.array_equal(attend(K1, V1).view(np.uint32), attend(K2, V2).view(np.uint32))
+
+
+# ---------------- layer stride: layers further apart than one dense layer (every layer has its own block array) -------
+def _strided_views(pool, L, stride, dense):
+    v = pool.reshape(L, stride)
+    return v[:, :dense], v[:, dense:]
+
+
+@pytest.mark.parametrize("order", [0, 1])
+@pytest.mark.parametrize("TP", [1, 2, 4])
+def test_layer_stride_places_layer_l_at_l_times_stride(oracle, TP, order):
+    """A pool whose layers are `stride` elements apart holds, at l*stride, exactly what the dense pool holds at
+    l*dense, and the words between two layers are never written (nor read back)."""
+    m, T, NB = dict(SMALL, L=3), 4, 7
+    seq_lens = [5, 0, 9, 4]
+    bt, nblk = _state(seq_lens, T, NB)
+    G = int(nblk.sum()) * T
+    KV = np.random.default_rng(21).integers(0, 65536, size=(m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    dense = oracle.pool_elems_per_layer(m, T, TP, NB)
+    gap = 24
+    stride = dense + gap
+    FILL = 0xBEEF
+    ref = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=FILL, order=order)
+    got = oracle.kv_shard(KV, m, T, TP, NB, seq_lens, bt, fill=FILL, order=order, layer_stride=stride)
+    for r in range(TP):
+        assert got[r].size == m["L"] * stride
+        body, between = _strided_views(got[r], m["L"], stride, dense)
+        assert np.array_equal(body, ref[r].reshape(m["L"], dense))
+        assert np.all(between == FILL)
+    # the inverse reads the same places: poison the gaps, the logical state must not change
+    for r in range(TP):
+        _strided_views(got[r], m["L"], stride, dense)[1][:] = 0x0BAD
+    assert np.array_equal(oracle.kv_reconstruct(got, m, T, TP, NB, seq_lens, bt, order=order, layer_stride=stride), KV)
+    # a stride counted in the wrong unit (bytes instead of elements) would land layer 1 elsewhere: the stamp of the
+    # first word of layer 1 sits at element `stride`, not at 2*stride or stride/2
+    l1 = oracle.kv_shard(KV[:2], dict(m, L=2), T, TP, NB, seq_lens, bt, fill=FILL, order=order, layer_stride=stride)
+    for r in range(TP):
+        assert np.array_equal(l1[r][stride:stride + dense], ref[r][dense:2 * dense])
+
+
+@pytest.mark.parametrize("a,b,so,do", [(1, 4, 0, 0), (4, 2, 0, 0), (2, 4, 1, 0), (2, 1, 0, 1)])
+def test_transform_with_layer_strides_equals_dense_transform(oracle, a, b, so, do):
+    m, T = dict(SMALL, L=3), 4
+    seq_lens = [9, 4, 0, 13, 2]
+    NB_a, NB_b = 10, 13
+    bt_a, nblk = _state(seq_lens, T, NB_a, seed=7)
+    G = int(nblk.sum()) * T
+    KV = np.random.default_rng(22).integers(0, 65536, size=(m["L"], G, m["Hkv"], 2, m["D"]), dtype=np.uint16)
+    da, db = oracle.pool_elems_per_layer(m, T, a, NB_a), oracle.pool_elems_per_layer(m, T, b, NB_b)
+    sa, sb = da + 40, db + 8
+    free_b = np.random.default_rng(3).permutation(NB_b).astype(np.int32)
+    bt_b, *_ = oracle.assign_blocks(seq_lens, T, bt_a, NB_a, NB_b, free_list=free_b)
+    src_d = oracle.kv_shard(KV, m, T, a, NB_a, seq_lens, bt_a, order=so)
+    src_s = oracle.kv_shard(KV, m, T, a, NB_a, seq_lens, bt_a, order=so, layer_stride=sa, fill=0x1111)
+    dst_d = [np.full(m["L"] * db, 0xA5A5, np.uint16) for _ in range(b)]
+    dst_s = [np.full(m["L"] * sb, 0xA5A5, np.uint16) for _ in range(b)]
+    oracle.kv_transform(m, T, seq_lens, a, NB_a, bt_a, src_d, b, NB_b, bt_b, dst_d, src_order=so, dst_order=do)
+    oracle.kv_transform(m, T, seq_lens, a, NB_a, bt_a, src_s, b, NB_b, bt_b, dst_s, src_order=so, dst_order=do,
+                        src_layer_stride=sa, dst_layer_stride=sb)
+    for r in range(b):
+        body, between = _strided_views(dst_s[r], m["L"], sb, db)
+        assert np.array_equal(body, dst_d[r].reshape(m["L"], db))
+        assert np.all(between == 0xA5A5)
+    # and it is the direct shard of the logical state at that stride
+    direct = oracle.kv_shard(KV, m, T, b, NB_b, seq_lens, bt_b, order=do, layer_stride=sb, fill=0xA5A5)
+    for x, y in zip(dst_s, direct):
+        assert np.array_equal(x, y)
