@@ -368,3 +368,29 @@ def weights_transform_any(src_shards, m, a, b, fused_qkv=True, fused_gate_up=Tru
         sh = _wstruct(out[r])
         lib().oracle_weights_shard(C.byref(mm), b, r, int(fused_qkv), int(fused_gate_up), C.byref(lg), C.byref(sh))
     return out
+
+
+# ---- Sec. 3.1, Improvement 1: in-place block reshaping of one instance ------------------------------------------
+def kv_reshape_inplace(direction, m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride=None, pairs_cap=None):
+    """One instance, in place: ``direction`` "split" (TP=a -> TP=N*a, table over NB ids) or "merge" (TP=N*a -> TP=a,
+    table over NB*N ids).  pools: list of N*a uint16 arrays, pools[w] = worker w of the TP=N*a side, worker r of the
+    TP=a side is pools[r*N]; NB = blocks per layer of the TP=a side.  Rewrites the pools in place and returns
+    (new_bt, pairs[n,2], n, free_mask, free_count, status)."""
+    assert direction in ("split", "merge")
+    sl, slp = _i32(seq_lens)
+    b, bp = _i32(bt)
+    assert b.ndim == 2 and b.shape[0] == len(sl) and len(pools) == N * a
+    S, maxb = b.shape
+    stride = pool_elems_per_layer(m, T, a, NB) if layer_stride is None else layer_stride
+    if pairs_cap is None:
+        pairs_cap = S * maxb
+    new_bt = np.empty_like(b)
+    pairs = np.full((max(pairs_cap, 1), 2), -7, dtype=np.int32)
+    free_mask = np.empty(NB * N if direction == "split" else NB, dtype=np.uint8)
+    n, left, st = C.c_int32(0), C.c_int32(0), C.c_int32(status)
+    mm = _model(m)
+    f = lib().oracle_kv_reshape_split if direction == "split" else lib().oracle_kv_reshape_merge
+    f(C.byref(mm), T, N, a, NB, C.c_int64(stride), S, slp, maxb, bp, _ptr_array(pools),
+      new_bt.ctypes.data_as(C.POINTER(C.c_int32)), pairs.ctypes.data_as(C.POINTER(C.c_int32)), pairs_cap,
+      C.byref(n), free_mask.ctypes.data_as(C.POINTER(C.c_uint8)), C.byref(left), C.byref(st))
+    return new_bt, pairs[:n.value].copy(), n.value, free_mask, left.value, st.value

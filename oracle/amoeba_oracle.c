@@ -570,3 +570,128 @@ void oracle_kv_split_inplace(const oracle_model* m, int T, int N, int a, int NB,
     for (int w = 0; w < N * a; ++w) free(old[w]);
     free(old);
 }
+
+
+/*
+ * In-place block reshaping of ONE instance (Sec. 3.1, "Improvement 1": a worker retains the headers the new TP degree
+ * assigns to it where they are, and the room the migrated headers leave inside a block is reused by reshaping the
+ * block into smaller blocks).  TP = a becomes TP = N*a (split) or TP = N*a becomes TP = a (merge back).
+ *
+ * Reading (the paper names no numbering): the header ranges are contiguous, so old worker r (0-indexed) of TP = a
+ * holds exactly the headers of workers r*N .. r*N+N-1 of TP = N*a; it becomes worker r*N, the one whose headers are
+ * the first N-th of each of its blocks.  Its pool of NB blocks of Hkv/a headers is re-read as NB*N blocks of
+ * Hkv/(N*a) headers, and old block p becomes new block p*N ON EVERY WORKER (the block table stays shared): on worker
+ * r*N that is the same memory, so the retained headers do not move; the headers of group k = 1..N-1 go to block p*N of
+ * worker r*N+k, whose pool (same capacity, NB*N blocks) is fresh.  Afterwards every id that is not p*N for a live p is
+ * free - in particular the ids p*N+1 .. p*N+N-1, which on worker r*N are the segments the migrated headers left.
+ *
+ * pools[w], w = 0 .. N*a-1, is the pool of worker w of the TP = N*a side; worker r of the TP = a side is pools[r*N].
+ * Both views use layer_stride elements between layers.
+ *
+ * split (dir = 0)  in : seq_lens[S], bt[S][maxb] over NB ids.   out: new_bt (p -> p*N), free_mask[NB*N].
+ * merge (dir = 1)  in : bt over NB*N ids; only ids = 0 (mod N) can be reshaped back (the caller first renumbers other
+ *                       blocks with the ordinary block-table rewrite and a free list of such ids whose N-1 followers
+ *                       are free).                              out: new_bt (q -> q/N), free_mask[NB].
+ * Both: pairs[k] = (old id, new id) of the k-th block in (sequence, logical block) order, (-1,-1) for a block that
+ * is not moved; *num_pairs; *free_count = number of set bytes of free_mask (1 = free).
+ *
+ * Every word is read from a snapshot of the pools taken before anything moves and written through its logical
+ * coordinates (block, token, header, K/V, dim); a word whose new place is its old place is written with the value
+ * it has.  Words of blocks no table names, and the segments the migrated headers leave, are never written.
+ *
+ * Errors.  Whole call (nothing moves; new_bt all -1, no pairs, free_mask all 1): a negative length, a sequence
+ * longer than maxb blocks, or more blocks than pairs_cap -> INVALID_ARG.  Per block -> BAD_BLOCK_ID, table entry -1,
+ * pair (-1,-1), block not moved: an id outside the pool, -1 inside a sequence, an id named a second time, and for the
+ * merge an id that is not a multiple of N.  status is sticky.
+ */
+static void kv_reshape_inplace(int dir, const oracle_model* m, int T, int N, int a, int NB, int64_t layer_stride,
+                               int S, const int32_t* seq_lens, int maxb, const int32_t* bt, uint16_t* const* pools,
+                               int32_t* new_bt, int32_t* pairs, int pairs_cap, int32_t* num_pairs,
+                               uint8_t* free_mask, int32_t* free_count, int32_t* status) {
+    const int TPn = N * a, Ha = m->Hkv / a, Hn = m->Hkv / TPn;
+    const int64_t NBn = (int64_t)NB * N;                 /* blocks of the TP = N*a side */
+    const int64_t ids_in = dir == 0 ? NB : NBn, ids_out = dir == 0 ? NBn : NB;
+    const int64_t pool_elems = (int64_t)m->L * layer_stride;
+    for (int64_t k = 0; k < (int64_t)S * maxb; ++k) new_bt[k] = -1;
+    for (int64_t k = 0; k < ids_out; ++k) free_mask[k] = 1;
+    *num_pairs = 0;
+    *free_count = (int32_t)ids_out;
+    int64_t total = 0;
+    int err = ORACLE_OK;
+    for (int s = 0; s < S; ++s) {
+        if (seq_lens[s] < 0 || blocks_of(seq_lens[s], T) > maxb) err = ORACLE_INVALID_ARG;
+        else total += blocks_of(seq_lens[s], T);
+    }
+    if (err == ORACLE_OK && total > pairs_cap) err = ORACLE_INVALID_ARG;
+    if (err != ORACLE_OK) {
+        if (*status == 0) *status = err;
+        return;
+    }
+    uint16_t** old = (uint16_t**)malloc(sizeof(uint16_t*) * (size_t)TPn);
+    for (int w = 0; w < TPn; ++w) {
+        old[w] = (uint16_t*)malloc((size_t)(pool_elems > 0 ? pool_elems : 1) * sizeof(uint16_t));
+        memcpy(old[w], pools[w], (size_t)pool_elems * sizeof(uint16_t));
+    }
+    int64_t k = 0, n_live = 0;
+    for (int s = 0; s < S; ++s)
+        for (int64_t j = 0; j < blocks_of(seq_lens[s], T); ++j, ++k) {
+            const int64_t e = (int64_t)s * maxb + j;
+            const int64_t id = bt[e];
+            pairs[2 * k] = pairs[2 * k + 1] = -1;
+            int ok = id >= 0 && id < ids_in && (dir == 0 || id % N == 0);
+            const int64_t nid = dir == 0 ? id * N : id / N;
+            if (ok && !free_mask[nid]) ok = 0; /* named a second time */
+            if (!ok) {
+                if (*status == 0) *status = ORACLE_BAD_BLOCK_ID;
+                continue;
+            }
+            new_bt[e] = (int32_t)nid;
+            pairs[2 * k] = (int32_t)id;
+            pairs[2 * k + 1] = (int32_t)nid;
+            free_mask[nid] = 0;
+            ++n_live;
+            const int64_t blk_a = dir == 0 ? id : nid;  /* the block's id on the TP = a side */
+            const int64_t blk_n = dir == 0 ? nid : id;  /* ... and on the TP = N*a side */
+            for (int l = 0; l < m->L; ++l)
+                for (int header = 1; header <= m->Hkv; ++header) {
+                    const int wa = oracle_worker_of_header(m->Hkv, a, header);   /* 1-indexed worker at TP = a */
+                    const int wn = oracle_worker_of_header(m->Hkv, TPn, header); /* ... at TP = N*a */
+                    int fa, fn, last;
+                    oracle_header_range(m->Hkv, a, wa, &fa, &last);
+                    oracle_header_range(m->Hkv, TPn, wn, &fn, &last);
+                    const int mem_a = (wa - 1) * N; /* whose memory the TP = a worker lives in */
+                    const int mem_n = wn - 1;
+                    const int64_t lo = (int64_t)l * layer_stride;
+                    for (int c = 0; c < 2; ++c)
+                        for (int tok = 0; tok < T; ++tok)
+                            for (int d = 0; d < m->D; ++d) {
+                                const int64_t oa = lo + pool_offset(ORACLE_HEADER_CENTRIC, NB, Ha, T, m->D, blk_a,
+                                                                    header - fa, c, tok, d);
+                                const int64_t on = lo + pool_offset(ORACLE_HEADER_CENTRIC, NBn, Hn, T, m->D, blk_n,
+                                                                    header - fn, c, tok, d);
+                                if (dir == 0) pools[mem_n][on] = old[mem_a][oa];
+                                else pools[mem_a][oa] = old[mem_n][on];
+                            }
+                }
+        }
+    *num_pairs = (int32_t)k;
+    *free_count = (int32_t)(ids_out - n_live);
+    for (int w = 0; w < TPn; ++w) free(old[w]);
+    free(old);
+}
+
+void oracle_kv_reshape_split(const oracle_model* m, int T, int N, int a, int NB, int64_t layer_stride, int S,
+                             const int32_t* seq_lens, int maxb, const int32_t* bt, uint16_t* const* pools,
+                             int32_t* new_bt, int32_t* pairs, int pairs_cap, int32_t* num_pairs, uint8_t* free_mask,
+                             int32_t* free_count, int32_t* status) {
+    kv_reshape_inplace(0, m, T, N, a, NB, layer_stride, S, seq_lens, maxb, bt, pools, new_bt, pairs, pairs_cap,
+                       num_pairs, free_mask, free_count, status);
+}
+
+void oracle_kv_reshape_merge(const oracle_model* m, int T, int N, int a, int NB, int64_t layer_stride, int S,
+                             const int32_t* seq_lens, int maxb, const int32_t* bt, uint16_t* const* pools,
+                             int32_t* new_bt, int32_t* pairs, int pairs_cap, int32_t* num_pairs, uint8_t* free_mask,
+                             int32_t* free_count, int32_t* status) {
+    kv_reshape_inplace(1, m, T, N, a, NB, layer_stride, S, seq_lens, maxb, bt, pools, new_bt, pairs, pairs_cap,
+                       num_pairs, free_mask, free_count, status);
+}
