@@ -18,7 +18,9 @@
  *   - Every data pointer is a DEVICE pointer unless its name starts with h_ or the comment says "host array".
  *     The caller owns every buffer and the stream; the library owns only the plan object.
  *   - Data calls are asynchronous on the given stream (a cudaStream_t passed as void*; NULL = default stream),
- *     never synchronise, never allocate, and are out of place: destination buffers must not overlap sources.
+ *     never synchronise and never allocate device memory.  amoeba_reshard_kv and amoeba_reshard_weights are out of
+ *     place: a destination buffer that is also a source buffer is refused (INVALID_ARG), and partial overlaps are
+ *     the caller's to avoid.  The calls whose names end in _inplace work on the buffers they are given.
  *   - Errors the host can see return a code and launch nothing.  Errors only the device can see (bad block ids,
  *     not enough free blocks) are written to *d_status: an int32 the caller zeroes beforehand; the first non-zero
  *     code sticks, offending items are skipped, the kernel never traps.
@@ -26,8 +28,15 @@
  *     written.  Every other destination byte keeps its value.
  *   - Block ids are int32; byte offsets are 64-bit.  Pointers, run lengths and pitches must be multiples of 16 B
  *     (checked: AMOEBA_ERR_ALIGNMENT).
- *   - Thread-compatible: no global mutable state besides an atomic launch counter; a plan may be used from several threads if its options are not
- *     changed concurrently.  No C++ exception crosses this boundary.
+ *   - Thread-compatible.  Process-wide state is limited to an atomic launch counter and a few lock-protected
+ *     look-up caches (device attributes, the shared-memory opt-in of each kernel, the driver's tensor-map encoder,
+ *     the built-in scratch address per device); a plan also caches the tensor maps it encoded for the last set of
+ *     pool addresses.  A plan may be used from several threads if its options are not changed concurrently.
+ *     No C++ exception crosses this boundary (a failed host allocation is AMOEBA_ERR_NO_MEMORY).
+ *   - AMOEBA_ERR_TIMEOUT: every on-device wait of a kernel on one of its own bulk copies is bounded.  A kernel whose
+ *     wait runs out records the code in *d_status, waits (bounded again) for the copies it still has in flight and
+ *     returns; the CUDA context stays usable, the destination holds a mix of copied and untouched items, and the
+ *     call can simply be issued again.
  */
 #ifndef AMOEBA_H_
 #define AMOEBA_H_
@@ -49,7 +58,8 @@ typedef enum {
     AMOEBA_ERR_BAD_BLOCK_ID = 5,   /* a block id outside its pool (or -1 inside a sequence) */
     AMOEBA_ERR_CUDA = 6,           /* a CUDA runtime call failed (launch error, no device) */
     AMOEBA_ERR_TIMEOUT = 7,        /* a bounded on-device wait on the kernel's own bulk copy ran out */
-    AMOEBA_ERR_TOO_LARGE = 8       /* the problem needs more scratch than the library's built-in scratch array holds */
+    AMOEBA_ERR_TOO_LARGE = 8,      /* the problem needs more scratch than the library's built-in scratch array holds */
+    AMOEBA_ERR_NO_MEMORY = 9       /* a host allocation inside the library failed */
 } amoeba_status;
 
 /* Storage order of one layer of a worker's KV pool (Sec. 3.1).  HEAD_MAJOR is the paper's header-centric layout
@@ -170,6 +180,9 @@ enum {
                                    so a cap below the SM count leaves SMs to kernels running on other streams - the
                                    paper starts its migration on a side stream once enough SMs are free (Sec. 3.1,
                                    Improvement 2) */
+    AMOEBA_OPT_WAIT_TRIES = 9,  /* bulk-copy paths: a kernel's wait on one of its own copies gives up after this many
+                                   non-blocking polls and reports AMOEBA_ERR_TIMEOUT (0 = the default, generous budget).
+                                   For tests of the give-up path; a small value makes healthy copies time out. */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };
@@ -192,12 +205,14 @@ AMOEBA_API amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t optio
  *     d_num_pairs, d_dst_free_count_out  int32 scalars: number of pairs, free blocks left
  *     d_status   int32 scalar, sticky (see conventions)
  * d_workspace: scratch of at least amoeba_rewrite_workspace_bytes(...) bytes, 16-byte aligned, contents irrelevant
- *     before and after; calls that overlap on the GPU need separate workspaces.
+ *     before and after; calls that overlap on the GPU need separate workspaces.  Its size depends on num_seqs and on
+ *     the plan's block counts (n_free_or_nb is only range-checked).
  *
  * Device-detected errors.  Whole call (d_dst_bt all -1, 0 pairs, free count unchanged): a negative length or a
  * sequence needing more than max_blocks_per_seq blocks, or more blocks than pairs_cap -> INVALID_ARG; more blocks
- * than free blocks -> NO_FREE_BLOCKS.  Per block -> BAD_BLOCK_ID: a free id outside [0, dst num_blocks) gives table
- * entry -1 and pair (-1,-1); a source id outside [0, src num_blocks) keeps the table entry, pair (-1,-1).
+ * than free blocks -> NO_FREE_BLOCKS.  Per block -> BAD_BLOCK_ID: a free id outside [0, dst num_blocks), or one that
+ * an earlier block (in sequence, block order) of this call was already given - a free list that names an id twice -
+ * gives table entry -1 and pair (-1,-1); a source id outside [0, src num_blocks) keeps the table entry, pair (-1,-1).
  * Host-detected: INVALID_ARG (null pointers, negative sizes, both or neither free form), ALIGNMENT, CUDA.
  */
 AMOEBA_API amoeba_status amoeba_rewrite_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs, int32_t n_free_or_nb,
@@ -222,13 +237,16 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
  * performs no cudaMalloc / cudaFree and calls no allocating routine of any library.
  *
  * Limit: the scratch array is AMOEBA_BUILTIN_SCRATCH_BYTES (1 MiB) per GPU, held by every GPU that loads the library
- * until the process exits.  It must cover amoeba_rewrite_workspace_bytes(num_seqs, n_free_or_nb), i.e. roughly
- * num_seqs + n_free_or_nb <= 262 000 table entries; larger problems are refused with AMOEBA_ERR_TOO_LARGE and
- * nothing is launched - use amoeba_rewrite_block_tables with your own workspace for those.
+ * until the process exits.  It must cover amoeba_rewrite_workspace_bytes(...), i.e. roughly num_seqs + the larger of
+ * the plan's two block counts <= 262 000 entries, in either free-block form; larger problems are refused with
+ * AMOEBA_ERR_TOO_LARGE and nothing is launched - use amoeba_rewrite_block_tables with your own workspace for those.
  *
  * First use on a device: the first call made while a given device is current looks up that device's address of the
- * array (one cudaGetSymbolAddress, checked; AMOEBA_ERR_CUDA if it fails) and remembers it.  Make that first call
- * during start-up, outside any stream capture; later calls on the device only launch the two kernels.
+ * array (one cudaGetSymbolAddress, checked; AMOEBA_ERR_CUDA if it fails, with the runtime's error state cleared) and
+ * remembers it per device ordinal (up to 64 ordinals; beyond that AMOEBA_ERR_UNSUPPORTED).  Make that first call
+ * during start-up, outside any stream capture; later calls on the device only launch the kernels.  The remembered
+ * address is the one of the device's primary context at that time: after a cudaDeviceReset of the device it is
+ * stale, so a process that resets a device must not use this entry point on it afterwards.
  *
  * Sharing: all calls on one GPU use the same array, and it keeps whatever the previous call left in it.  Nothing in
  * it has to start at zero (the kernels write every word before reading it), so no clearing is needed; but two calls
@@ -257,6 +275,48 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
 AMOEBA_API amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools, void* const* dst_pools,
                                 const int32_t* d_pairs, const int32_t* d_num_pairs, int32_t pairs_cap,
                                 int32_t layer_begin, int32_t layer_end, int32_t* d_status, void* cuda_stream);
+
+/*
+ * In-place block reshaping of ONE instance  (Sec. 3.1, "Improvement 1": a worker retains the headers the new TP degree
+ * gives it where they are; the room the migrated headers leave inside a block is reused by reshaping the block)
+ *
+ * Split: the plan's source layout is the instance at TP = a with NB blocks, the destination layout the same instance
+ * at TP = N*a with NB*N blocks; merge back: the other way round (source TP = N*a with NB*N blocks, destination TP = a
+ * with NB).  Both header-centric, same layer stride; anything else is UNSUPPORTED.  The header ranges are contiguous,
+ * so worker r of TP = a holds the headers of workers r*N .. r*N+N-1 of TP = N*a; the paper names no numbering and
+ * this one is used: worker r becomes worker r*N, and block p becomes block p*N on every worker (the block table stays
+ * shared).  In worker r's memory, read as NB*N blocks of Hkv/(N*a) headers, block p*N is exactly the retained N-th
+ * of old block p: it does not move.  The other N-1 header groups go to block p*N of workers r*N+1 .. r*N+N-1, whose
+ * pools have the same capacity and are otherwise untouched.  Afterwards every id that is not p*N for a live p is
+ * free - the ids p*N+1 .. p*N+N-1 are the segments the migrated headers left.  (N-1)/N of the live bytes move and
+ * the retained workers need no second pool.  The merge back brings the groups home: only blocks whose id is a
+ * multiple of N can be reshaped (the caller first renumbers other blocks with amoeba_rewrite_block_tables /
+ * amoeba_reshard_kv inside the TP = N*a pools, using free ids q = 0 mod N whose followers q+1 .. q+N-1 are free too).
+ *
+ * amoeba_reshape_block_tables: same inputs as amoeba_rewrite_block_tables without a free list.  Writes d_dst_bt
+ * (p -> p*N, or q -> q/N; -1 past each sequence's blocks), the pair list (old id, new id) in (sequence, block) order,
+ * d_dst_free_mask_out: uint8 [destination num_blocks], 1 = free afterwards, and the free count.  Workspace as for
+ * amoeba_rewrite_block_tables.  Device-detected errors: whole call as there (no NO_FREE_BLOCKS); per block ->
+ * BAD_BLOCK_ID, table entry -1, pair (-1,-1), block not moved: an id outside the source pool, -1 inside a sequence,
+ * an id an earlier block already named, and for the merge an id that is not a multiple of N.
+ *
+ * amoeba_reshape_kv_inplace: pools is a HOST array of N*a device pointers, pools[w] = worker w of the TP = N*a side;
+ * worker r of the TP = a side is pools[r*N].  All distinct.  For every pair (both ids >= 0), layer and header group
+ * k = 1 .. N-1 the group's bytes are copied between pools[r*N] and pools[r*N+k]; nothing is written into a pool
+ * that the same call reads (split: the old workers are only read; merge: they are only written), so no ordering
+ * between work items is needed.  A pair whose ids are not (p, p*N) resp. (q, q/N) is skipped with BAD_BLOCK_ID.
+ * All three copy paths apply.  amoeba_reshape_bytes: bytes read + written for n_live_blocks blocks over all layers.
+ */
+AMOEBA_API amoeba_status amoeba_reshape_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
+                                          const int32_t* d_seq_lens, int32_t num_seqs, int32_t max_blocks_per_seq,
+                                          int32_t* d_dst_bt, int32_t* d_pairs, int32_t pairs_cap, int32_t* d_num_pairs,
+                                          uint8_t* d_dst_free_mask_out, int32_t* d_dst_free_count_out,
+                                          int32_t* d_status, void* d_workspace, int64_t workspace_bytes,
+                                          void* cuda_stream);
+AMOEBA_API amoeba_status amoeba_reshape_kv_inplace(const amoeba_plan* plan, void* const* pools, const int32_t* d_pairs,
+                                        const int32_t* d_num_pairs, int32_t pairs_cap, int32_t layer_begin,
+                                        int32_t layer_end, int32_t* d_status, void* cuda_stream);
+AMOEBA_API amoeba_status amoeba_reshape_bytes(const amoeba_plan* plan, int64_t n_live_blocks, int64_t* kv_bytes_rw);
 
 /*
  * In-place merge of N instances of TP = a into one instance of TP = N*a  (Sec. 3.1, "Improvement 1": in-place

@@ -259,7 +259,9 @@ int oracle_weights_transform(const oracle_model* m, int fused_qkv, int fused_gat
  * Whole-call errors (nothing is assigned: dst_bt all -1, N = 0, free count unchanged):
  *   a negative length or a sequence longer than maxb blocks -> INVALID_ARG; more blocks than pairs_cap ->
  *   INVALID_ARG; more blocks than free blocks -> NO_FREE_BLOCKS (checked in this order).
- * Per-block errors -> BAD_BLOCK_ID: a free-list id outside [0, NB_dst) gives dst_bt entry -1 and pair (-1,-1);
+ * Per-block errors -> BAD_BLOCK_ID: a free-list id outside [0, NB_dst), or one that an earlier block of this walk
+ *   has already taken (a list that names an id twice: two blocks must never share a destination), gives dst_bt
+ *   entry -1 and pair (-1,-1);
  *   a source id outside [0, NB_src) keeps the dst_bt entry but gives pair (-1,-1), so nothing is copied for it.
  * status is sticky: it is only written while it still holds 0.
  */
@@ -293,12 +295,15 @@ void oracle_assign_blocks(int S, const int32_t* seq_lens, int T, const int32_t* 
         return;
     }
 
+    uint8_t* taken = (uint8_t*)calloc((size_t)(NB_dst > 0 ? NB_dst : 1), 1);
     int64_t k = 0;
     for (int s = 0; s < S; ++s) {
         for (int64_t i = 0; i < blocks_of(seq_lens[s], T); ++i) {
             const int32_t src = src_bt[(int64_t)s * maxb + i];
             const int32_t dst = ordered[k];
-            const int dst_ok = dst >= 0 && dst < NB_dst;
+            int dst_ok = dst >= 0 && dst < NB_dst;
+            if (dst_ok && taken[dst]) dst_ok = 0;
+            if (dst_ok) taken[dst] = 1;
             const int src_ok = src >= 0 && src < NB_src;
             dst_bt[(int64_t)s * maxb + i] = dst_ok ? dst : -1;
             pairs[2 * k + 0] = (dst_ok && src_ok) ? src : -1;
@@ -309,6 +314,7 @@ void oracle_assign_blocks(int S, const int32_t* seq_lens, int T, const int32_t* 
     }
     *num_pairs = (int32_t)k;
     *free_count_out = (int32_t)(n_free - k);
+    free(taken);
     free(ordered);
 }
 

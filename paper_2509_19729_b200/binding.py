@@ -21,14 +21,16 @@ __all__ = [
 ]
 
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NO_FREE_BLOCKS, ERR_BAD_BLOCK_ID, ERR_CUDA, ERR_TIMEOUT,
- ERR_TOO_LARGE) = range(9)
+ ERR_TOO_LARGE, ERR_NO_MEMORY) = range(10)
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS", "BAD_BLOCK_ID", "CUDA", "TIMEOUT",
-                "TOO_LARGE"]
+                "TOO_LARGE", "NO_MEMORY"]
 BUILTIN_SCRATCH_BYTES = 1 << 20
 __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
-            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "BUILTIN_SCRATCH_BYTES",
-            "amoeba_rewrite_block_tables_builtin_scratch"]
-OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS, OPT_MAX_CTAS = range(9)
+            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "ERR_NO_MEMORY", "BUILTIN_SCRATCH_BYTES", "OPT_WAIT_TRIES",
+            "amoeba_rewrite_block_tables_builtin_scratch", "amoeba_reshape_block_tables", "amoeba_reshape_kv_inplace",
+            "amoeba_reshape_bytes"]
+(OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS,
+ OPT_MAX_CTAS, OPT_WAIT_TRIES) = range(10)
 OPT_WEIGHTS_ONLY, OPT_KV_ONLY = 16, 32  # add to an option id to set one kernel only
 COPY_PATH_LDST, COPY_PATH_BULK, COPY_PATH_PAIR = 1, 2, 3
 KV_HEAD_MAJOR, KV_TOKEN_MAJOR = 0, 1  # [block][header][K/V][token][dim] / [K/V][block][token][header][dim]
@@ -108,6 +110,9 @@ def _load():
         "amoeba_rewrite_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP, I64, VP]),
         "amoeba_rewrite_block_tables_builtin_scratch": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, I32, VP, VP, VP, VP]),
         "amoeba_reshard_kv": (I32, [VP, P(VP), P(VP), VP, VP, I32, I32, I32, VP, VP]),
+        "amoeba_reshape_block_tables": (I32, [VP, VP, VP, I32, I32, VP, VP, I32, VP, VP, VP, VP, VP, I64, VP]),
+        "amoeba_reshape_kv_inplace": (I32, [VP, P(VP), VP, VP, I32, I32, I32, VP, VP]),
+        "amoeba_reshape_bytes": (I32, [VP, I64, P(I64)]),
         "amoeba_reshard_weights": (I32, [VP, P(LayerWeights), P(LayerWeights), I32, I32, VP, VP]),
         "amoeba_merge_live_bytes": (I32, [VP, P(I64)]),
         "amoeba_merge_bytes": (I32, [VP, I64, P(I64)]),
@@ -273,6 +278,32 @@ def amoeba_reshard_kv(plan: Plan, src_pools: Sequence, dst_pools: Sequence, pair
         raise AmoebaError(ERR_INVALID_ARG, "amoeba_reshard_kv (pool count != tp)")
     _check(_load().amoeba_reshard_kv(plan.handle, sp, dp, _ptr(pairs), _ptr(num_pairs), pairs_cap, layer_begin,
                                      layer_end, _ptr(status), _stream(stream)), "amoeba_reshard_kv")
+
+
+def amoeba_reshape_block_tables(plan: Plan, src_bt, seq_lens, num_seqs: int, max_blocks_per_seq: int, dst_bt, pairs,
+                                pairs_cap: int, num_pairs, dst_free_mask_out, dst_free_count_out, status, workspace,
+                                workspace_bytes: int, stream=None) -> None:
+    _check(_load().amoeba_reshape_block_tables(
+        plan.handle, _ptr(src_bt), _ptr(seq_lens), num_seqs, max_blocks_per_seq, _ptr(dst_bt), _ptr(pairs), pairs_cap,
+        _ptr(num_pairs), _ptr(dst_free_mask_out), _ptr(dst_free_count_out), _ptr(status), _ptr(workspace),
+        workspace_bytes, _stream(stream)), "amoeba_reshape_block_tables")
+
+
+def amoeba_reshape_kv_inplace(plan: Plan, pools: Sequence, pairs, num_pairs, pairs_cap: int, layer_begin: int,
+                              layer_end: int, status, stream=None) -> None:
+    """pools: max(a, b) tensors or addresses, pools[w] = worker w of the finer side; worker r of the coarser side is
+    pools[r * N]."""
+    if len(pools) != max(plan.src.tp, plan.dst.tp):
+        raise AmoebaError(ERR_INVALID_ARG, "amoeba_reshape_kv_inplace (need one pool per worker of the finer side)")
+    pp = (C.c_void_p * len(pools))(*[_ptr(x) for x in pools])
+    _check(_load().amoeba_reshape_kv_inplace(plan.handle, pp, _ptr(pairs), _ptr(num_pairs), pairs_cap, layer_begin,
+                                             layer_end, _ptr(status), _stream(stream)), "amoeba_reshape_kv_inplace")
+
+
+def amoeba_reshape_bytes(plan: Plan, n_live_blocks: int) -> int:
+    out = C.c_int64()
+    _check(_load().amoeba_reshape_bytes(plan.handle, n_live_blocks, C.byref(out)), "amoeba_reshape_bytes")
+    return out.value
 
 
 def pack_weights(shards: Sequence[Sequence[dict]]):

@@ -1,12 +1,17 @@
 // Destination block bookkeeping for the KV migration (Sec. 3.1: each worker prepares reserved pages for the KV it
-// receives).  Two launches, no CTA ever waits on another:
-//   bt_scan   (1 CTA)   blocks per sequence, exclusive prefix sum over the sequences, and - when the free blocks
-//                       come as a byte mask - their compaction into an ascending id list (ballot + popc prefix
-//                       sums, one warp-wide ballot per 32 mask bytes); decides the whole-call errors.
-//   bt_assign (grid)    one warp per 128-entry segment of a block-table row: k-th block overall takes the k-th free
-//                       id; writes the destination table (with -1 padding) and the (source, destination) pair list.
+// receives), and the block tables of the in-place block reshaping of one instance (Sec. 3.1, Improvement 1).
+// No CTA ever waits on another.  Two phases:
+//   scan   (1 CTA)  blocks per sequence and their exclusive prefix sum; when the free blocks come as a byte mask,
+//                   their compaction into an ascending id list (16 mask bytes per thread, popc + CTA prefix sum);
+//                   when destination ids can repeat (a free LIST, or ids derived from the source table), the first
+//                   user of every destination id in (sequence, block) order, by atomicMin; the whole-call errors.
+//   assign (grid)   one warp per 128-entry segment of a block-table row: the k-th block overall takes the k-th free
+//                   id (or the reshaped id of its source block); writes the destination table (with -1 padding) and
+//                   the (source, destination) pair list; an id whose first user is another block is refused.
+// Small tables run both phases in one launch of one CTA; large ones as two launches.
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <mutex>
 
 #include "launch.hpp"
@@ -21,7 +26,26 @@ struct BtHeader {  // first 64 bytes of the workspace
     int32_t pad[13];
 };
 
+struct BtArgs {
+    const int32_t* src_bt;
+    const int32_t* seq_lens;
+    const int32_t* free_list;  // list form, or null
+    const uint8_t* free_mask;  // mask form, or null
+    BtHeader* hdr;
+    int32_t* seq_off;     // [num_seqs] exclusive prefix sum of the blocks per sequence
+    int32_t* area;        // mask form: compacted ascending free ids; otherwise: first user of every destination id
+    int32_t* dst_bt;
+    int2* pairs;
+    int32_t* num_pairs;
+    int32_t* free_count_out;
+    int32_t* status;
+    uint8_t* free_mask_out;  // reshaping only: 1 = free id of the destination side
+    int32_t num_seqs, block_tokens, maxb, n_free_or_nb, pairs_cap, nb_src, nb_dst;
+    int32_t reshape;  // 0: ids from the free list / mask; +N: destination id = source id * N; -N: source id / N
+};
+
 constexpr int kScanThreads = 1024;
+constexpr int kSegment = 128;  // table entries one warp handles per step
 
 // Exclusive scan of one value per thread across the CTA; returns the thread's offset, *total = CTA sum.
 __device__ __forceinline__ int32_t cta_exclusive_scan(int32_t v, int32_t* warp_sums, int32_t* total) {
@@ -52,107 +76,207 @@ __device__ __forceinline__ int32_t cta_exclusive_scan(int32_t v, int32_t* warp_s
     return off;
 }
 
-__global__ void __launch_bounds__(kScanThreads) bt_scan(const int32_t* __restrict__ seq_lens, int32_t num_seqs,
-                                                        int32_t block_tokens, int32_t max_blocks_per_seq,
-                                                        const uint8_t* __restrict__ free_mask, int32_t n_free_or_nb,
-                                                        int32_t pairs_cap, BtHeader* hdr, int32_t* __restrict__ seq_off,
-                                                        int32_t* __restrict__ free_ids, int32_t* num_pairs,
-                                                        int32_t* free_count_out, int32_t* status) {
-    __shared__ int32_t warp_sums[33];
-    __shared__ int32_t bad_len;
-    if (threadIdx.x == 0) bad_len = 0;
+__device__ __forceinline__ int32_t blocks_needed(int32_t len, int32_t block_tokens) {
+    return (int32_t)(((int64_t)len + block_tokens - 1) / block_tokens);
+}
+
+// Destination id of the k-th block overall, whose source id is `src`; -1 if there is none.
+__device__ __forceinline__ int32_t dst_id_of(const BtArgs& a, int32_t k, int32_t src) {
+    if (a.reshape == 0) return a.free_mask ? a.area[k] : a.free_list[k];
+    if (src < 0 || src >= a.nb_src) return -1;
+    if (a.reshape > 0) return (int32_t)min((int64_t)src * a.reshape, (int64_t)INT32_MAX);
+    const int32_t n = -a.reshape;
+    return src % n == 0 ? src / n : -1;
+}
+
+// Bit j set = byte j of the word is non-zero.
+__device__ __forceinline__ uint32_t nonzero_bytes(uint32_t w) {
+    return (w & 0xffu ? 1u : 0u) | (w & 0xff00u ? 2u : 0u) | (w & 0xff0000u ? 4u : 0u) | (w & 0xff000000u ? 8u : 0u);
+}
+
+// All kScanThreads threads of ONE CTA.
+__device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) flags[0] = flags[1] = 0;  // [0] bad length, [1] whole-call error
     __syncthreads();
 
     // ---- blocks per sequence and their exclusive prefix sum
     int64_t carry = 0;
-    for (int32_t base = 0; base < num_seqs; base += kScanThreads) {
-        const int32_t s = base + threadIdx.x;
+    for (int32_t base = 0; base < a.num_seqs; base += kScanThreads) {
+        const int32_t s = base + tid;
         int32_t nb = 0;
-        if (s < num_seqs) {
-            const int32_t len = seq_lens[s];
-            const int64_t need = ((int64_t)len + block_tokens - 1) / block_tokens;
-            if (len < 0 || need > max_blocks_per_seq) bad_len = 1;
+        if (s < a.num_seqs) {
+            const int32_t len = a.seq_lens[s];
+            const int64_t need = ((int64_t)len + a.block_tokens - 1) / a.block_tokens;
+            if (len < 0 || need > a.maxb) flags[0] = 1;
             else nb = (int32_t)need;
         }
         int32_t tile_total;
         const int32_t off = cta_exclusive_scan(nb, warp_sums, &tile_total);
-        if (s < num_seqs) seq_off[s] = (int32_t)min(carry + off, (int64_t)INT32_MAX);
+        if (s < a.num_seqs) a.seq_off[s] = (int32_t)min(carry + off, (int64_t)INT32_MAX);
         carry += tile_total;
     }
     const int64_t total = carry;
 
-    // ---- ordered free list from the mask: ascending ids of the non-zero bytes
-    int64_t n_free = n_free_or_nb;
-    if (free_mask) {
-        const int lane = threadIdx.x & 31;
+    // ---- ordered free list from the mask: ascending ids of the non-zero bytes, 16 mask bytes per thread
+    int64_t n_free = a.reshape ? a.nb_dst : a.n_free_or_nb;
+    if (a.free_mask) {
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(a.free_mask) & 15) == 0;
         int32_t found = 0;
-        for (int32_t base = 0; base < n_free_or_nb; base += kScanThreads) {
-            const int32_t id = base + threadIdx.x;
-            const bool is_free = id < n_free_or_nb && free_mask[id] != 0;
-            const uint32_t ballot = __ballot_sync(0xffffffffu, is_free);
+        for (int32_t base = 0; base < a.n_free_or_nb; base += kScanThreads * 16) {
+            const int32_t i0 = base + tid * 16;
+            uint32_t bits = 0;
+            if (vec_ok && i0 + 16 <= a.n_free_or_nb) {
+                const uint4 v = *reinterpret_cast<const uint4*>(a.free_mask + i0);
+                bits = nonzero_bytes(v.x) | nonzero_bytes(v.y) << 4 | nonzero_bytes(v.z) << 8 | nonzero_bytes(v.w) << 12;
+            } else {
+                for (int j = 0; j < 16; ++j)
+                    if (i0 + j < a.n_free_or_nb && a.free_mask[i0 + j]) bits |= 1u << j;
+            }
             int32_t tile_total;
-            const int32_t warp_off = cta_exclusive_scan(lane == 0 ? __popc(ballot) : 0, warp_sums, &tile_total);
-            const int32_t my_warp_off = __shfl_sync(0xffffffffu, warp_off, 0);
-            if (is_free) free_ids[found + my_warp_off + __popc(ballot & ((1u << lane) - 1u))] = id;
+            int32_t pos = found + cta_exclusive_scan(__popc(bits), warp_sums, &tile_total);
+            while (bits) {
+                const int j = __ffs(bits) - 1;
+                bits &= bits - 1;
+                a.area[pos++] = i0 + j;
+            }
             found += tile_total;
         }
         n_free = found;
     }
 
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         int32_t err = 0;
-        if (bad_len) err = AMOEBA_ERR_INVALID_ARG;
-        else if (total > pairs_cap) err = AMOEBA_ERR_INVALID_ARG;
-        else if (total > n_free) err = AMOEBA_ERR_NO_FREE_BLOCKS;
+        if (flags[0]) err = AMOEBA_ERR_INVALID_ARG;
+        else if (total > a.pairs_cap) err = AMOEBA_ERR_INVALID_ARG;
+        else if (!a.reshape && total > n_free) err = AMOEBA_ERR_NO_FREE_BLOCKS;
         const int32_t assigned = err ? 0 : (int32_t)total;
-        hdr->total = assigned;
-        hdr->n_free = (int32_t)n_free;
-        hdr->err = err;
-        *num_pairs = assigned;
-        *free_count_out = (int32_t)n_free - assigned;
-        if (err) atomicCAS(status, 0, err);
+        a.hdr->total = assigned;
+        a.hdr->n_free = (int32_t)n_free;
+        a.hdr->err = err;
+        *a.num_pairs = assigned;
+        *a.free_count_out = (int32_t)n_free - assigned;
+        if (err) atomicCAS(a.status, 0, err);
+        flags[1] = err;
+    }
+    __syncthreads();
+
+    // ---- first user of every destination id (ids from a list or from the source table may repeat)
+    if (!a.free_mask) {
+        for (int32_t q = tid; q < a.nb_dst; q += kScanThreads) a.area[q] = INT32_MAX;
+        __syncthreads();
+        if (flags[1] == 0) {
+            for (int32_t s = warp; s < a.num_seqs; s += kScanThreads / 32) {
+                const int32_t nb = blocks_needed(a.seq_lens[s], a.block_tokens), off = a.seq_off[s];
+                for (int32_t i = lane; i < nb; i += 32) {
+                    const int32_t d = dst_id_of(a, off + i, a.src_bt[(int64_t)s * a.maxb + i]);
+                    if (d >= 0 && d < a.nb_dst) atomicMin(a.area + d, off + i);
+                }
+            }
+        }
     }
 }
 
-constexpr int kSegment = 128;  // table entries one warp handles per step
-
-__global__ void __launch_bounds__(256) bt_assign(const int32_t* __restrict__ src_bt,
-                                                 const int32_t* __restrict__ seq_lens, int32_t num_seqs,
-                                                 int32_t block_tokens, int32_t max_blocks_per_seq,
-                                                 const int32_t* __restrict__ free_ids, const BtHeader* hdr,
-                                                 const int32_t* __restrict__ seq_off, int32_t nb_src, int32_t nb_dst,
-                                                 int32_t* __restrict__ dst_bt, int2* __restrict__ pairs,
-                                                 int32_t* status) {
+// Any number of warps; warp `warp` of `n_warps`.  Runs after scan_phase has completed (next launch, or after a
+// __syncthreads() of the one CTA that ran it).
+__device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
     const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int32_t segs_per_row = (max_blocks_per_seq + kSegment - 1) / kSegment;
-    const bool call_failed = hdr->err != 0;
+    const int32_t segs_per_row = (a.maxb + kSegment - 1) / kSegment;
+    const bool call_failed = a.hdr->err != 0;
+    const bool check_first = a.free_mask == nullptr;
     bool bad = false;
-    for (int64_t unit = warp; unit < (int64_t)num_seqs * segs_per_row; unit += n_warps) {
+    int32_t refused = 0;  // reshaping: blocks that keep no destination id
+    for (int64_t unit = warp; unit < (int64_t)a.num_seqs * segs_per_row; unit += n_warps) {
         const int32_t s = (int32_t)(unit / segs_per_row);
         const int32_t col0 = (int32_t)(unit - (int64_t)s * segs_per_row) * kSegment;
-        const int32_t nb = call_failed ? 0 : (int32_t)(((int64_t)seq_lens[s] + block_tokens - 1) / block_tokens);
-        const int32_t off = seq_off[s];
-        for (int32_t i = col0 + lane; i < min(col0 + kSegment, max_blocks_per_seq); i += 32) {
+        const int32_t nb = call_failed ? 0 : blocks_needed(a.seq_lens[s], a.block_tokens);
+        const int32_t off = a.seq_off[s];
+        for (int32_t i = col0 + lane; i < min(col0 + kSegment, a.maxb); i += 32) {
             int32_t out = -1;
             if (i < nb) {
                 const int32_t k = off + i;
-                const int32_t dst = free_ids[k];
-                const int32_t src = src_bt[(int64_t)s * max_blocks_per_seq + i];
-                const bool dst_ok = dst >= 0 && dst < nb_dst, src_ok = src >= 0 && src < nb_src;
+                const int32_t src = a.src_bt[(int64_t)s * a.maxb + i];
+                const int32_t dst = dst_id_of(a, k, src);
+                bool dst_ok = dst >= 0 && dst < a.nb_dst;
+                if (dst_ok && check_first && a.area[dst] != k) dst_ok = false;  // an earlier block holds this id
+                const bool src_ok = src >= 0 && src < a.nb_src;
                 out = dst_ok ? dst : -1;
-                pairs[k] = (dst_ok && src_ok) ? make_int2(src, dst) : make_int2(-1, -1);
+                a.pairs[k] = (dst_ok && src_ok) ? make_int2(src, dst) : make_int2(-1, -1);
                 bad |= !(dst_ok && src_ok);
+                refused += !dst_ok;
             }
-            dst_bt[(int64_t)s * max_blocks_per_seq + i] = out;
+            a.dst_bt[(int64_t)s * a.maxb + i] = out;
         }
     }
-    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(a.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+    if (a.reshape) {
+        refused = __reduce_add_sync(0xffffffffu, refused);
+        if (refused && lane == 0) atomicAdd(a.free_count_out, refused);
+        for (int64_t q = warp * 32 + lane; q < a.nb_dst; q += n_warps * 32)
+            a.free_mask_out[q] = (call_failed || a.area[q] == INT32_MAX) ? 1 : 0;
+    }
 }
 
+__global__ void __launch_bounds__(kScanThreads) bt_scan(const __grid_constant__ BtArgs a) {
+    __shared__ int32_t warp_sums[33];
+    __shared__ int32_t flags[2];
+    scan_phase(a, warp_sums, flags);
+}
+
+__global__ void __launch_bounds__(256) bt_assign(const __grid_constant__ BtArgs a) {
+    assign_phase(a, ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, ((int64_t)gridDim.x * blockDim.x) >> 5);
+}
+
+// Both phases in one CTA: what the CTA wrote to global memory in the scan is visible to all its threads after the
+// barrier.
+__global__ void __launch_bounds__(kScanThreads) bt_fused(const __grid_constant__ BtArgs a) {
+    __shared__ int32_t warp_sums[33];
+    __shared__ int32_t flags[2];
+    scan_phase(a, warp_sums, flags);
+    __threadfence_block();
+    __syncthreads();
+    assign_phase(a, threadIdx.x >> 5, kScanThreads / 32);
+}
+
+constexpr int64_t kFusedEntries = 128 * 1024;  // up to this many table entries (and destination ids): one launch
+
 static int64_t align16(int64_t x) { return (x + 15) & ~int64_t(15); }
+
+static int64_t tables_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs) {
+    return (int64_t)sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)) +
+           align16(4 * (int64_t)std::max(plan->src.num_blocks, plan->dst.num_blocks));
+}
+
+static amoeba_status launch_tables(const amoeba_plan* plan, BtArgs a, void* d_workspace, cudaStream_t stream) {
+    char* ws = static_cast<char*>(d_workspace);
+    a.hdr = reinterpret_cast<BtHeader*>(ws);
+    a.seq_off = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader));
+    a.area = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader) + align16(4 * ((int64_t)a.num_seqs + 1)));
+    a.block_tokens = plan->src.block_tokens;
+    a.nb_src = plan->src.num_blocks;
+    a.nb_dst = plan->dst.num_blocks;
+    const int64_t entries = (int64_t)a.num_seqs * a.maxb;
+    if (entries <= kFusedEntries && a.nb_dst <= kFusedEntries) {
+        bt_fused<<<1, kScanThreads, 0, stream>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+        count_launch();
+        return AMOEBA_OK;
+    }
+    bt_scan<<<1, kScanThreads, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    if (a.num_seqs == 0 && !a.reshape) return AMOEBA_OK;
+    const int sms = cached_device_info().sms;
+    if (sms <= 0) return AMOEBA_ERR_CUDA;
+    const int64_t units = std::max<int64_t>((int64_t)a.num_seqs * ((a.maxb + kSegment - 1) / kSegment),
+                                            a.reshape ? (a.nb_dst + 31) / 32 : 0);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((units + 7) / 8, (int64_t)sms * 8));
+    bt_assign<<<grid, 256, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+    count_launch();
+    return AMOEBA_OK;
+}
 
 }  // namespace amoeba
 
@@ -161,7 +285,7 @@ using namespace amoeba;
 extern "C" amoeba_status amoeba_rewrite_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs,
                                                         int32_t n_free_or_nb, int64_t* bytes) {
     if (!plan || !bytes || num_seqs < 0 || n_free_or_nb < 0) return AMOEBA_ERR_INVALID_ARG;
-    *bytes = (int64_t)sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)) + align16(4 * (int64_t)n_free_or_nb);
+    *bytes = tables_workspace_bytes(plan, num_seqs);
     return AMOEBA_OK;
 }
 
@@ -180,36 +304,58 @@ extern "C" amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
     if (num_seqs > 0 && (!d_src_bt || !d_seq_lens || !d_dst_bt)) return AMOEBA_ERR_INVALID_ARG;
     if (pairs_cap > 0 && !d_pairs) return AMOEBA_ERR_INVALID_ARG;
     if (d_dst_free_mask && n_free_or_nb != plan->dst.num_blocks) return AMOEBA_ERR_INVALID_ARG;
-    int64_t need = 0;
-    amoeba_rewrite_workspace_bytes(plan, num_seqs, n_free_or_nb, &need);
-    if (workspace_bytes < need) return AMOEBA_ERR_INVALID_ARG;
+    if (workspace_bytes < tables_workspace_bytes(plan, num_seqs)) return AMOEBA_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_workspace) % 16 || reinterpret_cast<uintptr_t>(d_pairs) % 8)
         return AMOEBA_ERR_ALIGNMENT;
+    BtArgs a{};
+    a.src_bt = d_src_bt;
+    a.seq_lens = d_seq_lens;
+    a.free_list = d_dst_free_list;
+    a.free_mask = d_dst_free_mask;
+    a.dst_bt = d_dst_bt;
+    a.pairs = reinterpret_cast<int2*>(d_pairs);
+    a.num_pairs = d_num_pairs;
+    a.free_count_out = d_dst_free_count_out;
+    a.status = d_status;
+    a.num_seqs = num_seqs;
+    a.maxb = max_blocks_per_seq;
+    a.n_free_or_nb = n_free_or_nb;
+    a.pairs_cap = pairs_cap;
+    return launch_tables(plan, a, d_workspace, static_cast<cudaStream_t>(cuda_stream));
+}
 
-    char* ws = static_cast<char*>(d_workspace);
-    BtHeader* hdr = reinterpret_cast<BtHeader*>(ws);
-    int32_t* seq_off = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader));
-    int32_t* compact = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)));
-    const int32_t* free_ids = d_dst_free_mask ? compact : d_dst_free_list;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-
-    bt_scan<<<1, kScanThreads, 0, stream>>>(d_seq_lens, num_seqs, plan->src.block_tokens, max_blocks_per_seq,
-                                            d_dst_free_mask, n_free_or_nb, pairs_cap, hdr, seq_off, compact,
-                                            d_num_pairs, d_dst_free_count_out, d_status);
-    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
-    count_launch();
-    if (num_seqs == 0) return AMOEBA_OK;
-
-    DeviceInfo dev;
-    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
-    const int64_t units = (int64_t)num_seqs * ((max_blocks_per_seq + kSegment - 1) / kSegment);
-    const int grid = (int)std::min<int64_t>((units + 7) / 8, (int64_t)dev.sms * 8);
-    bt_assign<<<grid, 256, 0, stream>>>(d_src_bt, d_seq_lens, num_seqs, plan->src.block_tokens, max_blocks_per_seq,
-                                        free_ids, hdr, seq_off, plan->src.num_blocks, plan->dst.num_blocks, d_dst_bt,
-                                        reinterpret_cast<int2*>(d_pairs), d_status);
-    if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
-    count_launch();
-    return AMOEBA_OK;
+extern "C" amoeba_status amoeba_reshape_block_tables(const amoeba_plan* plan, const int32_t* d_src_bt,
+                                                     const int32_t* d_seq_lens, int32_t num_seqs,
+                                                     int32_t max_blocks_per_seq, int32_t* d_dst_bt, int32_t* d_pairs,
+                                                     int32_t pairs_cap, int32_t* d_num_pairs,
+                                                     uint8_t* d_dst_free_mask_out, int32_t* d_dst_free_count_out,
+                                                     int32_t* d_status, void* d_workspace, int64_t workspace_bytes,
+                                                     void* cuda_stream) {
+    if (!plan || num_seqs < 0 || max_blocks_per_seq <= 0 || pairs_cap < 0) return AMOEBA_ERR_INVALID_ARG;
+    const int n = reshape_factor(plan);
+    if (!n) return AMOEBA_ERR_UNSUPPORTED;
+    if (!d_num_pairs || !d_dst_free_count_out || !d_dst_free_mask_out || !d_status || !d_workspace)
+        return AMOEBA_ERR_INVALID_ARG;
+    if (num_seqs > 0 && (!d_src_bt || !d_seq_lens || !d_dst_bt)) return AMOEBA_ERR_INVALID_ARG;
+    if (pairs_cap > 0 && !d_pairs) return AMOEBA_ERR_INVALID_ARG;
+    if (workspace_bytes < tables_workspace_bytes(plan, num_seqs)) return AMOEBA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_workspace) % 16 || reinterpret_cast<uintptr_t>(d_pairs) % 8)
+        return AMOEBA_ERR_ALIGNMENT;
+    BtArgs a{};
+    a.src_bt = d_src_bt;
+    a.seq_lens = d_seq_lens;
+    a.dst_bt = d_dst_bt;
+    a.pairs = reinterpret_cast<int2*>(d_pairs);
+    a.num_pairs = d_num_pairs;
+    a.free_count_out = d_dst_free_count_out;
+    a.free_mask_out = d_dst_free_mask_out;
+    a.status = d_status;
+    a.num_seqs = num_seqs;
+    a.maxb = max_blocks_per_seq;
+    a.n_free_or_nb = plan->dst.num_blocks;
+    a.pairs_cap = pairs_cap;
+    a.reshape = n;
+    return launch_tables(plan, a, d_workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -284,8 +430,8 @@ static amoeba_status merge_or_split_tables(bool split, const amoeba_plan* plan, 
     if (cudaMemsetAsync(d_live, 0, (size_t)live_bytes, stream) != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();
     if (num_seqs == 0) return AMOEBA_OK;
-    DeviceInfo dev;
-    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    const DeviceInfo dev = cached_device_info();
+    if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     const int64_t units = (int64_t)n * num_seqs * ((max_blocks_per_seq + kSegment - 1) / kSegment);
     const int grid = (int)std::min<int64_t>((units + 7) / 8, (int64_t)dev.sms * 4);
     auto kernel = split ? merge_tables<true> : merge_tables<false>;
@@ -320,8 +466,9 @@ namespace amoeba {
 static __device__ __align__(256) unsigned char g_builtin_scratch[AMOEBA_BUILTIN_SCRATCH_BYTES];
 
 // In host code `g_builtin_scratch` is only a handle for the runtime, not an address a kernel could use; the
-// device-side address is asked for once per device and remembered here (index = device ordinal).
-constexpr int kMaxDevices = 64;
+// device-side address is asked for once per device and remembered here (index = device ordinal).  The remembered
+// address belongs to the device's primary context as it was at that first call: it does not survive a
+// cudaDeviceReset of that device.
 static void* g_builtin_scratch_addr[kMaxDevices];
 static std::mutex g_builtin_scratch_mutex;
 
@@ -332,19 +479,24 @@ extern "C" amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
     int32_t max_blocks_per_seq, const int32_t* d_dst_free_list, const uint8_t* d_dst_free_mask, int32_t n_free_or_nb,
     int32_t* d_dst_bt, int32_t* d_pairs, int32_t pairs_cap, int32_t* d_num_pairs, int32_t* d_dst_free_count_out,
     int32_t* d_status, void* cuda_stream) {
-    int64_t need = 0;
-    const amoeba_status st = amoeba_rewrite_workspace_bytes(plan, num_seqs, n_free_or_nb, &need);
-    if (st != AMOEBA_OK) return st;
-    if (need > (int64_t)AMOEBA_BUILTIN_SCRATCH_BYTES) return AMOEBA_ERR_TOO_LARGE;
+    if (!plan || num_seqs < 0 || n_free_or_nb < 0) return AMOEBA_ERR_INVALID_ARG;
+    if (tables_workspace_bytes(plan, num_seqs) > (int64_t)AMOEBA_BUILTIN_SCRATCH_BYTES) return AMOEBA_ERR_TOO_LARGE;
 
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AMOEBA_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) {
+        (void)cudaGetLastError();  // do not leave the runtime's error state set for a later, unrelated check
+        return AMOEBA_ERR_CUDA;
+    }
+    if (dev >= kMaxDevices) return AMOEBA_ERR_UNSUPPORTED;  // more device ordinals than this table remembers
     void* scratch = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_builtin_scratch_mutex);
         if (!g_builtin_scratch_addr[dev]) {  // first use with this device current
             void* p = nullptr;
-            if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) return AMOEBA_ERR_CUDA;
+            if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) {
+                (void)cudaGetLastError();
+                return AMOEBA_ERR_CUDA;
+            }
             g_builtin_scratch_addr[dev] = p;
         }
         scratch = g_builtin_scratch_addr[dev];

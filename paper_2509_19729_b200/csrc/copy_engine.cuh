@@ -39,6 +39,7 @@ struct RingShape {
     int32_t lag;          // warp ring: loads lead stores by this many items; pair ring: stores kept in flight
     int32_t stage_bytes;  // bytes per stage
     int32_t hint;         // bit 0: loads evict-first in L2, bit 1: stores evict-first in L2
+    int32_t max_polls;    // 0: default wait budget; > 0: every mbarrier wait gives up after this many non-blocking polls
 };
 
 // ------------------------------------------------------------------ vector load/store path
@@ -130,11 +131,39 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within the try budget.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_tries = (1u << 22)) {
-    for (uint32_t i = 0; i < max_tries; ++i)
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+constexpr uint32_t kDefaultWaitTries = 1u << 22;
+constexpr uint32_t kDrainWaitTries = 1u << 16;
+// Bounded wait: false if the phase did not complete within the budget, or if *abort became non-zero meanwhile (the
+// other warp of the ring gave up).  max_polls == 0: the default budget of potentially-suspending try_wait calls;
+// max_polls > 0: that many non-blocking polls (a caller-chosen, short limit).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_polls = 0,
+                                                  const volatile int32_t* abort = nullptr) {
+    if (max_polls) {
+        for (uint32_t i = 0; i < max_polls; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
+        return false;
+    }
+    for (uint32_t i = 0; i < kDefaultWaitTries; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (abort && (i & 15) == 15 && *abort) return false;
+    }
     return false;
+}
+// Give copies that are still in flight a bounded chance to land: waits for the phase, never reports.
+__device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kDrainWaitTries; ++i)
+        if (mbar_try_wait(bar, parity)) return;
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
     uint64_t p;
@@ -221,6 +250,10 @@ __device__ __forceinline__ void bulk_wait_read(int n) {
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 constexpr int kMaxStages = 16;
+// Head of a ring kernel's dynamic shared memory: mbarriers, then one abort word per producer/consumer ring.
+constexpr int kBarrierBytes = 1024;
+constexpr int kBarrierSlots = 112;                 // 8-byte mbarriers
+constexpr int kAbortOffset = kBarrierSlots * 8;    // 32 int32 abort words behind them
 
 // One item between global memory and a shared-memory stage (rows packed densely in the stage).  A side whose rows
 // are adjacent in global memory (pitch == row_bytes, or a single row) moves as ONE bulk copy issued by lane 0;
@@ -283,7 +316,7 @@ __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, 
             if (++s_load == NS) s_load = 0;
         }
         if (k >= LAG) {
-            ok = mbar_wait_bounded(&bars[s_store], store_parity);
+            ok = mbar_wait_bounded(&bars[s_store], store_parity, (uint32_t)rs.max_polls);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 ++loads_waited;
@@ -299,31 +332,37 @@ __device__ __forceinline__ bool warp_bulk_ring(ItemFn item_of, int64_t n_items, 
     }
     bulk_wait_all();  // this lane's stores are complete
     if (!ok) {        // give the loads still in flight a bounded chance to land before the CTA's smem goes away
-        for (int64_t j = loads_waited; j < loads_issued; ++j)
-            mbar_wait_bounded(&bars[j % NS], (uint32_t)((j / NS) & 1), 1u << 16);
+        for (int64_t j = loads_waited; j < loads_issued; ++j) mbar_drain(&bars[j % NS], (uint32_t)((j / NS) & 1));
     }
     __syncwarp();
     return ok;
 }
 
 // ------------------------------------------------------------------ producer warp + consumer warp on one ring
-// `role` 0 = producer (loads), 1 = consumer (stores).  full/empty: `stages` mbarriers each, initialised by
-// pair_ring_init before both warps start.  rs.lag = number of store groups the consumer keeps in flight before it
-// hands a slot back.
-__device__ __forceinline__ void pair_ring_init(uint64_t* full, uint64_t* empty, int stages) {
+// `role` 0 = producer (loads), 1 = consumer (stores).  full/empty: `stages` mbarriers each, and the ring's abort
+// word, initialised by pair_ring_init before both warps start.  rs.lag = number of store groups the consumer keeps
+// in flight before it hands a slot back.
+// Giving up: a warp whose bounded wait runs out raises the ring's abort word and leaves; the other warp sees the word
+// (at its next item, or while it polls) and leaves too.  Before the CTA may exit, the consumer has waited for its own
+// stores, and the producer has waited - bounded again - for every load it armed, so that no copy of this ring is still
+// writing into the CTA's shared memory.  Both return false.
+__device__ __forceinline__ void pair_ring_init(uint64_t* full, uint64_t* empty, int32_t* abort, int stages) {
     for (int s = 0; s < stages; ++s) {
         mbar_init(&full[s], 1);
         mbar_init(&empty[s], 1);
     }
+    *abort = 0;
     fence_async_smem();
 }
 
 template <class ItemFn>
 __device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t n_items, int64_t first,
                                                int64_t stride, char* stages, uint64_t* full, uint64_t* empty,
-                                               const RingShape rs) {
+                                               int32_t* abort_word, const RingShape rs) {
     const int lane = threadIdx.x & 31;
     const int NS = rs.stages, D = rs.lag;
+    const uint32_t polls = (uint32_t)rs.max_polls;
+    volatile int32_t* abort = abort_word;
     const uint64_t policy = policy_evict_first();
     const int64_t n_local = n_items > first ? (n_items - first + stride - 1) / stride : 0;
     bool ok = true;
@@ -331,26 +370,35 @@ __device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t
     uint32_t parity = 0;
     if (role == 0) {
         const bool hl = rs.hint & 1;
-        for (int64_t k = 0; k < n_local && ok; ++k) {
-            if (k >= NS) {  // wait until the consumer has handed this slot back (its previous use)
-                ok = mbar_wait_bounded(&empty[slot], parity ^ 1);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
+        int64_t armed = 0;  // "full" phases armed so far
+        for (int64_t k = 0; k < n_local; ++k) {
+            if (*abort) ok = false;
+            if (ok && k >= NS)  // wait until the consumer has handed this slot back (its previous use)
+                ok = mbar_wait_bounded(&empty[slot], parity ^ 1, polls, abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
             const Item it = item_of(first + k * stride);
             if (lane == 0) mbar_arrive_expect_tx(&full[slot], (uint32_t)it.n_rows * (uint32_t)it.row_bytes);
             __syncwarp();
             item_load(it, stages + (int64_t)slot * rs.stage_bytes, &full[slot], hl, policy);
+            ++armed;
             if (++slot == NS) {
                 slot = 0;
                 parity ^= 1;
             }
         }
+        if (!ok) {
+            if (lane == 0) *abort = 1;
+            // the last min(NS, armed) uses of the ring may still have loads in flight
+            for (int64_t j = armed > NS ? armed - NS : 0; j < armed; ++j)
+                mbar_drain(&full[j % NS], (uint32_t)((j / NS) & 1));
+        }
     } else {
         const bool hs = rs.hint & 2;
         int release = 0;  // slot of the oldest store not yet handed back
-        for (int64_t k = 0; k < n_local && ok; ++k) {
-            ok = mbar_wait_bounded(&full[slot], parity);
+        for (int64_t k = 0; k < n_local; ++k) {
+            if (*abort) ok = false;
+            if (ok) ok = mbar_wait_bounded(&full[slot], parity, polls, abort);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const Item it = item_of(first + k * stride);
@@ -367,10 +415,34 @@ __device__ __forceinline__ bool pair_bulk_ring(int role, ItemFn item_of, int64_t
                 parity ^= 1;
             }
         }
+        if (!ok && lane == 0) *abort = 1;
         bulk_wait_all();
     }
     __syncwarp();
     return ok;
+}
+
+// The calling warp's place in a CTA of producer/consumer rings: warps 2r and 2r+1 are the producer and the consumer of
+// ring r.  Initialises the ring's barriers and ends with a CTA-wide barrier: call it from every thread.
+struct PairRing {
+    uint64_t *full, *empty;
+    int32_t* abort;
+    char* stages;
+    int ring, role, nrings;
+};
+__device__ __forceinline__ PairRing pair_ring_setup(char* smem, const RingShape& rs) {
+    PairRing r;
+    const int warp = threadIdx.x >> 5;
+    r.ring = warp >> 1;
+    r.role = warp & 1;
+    r.nrings = blockDim.x >> 6;
+    r.full = reinterpret_cast<uint64_t*>(smem) + r.ring * 2 * rs.stages;
+    r.empty = r.full + rs.stages;
+    r.abort = reinterpret_cast<int32_t*>(smem + kAbortOffset) + r.ring;
+    r.stages = smem + kBarrierBytes + (int64_t)r.ring * rs.stages * rs.stage_bytes;
+    if (r.role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(r.full, r.empty, r.abort, rs.stages);
+    __syncthreads();
+    return r;
 }
 
 }  // namespace amoeba

@@ -14,6 +14,7 @@
 
 #include <cstring>
 #include <mutex>
+#include <new>
 
 #include "copy_engine.cuh"
 #include "launch.hpp"
@@ -36,6 +37,10 @@ struct KvParams {
     int32_t rows, rows_per_item, row_groups, col_chunks, chunk_bytes;
     // box items (tensor-map path)
     int32_t heads_per_run, runs_per_block, box_heads, box_tokens, box_sub_runs, box_tok_groups;
+    // In-place block reshaping of one instance (0 = off): +N, the destination has N times the source's workers and
+    // destination worker r*N IS source worker r; -N, the other way round.  The header unit a worker retains
+    // (every N-th) is not a work item at all: `moving_units` counts the others.
+    int32_t reshape, moving_units;
 };
 
 // Tensor maps of the token-first pools, one per worker: dimensions {dim, token of the layer's K or V region,
@@ -65,7 +70,7 @@ struct KvItems {
     const KvParams& p;
     int32_t n_pairs;
     __device__ __forceinline__ int32_t items_per_pair() const {
-        return p.planes * p.head_units * p.row_groups * p.col_chunks;
+        return p.planes * p.moving_units * p.row_groups * p.col_chunks;
     }
     __device__ __forceinline__ int64_t count() const { return (int64_t)n_pairs * p.n_layers * items_per_pair(); }
     // n_rows == 0 marks a skipped pair.
@@ -77,8 +82,13 @@ struct KvItems {
         uint32_t rem = (uint32_t)(w - lp * ipp);
         const int32_t col = take_digit(rem, p.col_chunks);
         const int32_t rg = take_digit(rem, p.row_groups);
-        const int32_t hu = take_digit(rem, p.head_units);
+        int32_t hu = take_digit(rem, p.moving_units);
         const int32_t c = (int32_t)rem;  // < planes
+        if (p.reshape) {  // skip every N-th unit: the m-th moving unit is unit (m / (N-1)) * N + 1 + m % (N-1)
+            const int32_t n = p.reshape > 0 ? p.reshape : -p.reshape;
+            const int32_t grp = hu / (n - 1);
+            hu = grp * n + 1 + (hu - grp * (n - 1));
+        }
         const int32_t pair = (int32_t)(lp % n_pairs);
         const int32_t layer = p.layer_begin + (int32_t)(lp / n_pairs);
         const int2 ids = __ldg(reinterpret_cast<const int2*>(p.pairs) + pair);
@@ -91,8 +101,11 @@ struct KvItems {
         it.src = nullptr;
         it.dst = nullptr;
         if (ids.x < 0 || ids.y < 0) return it;  // the table rewrite already reported this one
-        if (ids.x >= p.nb_src || ids.y >= p.nb_dst) {
-            if (hu == 0 && c == 0 && rg == 0 && col == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+        // Reshaping in place: the retained headers only stay where they are if the finer side's id is N times the other.
+        const bool reshaped_ok = p.reshape == 0 || (p.reshape > 0 ? (int64_t)ids.x * p.reshape == ids.y
+                                                                  : (int64_t)ids.y * -p.reshape == ids.x);
+        if (ids.x >= p.nb_src || ids.y >= p.nb_dst || !reshaped_ok) {
+            if (c == 0 && rg == 0 && col == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
             return it;
         }
         const int32_t h0 = hu * p.heads_per_unit;  // first header of the unit
@@ -204,15 +217,10 @@ __global__ void __launch_bounds__(1024) kv_reshard_bulk(const __grid_constant__ 
 // Warps 2r and 2r+1 are the producer and the consumer of ring r.
 __global__ void __launch_bounds__(1024) kv_reshard_pair(const __grid_constant__ KvParams p, const RingShape rs) {
     extern __shared__ __align__(128) char smem[];
-    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
-    uint64_t* empty = full + rs.stages;
-    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
-    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
-    __syncthreads();
+    const PairRing r = pair_ring_setup(smem, rs);
     const KvItems items{p, clamp_pairs(p)};
-    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
-                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    const bool ok = pair_bulk_ring(r.role, items, items.count(), (int64_t)blockIdx.x * r.nrings + r.ring,
+                                   (int64_t)gridDim.x * r.nrings, r.stages, r.full, r.empty, r.abort, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
@@ -232,15 +240,10 @@ __global__ void __launch_bounds__(1024) kv_reshard_bulk_box(const __grid_constan
 __global__ void __launch_bounds__(1024) kv_reshard_pair_box(const __grid_constant__ KvParams p,
                                                             const __grid_constant__ KvMaps maps, const RingShape rs) {
     extern __shared__ __align__(128) char smem[];
-    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
-    uint64_t* empty = full + rs.stages;
-    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
-    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
-    __syncthreads();
+    const PairRing r = pair_ring_setup(smem, rs);
     const KvBoxItems items{p, maps, clamp_pairs(p)};
-    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
-                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    const bool ok = pair_bulk_ring(r.role, items, items.count(), (int64_t)blockIdx.x * r.nrings + r.ring,
+                                   (int64_t)gridDim.x * r.nrings, r.stages, r.full, r.empty, r.abort, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
@@ -322,15 +325,10 @@ __global__ void __launch_bounds__(1024) kv_merge_bulk(const __grid_constant__ Me
 __global__ void __launch_bounds__(1024) kv_merge_pair(const __grid_constant__ MergeParams p, const RingShape rs,
                                                       int32_t* status) {
     extern __shared__ __align__(128) char smem[];
-    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
-    uint64_t* empty = full + rs.stages;
-    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
-    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
-    __syncthreads();
+    const PairRing r = pair_ring_setup(smem, rs);
     const MergeItems items{p};
-    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
-                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    const bool ok = pair_bulk_ring(r.role, items, items.count(), (int64_t)blockIdx.x * r.nrings + r.ring,
+                                   (int64_t)gridDim.x * r.nrings, r.stages, r.full, r.empty, r.abort, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
@@ -376,30 +374,58 @@ static bool encode_pool_map(CUtensorMap* out, const void* pool, const amoeba_lay
 
 using namespace amoeba;
 
-extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools,
-                                           void* const* dst_pools, const int32_t* d_pairs, const int32_t* d_num_pairs,
-                                           int32_t pairs_cap, int32_t layer_begin, int32_t layer_end, int32_t* d_status,
-                                           void* cuda_stream) {
-    if (!plan || !src_pools || !dst_pools || !d_pairs || !d_num_pairs || !d_status || pairs_cap < 0)
-        return AMOEBA_ERR_INVALID_ARG;
-    const amoeba_model& m = plan->src.model;
-    if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_pairs) % 8) return AMOEBA_ERR_ALIGNMENT;
-    KvParams p{};
-    for (int r = 0; r < plan->src.tp; ++r) {
-        if (!src_pools[r]) return AMOEBA_ERR_INVALID_ARG;
-        if (reinterpret_cast<uintptr_t>(src_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
-        p.src[r] = static_cast<const char*>(src_pools[r]);
+// Encoded tensor maps of a plan's token-first pools, kept while the pool addresses and the plan's options stay the same.
+struct LaunchCache {
+    std::mutex mutex;
+    uint64_t generation = 0;  // plan generation the maps were encoded for (0 = none yet)
+    const void* src[AMOEBA_MAX_TP] = {};
+    const void* dst[AMOEBA_MAX_TP] = {};
+    amoeba::KvMaps maps;
+};
+
+amoeba_plan::~amoeba_plan() { delete cache; }
+
+namespace amoeba {
+
+// Fills *maps for the given pools: from the plan's cache when nothing changed since they were last encoded.
+static bool pool_maps(const amoeba_plan* plan, const KvParams& p, KvMaps* maps) {
+    static std::mutex create_mutex;
+    amoeba_plan* mp = const_cast<amoeba_plan*>(plan);  // the cache is the plan's only state that data calls change
+    {
+        std::lock_guard<std::mutex> lock(create_mutex);
+        if (!mp->cache) mp->cache = new (std::nothrow) LaunchCache();
+        if (!mp->cache) return false;
     }
-    for (int r = 0; r < plan->dst.tp; ++r) {
-        if (!dst_pools[r]) return AMOEBA_ERR_INVALID_ARG;
-        if (reinterpret_cast<uintptr_t>(dst_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
-        p.dst[r] = static_cast<char*>(dst_pools[r]);
+    LaunchCache& c = *mp->cache;
+    std::lock_guard<std::mutex> lock(c.mutex);
+    const uint64_t gen = plan->generation.load(std::memory_order_relaxed);
+    bool same = c.generation == gen;
+    for (int r = 0; same && r < plan->src.tp; ++r) same = c.src[r] == p.src[r];
+    for (int r = 0; same && r < plan->dst.tp; ++r) same = c.dst[r] == p.dst[r];
+    if (!same) {
+        c.generation = 0;
+        std::memset(&c.maps, 0, sizeof(c.maps));
+        if (p.src_token_major)
+            for (int r = 0; r < plan->src.tp; ++r)
+                if (!encode_pool_map(&c.maps.src[r], p.src[r], plan->src, plan->src_layer_stride, plan->heads_src,
+                                     plan->vec_bytes, plan->kvbox))
+                    return false;
+        if (p.dst_token_major)
+            for (int r = 0; r < plan->dst.tp; ++r)
+                if (!encode_pool_map(&c.maps.dst[r], p.dst[r], plan->dst, plan->dst_layer_stride, plan->heads_dst,
+                                     plan->vec_bytes, plan->kvbox))
+                    return false;
+        for (int r = 0; r < plan->src.tp; ++r) c.src[r] = p.src[r];
+        for (int r = 0; r < plan->dst.tp; ++r) c.dst[r] = p.dst[r];
+        c.generation = gen;
     }
-    if (pairs_cap == 0 || layer_begin == layer_end) return AMOEBA_OK;
-    p.pairs = d_pairs;
-    p.num_pairs = d_num_pairs;
-    p.status = d_status;
+    *maps = c.maps;
+    return true;
+}
+
+// Geometry from the plan, then the launch of the chosen copy kernel.  p.src / p.dst / pairs / status / layer range /
+// reshape are set by the caller.
+static amoeba_status launch_kv(const amoeba_plan* plan, KvParams& p, cudaStream_t stream) {
     const KvGeom& g = plan->kv;
     p.vec_bytes = plan->vec_bytes;
     p.row_bytes = g.row_bytes;
@@ -425,27 +451,28 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     p.box_tok_groups = bx.tok_groups;
     p.src_layer_stride = plan->src_layer_stride;
     p.dst_layer_stride = plan->dst_layer_stride;
-    p.pairs_cap = pairs_cap;
-    p.layer_begin = layer_begin;
-    p.n_layers = layer_end - layer_begin;
     p.nb_src = plan->src.num_blocks;
     p.nb_dst = plan->dst.num_blocks;
     p.heads_src = plan->heads_src;
     p.heads_dst = plan->heads_dst;
+    p.moving_units = g.head_units;
+    if (p.reshape) {  // one unit = the headers of one worker of the finer side; every N-th stays
+        const int n = p.reshape > 0 ? p.reshape : -p.reshape;
+        p.moving_units = g.head_units - g.head_units / n;
+    }
 
-    DeviceInfo dev;
-    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const DeviceInfo dev = cached_device_info();
+    if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     cudaError_t e;
     const KernelOpts& opt = plan->opt.kv;
     const int path = opt.copy_path ? opt.copy_path : kKvDefaults.copy_path;
     const bool token_side = p.src_token_major || p.dst_token_major;
     const bool boxes = path != 1 && token_side && bx.usable && opt.tensor_maps != 1;
     const int64_t items_per_pair = boxes ? (int64_t)p.runs_per_block * bx.sub_runs * bx.tok_groups
-                                         : (int64_t)g.planes * g.head_units * g.row_groups * g.col_chunks;
-    const int64_t max_items = (int64_t)pairs_cap * p.n_layers * items_per_pair;
+                                         : (int64_t)g.planes * p.moving_units * g.row_groups * g.col_chunks;
+    const int64_t max_items = (int64_t)p.pairs_cap * p.n_layers * items_per_pair;
+    if (max_items == 0) return AMOEBA_OK;
     if (path == 1) {
-        // loads in flight per lane x resident CTAs: 8 x 2, 6 x 3 or 4 x 4 and more
         const int per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : kLdstCtasPerSm;
         const int grid = (int)std::min<int64_t>((max_items + 7) / 8, grid_cap(opt, (int64_t)dev.sms * per_sm));
         if (per_sm <= 2) kv_reshard_ldst<8, 2><<<grid, 256, 0, stream>>>(p);
@@ -453,23 +480,13 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
         else kv_reshard_ldst<4, 4><<<grid, 256, 0, stream>>>(p);
         e = cudaGetLastError();
     } else if (boxes) {
-        KvMaps maps;  // encoded per call: the pool addresses are arguments of this call
-        std::memset(&maps, 0, sizeof(maps));
-        if (p.src_token_major)
-            for (int r = 0; r < plan->src.tp; ++r)
-                if (!encode_pool_map(&maps.src[r], src_pools[r], plan->src, plan->src_layer_stride, plan->heads_src,
-                                     plan->vec_bytes, bx))
-                    return AMOEBA_ERR_CUDA;
-        if (p.dst_token_major)
-            for (int r = 0; r < plan->dst.tp; ++r)
-                if (!encode_pool_map(&maps.dst[r], dst_pools[r], plan->dst, plan->dst_layer_stride, plan->heads_dst,
-                                     plan->vec_bytes, bx))
-                    return AMOEBA_ERR_CUDA;
+        KvMaps maps;
+        if (!pool_maps(plan, p, &maps)) return AMOEBA_ERR_CUDA;
         const int stage_bytes = (int)((bx.item_bytes + 127) / 128 * 128);  // tiled copies want 128-byte aligned stages
         const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, stage_bytes);
         const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
         auto kernel = path == 3 ? kv_reshard_pair_box : kv_reshard_bulk_box;
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+        e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)bs.smem);
         if (e == cudaSuccess) {
             kernel<<<grid, bs.threads, bs.smem, stream>>>(p, maps, bs.ring);
             e = cudaGetLastError();
@@ -478,7 +495,7 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
         const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)g.item_bytes);
         const int grid = (int)std::min<int64_t>((max_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
         auto kernel = path == 3 ? kv_reshard_pair : kv_reshard_bulk;
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+        e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)bs.smem);
         if (e == cudaSuccess) {
             kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring);
             e = cudaGetLastError();
@@ -487,6 +504,72 @@ extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
     if (e != cudaSuccess) return AMOEBA_ERR_CUDA;
     count_launch();
     return AMOEBA_OK;
+}
+
+}  // namespace amoeba
+
+extern "C" amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools,
+                                           void* const* dst_pools, const int32_t* d_pairs, const int32_t* d_num_pairs,
+                                           int32_t pairs_cap, int32_t layer_begin, int32_t layer_end, int32_t* d_status,
+                                           void* cuda_stream) {
+    if (!plan || !src_pools || !dst_pools || !d_pairs || !d_num_pairs || !d_status || pairs_cap < 0)
+        return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_model& m = plan->src.model;
+    if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_pairs) % 8) return AMOEBA_ERR_ALIGNMENT;
+    KvParams p{};
+    for (int r = 0; r < plan->src.tp; ++r) {
+        if (!src_pools[r]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(src_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        p.src[r] = static_cast<const char*>(src_pools[r]);
+    }
+    for (int r = 0; r < plan->dst.tp; ++r) {
+        if (!dst_pools[r]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(dst_pools[r]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        for (int q = 0; q < plan->src.tp; ++q)  // out of place: a destination pool is never a source pool
+            if (dst_pools[r] == src_pools[q]) return AMOEBA_ERR_INVALID_ARG;
+        p.dst[r] = static_cast<char*>(dst_pools[r]);
+    }
+    if (pairs_cap == 0 || layer_begin == layer_end) return AMOEBA_OK;
+    p.pairs = d_pairs;
+    p.num_pairs = d_num_pairs;
+    p.status = d_status;
+    p.pairs_cap = pairs_cap;
+    p.layer_begin = layer_begin;
+    p.n_layers = layer_end - layer_begin;
+    return launch_kv(plan, p, static_cast<cudaStream_t>(cuda_stream));
+}
+
+extern "C" amoeba_status amoeba_reshape_kv_inplace(const amoeba_plan* plan, void* const* pools, const int32_t* d_pairs,
+                                                   const int32_t* d_num_pairs, int32_t pairs_cap, int32_t layer_begin,
+                                                   int32_t layer_end, int32_t* d_status, void* cuda_stream) {
+    if (!plan || !pools || !d_pairs || !d_num_pairs || !d_status || pairs_cap < 0) return AMOEBA_ERR_INVALID_ARG;
+    const int f = reshape_factor(plan);
+    if (!f) return AMOEBA_ERR_UNSUPPORTED;
+    const int n = f > 0 ? f : -f;
+    const amoeba_model& m = plan->src.model;
+    if (layer_begin < 0 || layer_end > m.num_layers || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_pairs) % 8) return AMOEBA_ERR_ALIGNMENT;
+    const int fine = std::max(plan->src.tp, plan->dst.tp);
+    KvParams p{};
+    for (int w = 0; w < fine; ++w) {
+        if (!pools[w]) return AMOEBA_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(pools[w]) % 16) return AMOEBA_ERR_ALIGNMENT;
+        for (int v = 0; v < w; ++v)
+            if (pools[v] == pools[w]) return AMOEBA_ERR_INVALID_ARG;  // every worker has its own memory
+    }
+    // the finer side indexes pools directly; worker r of the coarser side lives in pools[r * N]
+    for (int r = 0; r < plan->src.tp; ++r) p.src[r] = static_cast<const char*>(pools[f > 0 ? r * n : r]);
+    for (int r = 0; r < plan->dst.tp; ++r) p.dst[r] = static_cast<char*>(pools[f > 0 ? r : r * n]);
+    if (pairs_cap == 0 || layer_begin == layer_end) return AMOEBA_OK;
+    p.pairs = d_pairs;
+    p.num_pairs = d_num_pairs;
+    p.status = d_status;
+    p.pairs_cap = pairs_cap;
+    p.layer_begin = layer_begin;
+    p.n_layers = layer_end - layer_begin;
+    p.reshape = f;
+    return launch_kv(plan, p, static_cast<cudaStream_t>(cuda_stream));
 }
 
 static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void* const* pools, const uint8_t* d_live,
@@ -528,15 +611,15 @@ static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void
     p.n_pairs = n * (n - 1) / 2;
     p.split = split ? 1 : 0;
 
-    DeviceInfo dev;
-    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    const DeviceInfo dev = cached_device_info();
+    if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int path = opt.copy_path == 2 ? 2 : 3;  // a swap needs a staged copy: the rings only
     const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)(2 * p.chunk_bytes));
     const int64_t n_items = (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
     const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
     auto kernel = path == 3 ? kv_merge_pair : kv_merge_bulk;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)bs.smem);
     if (e == cudaSuccess) {
         kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring, d_status);
         e = cudaGetLastError();

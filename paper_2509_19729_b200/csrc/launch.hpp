@@ -1,6 +1,7 @@
 // Launch-shape helpers shared by the kernel launchers.
 #pragma once
 #include <algorithm>
+#include <mutex>
 #include <cuda_runtime.h>
 
 #include "copy_engine.cuh"
@@ -33,12 +34,55 @@ inline bool device_info(DeviceInfo* out) {
     return out->sms > 0;
 }
 
+// The same, looked up once per device ordinal and remembered (the attributes of a device do not change); sms == 0 if
+// the query failed.  Only cudaGetDevice runs per call.
+constexpr int kMaxDevices = 64;
+inline DeviceInfo cached_device_info() {
+    static DeviceInfo cache[kMaxDevices];
+    static bool known[kMaxDevices];
+    static std::mutex mutex;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DeviceInfo{};
+    DeviceInfo d;
+    if (dev < 0 || dev >= kMaxDevices) return device_info(&d) ? d : DeviceInfo{};
+    std::lock_guard<std::mutex> lock(mutex);
+    if (!known[dev]) {
+        if (!device_info(&d)) return DeviceInfo{};
+        cache[dev] = d;
+        known[dev] = true;
+    }
+    return cache[dev];
+}
+
+// Opt a kernel in to `bytes` of dynamic shared memory, once per (device, kernel) and size: the attribute sticks, so
+// later launches with the same or a smaller size skip the call.
+inline cudaError_t ensure_dynamic_smem(const void* kernel, int bytes) {
+    struct Entry {
+        int dev;
+        const void* kernel;
+        int bytes;
+    };
+    static Entry table[256];
+    static int used = 0;
+    static std::mutex mutex;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mutex);
+    Entry* e = nullptr;
+    for (int i = 0; i < used; ++i)
+        if (table[i].dev == dev && table[i].kernel == kernel) e = &table[i];
+    if (e && e->bytes >= bytes) return cudaSuccess;
+    const cudaError_t rc = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (rc != cudaSuccess) return rc;
+    if (!e && used < 256) e = &table[used++];
+    if (e) *e = Entry{dev, kernel, bytes};
+    return cudaSuccess;
+}
+
 // Persistent grid size: the default (a multiple of the SM count), or the caller's cap when it leaves SMs to other work.
 inline int64_t grid_cap(const KernelOpts& opt, int64_t grid) {
     return opt.max_ctas > 0 ? std::min<int64_t>(grid, opt.max_ctas) : grid;
 }
-
-constexpr int kBarrierBytes = 1024;  // head of dynamic shared memory: up to 128 mbarriers
 
 struct BulkShape {
     RingShape ring;
@@ -64,7 +108,7 @@ inline BulkShape bulk_shape(const DeviceInfo& dev, const KernelOpts& opt, const 
     const int bars_per_ring = path == 3 ? 2 * stages : stages;
     int rings = opt.warps ? opt.warps : def.warps;
     rings = (int)std::min<int64_t>(rings, budget / ((int64_t)stages * stage_bytes));
-    rings = std::min(rings, kBarrierBytes / 8 / bars_per_ring);
+    rings = std::min(rings, kBarrierSlots / bars_per_ring);
     rings = std::max(1, std::min(rings, path == 3 ? 16 : 32));
     b.rings = rings;
     b.threads = 32 * rings * (path == 3 ? 2 : 1);
@@ -73,6 +117,7 @@ inline BulkShape bulk_shape(const DeviceInfo& dev, const KernelOpts& opt, const 
     b.ring.stage_bytes = stage_bytes;
     const int hint = opt.hint ? opt.hint : (def.hint ? def.hint : 1);
     b.ring.hint = hint - 1;
+    b.ring.max_polls = opt.wait_tries;
     b.smem = kBarrierBytes + (size_t)rings * stages * stage_bytes;
     return b;
 }

@@ -3,7 +3,6 @@
 // which byte ranges go from which source worker to which destination worker.  No CUDA in this file.
 #include <algorithm>
 #include <atomic>
-#include <cstdlib>
 #include <new>
 #include <numeric>
 
@@ -195,6 +194,17 @@ int merge_instances(const amoeba_plan* p) {
     return (int)n;
 }
 
+int reshape_factor(const amoeba_plan* p) {
+    const amoeba_layout &s = p->src, &d = p->dst;
+    if (s.kv_order != AMOEBA_KV_HEAD_MAJOR || d.kv_order != AMOEBA_KV_HEAD_MAJOR) return 0;
+    if (p->src_layer_stride != p->dst_layer_stride) return 0;
+    if (d.tp > s.tp && d.tp % s.tp == 0 && (int64_t)d.num_blocks == (int64_t)s.num_blocks * (d.tp / s.tp))
+        return d.tp / s.tp;
+    if (s.tp > d.tp && s.tp % d.tp == 0 && (int64_t)s.num_blocks == (int64_t)d.num_blocks * (s.tp / d.tp))
+        return -(s.tp / d.tp);
+    return 0;
+}
+
 struct Range {
     int64_t lo, hi;
 };
@@ -268,9 +278,7 @@ using namespace amoeba;
 
 extern "C" {
 
-amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* dst, amoeba_plan** out) {
-    if (!src || !dst || !out) return AMOEBA_ERR_INVALID_ARG;
-    *out = nullptr;
+static amoeba_status plan_create(const amoeba_layout* src, const amoeba_layout* dst, amoeba_plan** out) {
     amoeba_status st = check_layout(*src);
     if (st != AMOEBA_OK) return st;
     st = check_layout(*dst);
@@ -337,10 +345,6 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
         p->weight_bytes_per_layer += d.row_bytes * d.n_rows;
     }
 
-    if (const char* env = std::getenv("AMOEBA_COPY_PATH")) {  // "ldst", "bulk" (ring per warp), "pair"
-        const int path = env[0] == 'l' ? 1 : env[0] == 'b' || env[0] == 't' ? 2 : env[0] == 'p' ? 3 : 0;
-        p->opt.kv.copy_path = p->opt.w.copy_path = path;
-    }
     st = finalize_chunks(p);
     if (st != AMOEBA_OK) {
         delete p;
@@ -348,6 +352,17 @@ amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* 
     }
     *out = p;
     return AMOEBA_OK;
+}
+
+// The containers of a plan allocate; an allocation failure is reported as a status, never thrown across the C ABI.
+amoeba_status amoeba_plan_create(const amoeba_layout* src, const amoeba_layout* dst, amoeba_plan** out) {
+    if (!src || !dst || !out) return AMOEBA_ERR_INVALID_ARG;
+    *out = nullptr;
+    try {
+        return plan_create(src, dst, out);
+    } catch (...) {
+        return AMOEBA_ERR_NO_MEMORY;
+    }
 }
 
 void amoeba_plan_destroy(amoeba_plan* plan) { delete plan; }
@@ -463,15 +478,26 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
                 if (value > 2) return AMOEBA_ERR_INVALID_ARG;
                 k->tensor_maps = (int)value;
                 break;
+            case AMOEBA_OPT_WAIT_TRIES:
+                if (value > (int64_t(1) << 30)) return AMOEBA_ERR_INVALID_ARG;
+                k->wait_tries = (int)value;
+                break;
             default:
                 return AMOEBA_ERR_INVALID_ARG;
         }
     }
-    amoeba_status st = finalize_chunks(plan);
-    if (st != AMOEBA_OK) {
+    amoeba_status st;
+    try {
+        st = finalize_chunks(plan);
+        if (st != AMOEBA_OK) {
+            plan->opt = old;
+            finalize_chunks(plan);
+        }
+    } catch (...) {
         plan->opt = old;
-        finalize_chunks(plan);
+        return AMOEBA_ERR_NO_MEMORY;
     }
+    plan->bump_generation();
     return st;
 }
 
@@ -489,6 +515,17 @@ amoeba_status amoeba_merge_bytes(const amoeba_plan* plan, int64_t n_live_blocks,
     if (!n) return AMOEBA_ERR_UNSUPPORTED;
     const amoeba_model& m = plan->src.model;
     // one old block on all a workers of its instance: Hkv headers; (n-1)/n of them move, read once and written once
+    *kv_bytes_rw = 2 * n_live_blocks * m.num_layers * (m.num_kv_heads / n) * (n - 1) * plan->unit_bytes;
+    return AMOEBA_OK;
+}
+
+amoeba_status amoeba_reshape_bytes(const amoeba_plan* plan, int64_t n_live_blocks, int64_t* kv_bytes_rw) {
+    if (!plan || !kv_bytes_rw || n_live_blocks < 0) return AMOEBA_ERR_INVALID_ARG;
+    const int f = reshape_factor(plan);
+    if (!f) return AMOEBA_ERR_UNSUPPORTED;
+    const int n = f > 0 ? f : -f;
+    const amoeba_model& m = plan->src.model;
+    // of the N header groups of a block one stays where it is; the others are read once and written once
     *kv_bytes_rw = 2 * n_live_blocks * m.num_layers * (m.num_kv_heads / n) * (n - 1) * plan->unit_bytes;
     return AMOEBA_OK;
 }
@@ -524,6 +561,7 @@ const char* amoeba_status_string(amoeba_status s) {
         case AMOEBA_ERR_CUDA: return "CUDA runtime error";
         case AMOEBA_ERR_TIMEOUT: return "on-device wait for a bulk copy ran out";
         case AMOEBA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch array";
+        case AMOEBA_ERR_NO_MEMORY: return "host memory allocation failed";
     }
     return "unknown status";
 }

@@ -1,5 +1,6 @@
 // Internal definitions shared by the host planner and the kernel launchers of the re-layout library.
 #pragma once
+#include <atomic>
 #include <cstdint>
 #include <vector>
 
@@ -53,6 +54,7 @@ struct KernelOpts {
     int hint = 0;         // 1 + bit mask: bit 0 loads evict-first, bit 1 stores evict-first (0 = default)
     int max_ctas = 0;     // cap on the persistent grid (0 = none): leaves SMs free for kernels that run beside the copy
     int tensor_maps = 0;  // KV only: 1 = row copies on token-first sides, 2 = tensor-map boxes (0 = default)
+    int wait_tries = 0;   // polls of one bounded mbarrier wait before the kernel gives up (0 = default)
 };
 
 struct Options {
@@ -98,11 +100,20 @@ struct amoeba_plan {
     int32_t items_per_layer;
     int64_t weight_bytes_per_layer;  // one copy (read side)
     amoeba::Options opt;
+    // Bumped whenever the options change: anything a launcher has cached for this plan (encoded tensor maps) is
+    // re-derived when its generation differs.
+    std::atomic<uint64_t> generation{1};
+    void bump_generation() { generation.fetch_add(1, std::memory_order_relaxed); }
+    struct LaunchCache* cache = nullptr;  // owned; created on first use by the KV launcher
+    ~amoeba_plan();
 };
 
 namespace amoeba {
 // Number of instances N if the plan describes an in-place merge of N instances (see amoeba.h), else 0.
 int merge_instances(const amoeba_plan* p);
+// In-place block reshaping of one instance: +N if the destination has N times the source's TP degree and blocks,
+// -N if the source has N times the destination's, 0 if the plan describes neither.
+int reshape_factor(const amoeba_plan* p);
 // One public weight descriptor in kernel form; *item is the running count of work items.
 WDescDev chunk_desc(const amoeba_weight_desc& d, int64_t cap, int64_t* item);
 // Re-derives chunk sizes and the per-descriptor work-item split from plan->opt.

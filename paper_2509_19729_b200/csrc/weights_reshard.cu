@@ -79,15 +79,10 @@ __global__ void __launch_bounds__(1024) w_reshard_bulk(const __grid_constant__ W
 __global__ void __launch_bounds__(1024) w_reshard_pair(const __grid_constant__ WParams p, const RingShape rs,
                                                         int32_t* status) {
     extern __shared__ __align__(128) char smem[];
-    const int warp = threadIdx.x >> 5, ring = warp >> 1, role = warp & 1, nrings = blockDim.x >> 6;
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem) + ring * 2 * rs.stages;
-    uint64_t* empty = full + rs.stages;
-    char* stages = smem + kBarrierBytes + (int64_t)ring * rs.stages * rs.stage_bytes;
-    if (role == 0 && (threadIdx.x & 31) == 0) pair_ring_init(full, empty, rs.stages);
-    __syncthreads();
+    const PairRing r = pair_ring_setup(smem, rs);
     const WItems items{p};
-    const bool ok = pair_bulk_ring(role, items, items.count(), (int64_t)blockIdx.x * nrings + ring,
-                                   (int64_t)gridDim.x * nrings, stages, full, empty, rs);
+    const bool ok = pair_bulk_ring(r.role, items, items.count(), (int64_t)blockIdx.x * r.nrings + r.ring,
+                                   (int64_t)gridDim.x * r.nrings, r.stages, r.full, r.empty, r.abort, rs);
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
@@ -101,8 +96,8 @@ static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDe
                                   cudaStream_t stream) {
     const int n_descs = (int)descs.size();
     if (layer_begin == layer_end || n_descs == 0 || items_per_layer == 0) return AMOEBA_OK;
-    DeviceInfo dev;
-    if (!device_info(&dev)) return AMOEBA_ERR_CUDA;
+    const DeviceInfo dev = cached_device_info();
+    if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     const KernelOpts& opt = plan->opt.w;
     const int path = opt.copy_path ? opt.copy_path : kWDefaults.copy_path;
     int stage_bytes = 16;
@@ -143,7 +138,7 @@ static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDe
             const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings,
                                                     grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
             auto kernel = path == 3 ? w_reshard_pair : w_reshard_bulk;
-            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bs.smem);
+            e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)bs.smem);
             if (e == cudaSuccess) {
                 kernel<<<grid, bs.threads, bs.smem, stream>>>(p, bs.ring, d_status);
                 e = cudaGetLastError();
@@ -180,7 +175,7 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
             const void* t = slots(&dst[(size_t)dst_rank * L + l])[d.dst_slot % kNumTensors];
             if (!t && left_out(dst_rank, l)) continue;
             const void* s = slots(&src[(size_t)(d.src_slot / kNumTensors) * L + l])[d.src_slot % kNumTensors];
-            if (!s || !t) return AMOEBA_ERR_INVALID_ARG;
+            if (!s || !t || s == t) return AMOEBA_ERR_INVALID_ARG;  // out of place: never the same buffer
             if (reinterpret_cast<uintptr_t>(s) % 16 || reinterpret_cast<uintptr_t>(t) % 16) return AMOEBA_ERR_ALIGNMENT;
         }
     return launch_descs(plan, plan->wdev, plan->items_per_layer, src, a, dst, b, L, layer_begin, layer_end, d_status,
@@ -196,9 +191,9 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
 //   columns (o_proj, down_proj): row j of the kept column range moves from j*w + keep*w/N to j*w/N; rows are done in
 //     waves [0,1), [1,N), [N,N^2), ...: the destination of wave [m, N*m) ends at byte m*w, where its sources begin.
 // Phases are separate launches on the stream; within a phase all copies are disjoint.
-extern "C" amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
-                                                        const int32_t* keep, int32_t layer_begin, int32_t layer_end,
-                                                        int32_t* d_status, void* cuda_stream) {
+static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
+                                             const int32_t* keep, int32_t layer_begin, int32_t layer_end,
+                                             int32_t* d_status, void* cuda_stream) {
     if (!plan || !bufs || !keep || !d_status) return AMOEBA_ERR_INVALID_ARG;
     const amoeba_layout &sl = plan->src, &dl = plan->dst;
     const amoeba_model& m = sl.model;
@@ -298,4 +293,15 @@ extern "C" amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan,
         if (st != AMOEBA_OK) return st;
     }
     return AMOEBA_OK;
+}
+
+// The phase lists are host containers: an allocation failure becomes a status, no exception leaves the library.
+extern "C" amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
+                                                        const int32_t* keep, int32_t layer_begin, int32_t layer_end,
+                                                        int32_t* d_status, void* cuda_stream) {
+    try {
+        return compact_weights_inplace(plan, bufs, keep, layer_begin, layer_end, d_status, cuda_stream);
+    } catch (...) {
+        return AMOEBA_ERR_NO_MEMORY;
+    }
 }

@@ -140,6 +140,62 @@ class Session:
 
 
 
+class ReshapeSession:
+    """Buffers of the in-place block reshaping of ONE instance between TP=a (NB blocks) and TP=N*a (NB*N blocks).
+
+    pools[w] is worker w of the TP=N*a side; worker r of the TP=a side is pools[r*N].  direction "split": the tables
+    are over NB ids and the instance goes a -> N*a; "merge": over NB*N ids and it goes N*a -> a."""
+
+    def __init__(self, model: dict, N: int, a: int, NB: int, num_seqs: int, max_blocks_per_seq: int, pairs_cap: int,
+                 direction: str = "split", kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0"):
+        assert direction in ("split", "merge")
+        self.model, self.N, self.a, self.NB, self.direction = model, N, a, NB, direction
+        self.device = dev = torch.device(device)
+        coarse = A.make_layout(model, a, NB, block_tokens)
+        fine = A.make_layout(model, N * a, NB * N, block_tokens)
+        self.src_layout, self.dst_layout = (coarse, fine) if direction == "split" else (fine, coarse)
+        self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
+        self.L = model["L"]
+        self.kv_layers = self.L if kv_layers is None else kv_layers
+        self.num_seqs, self.maxb, self.pairs_cap = num_seqs, max_blocks_per_seq, pairs_cap
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.src_bt = torch.full((num_seqs, max_blocks_per_seq), -1, **i32)
+        self.dst_bt = torch.full((num_seqs, max_blocks_per_seq), -2, **i32)
+        self.seq_lens = torch.zeros(num_seqs, **i32)
+        self.pairs = torch.full((max(pairs_cap, 1), 2), -3, **i32)
+        self.num_pairs = torch.zeros(1, **i32)
+        self.free_count = torch.zeros(1, **i32)
+        self.status = torch.zeros(1, **i32)
+        self.free_mask = torch.full((self.dst_layout.num_blocks,), 7, dtype=torch.uint8, device=dev)
+        self.workspace_bytes = A.amoeba_rewrite_workspace_bytes(self.plan, num_seqs, 0)
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=dev)
+        per_layer = A.amoeba_layout_kv_pool_bytes(coarse) // self.L
+        self.pools = [torch.empty(per_layer * self.kv_layers, dtype=torch.uint8, device=dev) for _ in range(N * a)]
+
+    def set_tables(self, seq_lens, src_bt) -> None:
+        self.seq_lens.copy_(torch.as_tensor(seq_lens, dtype=torch.int32))
+        self.src_bt.copy_(torch.as_tensor(src_bt, dtype=torch.int32))
+
+    def reshape_block_tables(self, stream=None) -> None:
+        A.amoeba_reshape_block_tables(self.plan, self.src_bt, self.seq_lens, self.num_seqs, self.maxb, self.dst_bt,
+                                      self.pairs, self.pairs_cap, self.num_pairs, self.free_mask, self.free_count,
+                                      self.status, self.workspace, self.workspace_bytes, stream)
+
+    def reshape_kv(self, stream=None, layer_begin: int = 0, layer_end: Optional[int] = None) -> None:
+        A.amoeba_reshape_kv_inplace(self.plan, self.pools, self.pairs, self.num_pairs, self.pairs_cap, layer_begin,
+                                    self.kv_layers if layer_end is None else layer_end, self.status, stream)
+
+    def step(self, stream=None) -> None:
+        self.reshape_block_tables(stream)
+        self.reshape_kv(stream)
+
+    def set_option(self, option: int, value: int) -> None:
+        A.amoeba_plan_set_option(self.plan, option, value)
+
+    def bytes_rw(self, n_live: int) -> int:
+        return A.amoeba_reshape_bytes(self.plan, n_live) * self.kv_layers // self.L
+
+
 class MergeSession:
     """Buffers of one in-place merge of N instances of TP=a into one instance of TP=N*a on one GPU.
 

@@ -634,3 +634,60 @@ def test_weights_compaction_host_errors():
     p3 = A.amoeba_plan_create(A.make_layout(m, 4, 4), A.make_layout(m, 2, 4))  # scale-down is not a compaction
     assert status_of(lambda: A.amoeba_compact_weights_inplace(p3, buf(A.make_layout(m, 4, 4)), [0] * 4, 0, 1, z)) \
         == A.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_free_list_that_names_an_id_twice(path):
+    """Two blocks must never share a destination: the first block (in sequence, block order) given an id keeps it,
+    a later one gets none (entry -1, pair (-1,-1), BAD_BLOCK_ID) and is not copied."""
+    lens = [160, 48, 300]
+    base = make_case(GQA, 2, 1, lens, weights=False, seed=6)
+    free = base.free_list.copy()
+    free[7] = free[2]
+    free[20] = free[2]
+    free[11] = free[30]  # the later entry (30) loses
+    c = make_case(GQA, 2, 1, lens, weights=False, seed=6, free_override=(free, None))
+    assert c.exp_status == 5 and (c.exp_pairs[[7, 20, 30]] == -1).all() and c.exp_pairs[11, 1] == free[30]
+    check_case(c, run_case(c, path))
+
+
+def test_out_of_place_calls_refuse_a_buffer_on_both_sides():
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 2, 2, [40], seed=1)
+    s = run_case(c, PAIR)
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_reshard_kv(s.plan, s.src_pools, [s.dst_pools[0], s.src_pools[1]], s.pairs, s.num_pairs, s.pairs_cap,
+                            0, 1, s.status)
+    assert e.value.status == A.ERR_INVALID_ARG
+    dst = [[dict(d) for d in r] for r in s.dst_w]
+    dst[1][0]["o"] = s.src_w[1][0]["o"]
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_reshard_weights(s.plan, s.src_w, dst, 0, 1, s.status)
+    assert e.value.status == A.ERR_INVALID_ARG
+    check_case(c, s)  # the refused calls launched nothing
+
+
+@pytest.mark.parametrize("path", [BULK, PAIR])
+def test_wait_budget_running_out_is_reported_and_the_next_call_is_exact(path):
+    """Every wait of a copy kernel on its own bulk copies is bounded.  With a budget of ONE non-blocking poll the
+    first wait of every ring runs out before its (healthy) load can have landed: the kernel must record TIMEOUT, let
+    the copies it has in flight land, and return - nothing outside the destination buffers is touched, the context
+    stays usable, and the same call with the default budget then gives the exact result."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    c = make_case(GQA, 2, 4, [300, 77, 1024, 5, 640], seed=12)
+    s = run_case(c, path, options=[(A.OPT_WAIT_TRIES, 1)])
+    assert int(s.status.item()) == A.ERR_TIMEOUT
+    for t, e in zip(s.src_pools, c.src_pools):  # sources are never written
+        assert np.array_equal(t.cpu().numpy().view(np.uint16), e)
+    for t, e in zip(s.dst_pools, c.exp_dst_pools):  # every destination word is either untouched or already right
+        got = t.cpu().numpy().view(np.uint16)
+        assert np.all((got == e) | (got == 0xA5A5))
+    s.set_option(A.OPT_WAIT_TRIES, 0)
+    s.status.zero_()
+    s.step()
+    torch.cuda.synchronize()
+    check_case(c, s)

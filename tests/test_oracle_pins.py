@@ -580,3 +580,19 @@ def test_transform_with_layer_strides_equals_dense_transform(oracle, a, b, so, d
     direct = oracle.kv_shard(KV, m, T, b, NB_b, seq_lens, bt_b, order=do, layer_stride=sb, fill=0xA5A5)
     for x, y in zip(dst_s, direct):
         assert np.array_equal(x, y)
+
+
+def test_assign_blocks_refuses_an_id_handed_out_twice(oracle):
+    """Brute force on a tiny input: a free list that names id 7 twice.  The first block that is given 7 keeps it, the
+    later one gets no destination (entry -1, pair (-1,-1)), so no two blocks ever share a destination block."""
+    T, NB = 16, 32
+    seq_lens = [40, 16, 20]                       # 3 + 1 + 2 blocks
+    bt, nblk = _state(seq_lens, T, NB)
+    free = np.array([3, 7, 9, 7, 11, 12, 13], np.int32)
+    dst_bt, pairs, n, left, st = oracle.assign_blocks(seq_lens, T, bt, NB, NB, free_list=free)
+    assert st == oracle.BAD_BLOCK_ID and n == 6 and left == 1
+    flat = [int(dst_bt[s, i]) for s in range(3) for i in range(nblk[s])]
+    assert flat == [3, 7, 9, -1, 11, 12]
+    assert tuple(pairs[3]) == (-1, -1) and tuple(pairs[1]) == (int(bt[0, 1]), 7)
+    given = [x for x in flat if x >= 0]
+    assert len(set(given)) == len(given)
