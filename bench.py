@@ -32,12 +32,14 @@ DEFAULT_CONFIG = "llama3_8b_1to4"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes (read + written) per algorithmic byte of kv_reshard_pair (the default copy path), from the ncu capture
-# summarised in profiles/kv_reshard_pair_llama3_8b_1to4_1layer.md: taken on a one-layer slice and scaled by the
-# bytes of a full launch (every layer repeats the same work on disjoint memory).  Only quoted for that workload
-# with default kernel options.
-NCU_KV_TRAFFIC_RATIO = 0.9895
+# DRAM bytes (read + written) per algorithmic byte of kv_reshard_pair (the default copy path), from an ncu capture of
+# a one-layer slice of the workload below, scaled by the bytes of a full launch (every layer repeats the same work on
+# disjoint memory).  It is a stored counter reading, not something this script measures: the line says so in
+# "traffic_source", and it is only quoted for that workload with default kernel options (None = no reading for the
+# current kernel).
+NCU_KV_TRAFFIC_RATIO = None
 NCU_KV_TRAFFIC_CONFIG = "llama3_8b_1to4"
+NCU_KV_TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1-layer slice, scaled by units processed"
 
 
 def peaks():
@@ -136,10 +138,14 @@ def barrier(world: int):
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(cfg_name: str, kv_layers=4, n_seqs=None, w_layers=4, threads=1):
+def oracle_sample(cfg_name: str, kv_layers=4, n_seqs=None, w_layers=4, threads=1, dist="words"):
     """A bounded sample of the workload for the CPU oracle: the first n_seqs sequences (None = all) over kv_layers
-    layers of KV, and w_layers layers of weights; values are uniform 16-bit words (the movement does not depend on
-    them).  Returns a closure that runs one oracle a->b pass and the bytes it moves."""
+    layers of KV, and w_layers layers of weights; values are uniform 16-bit words or a counter pattern (the movement
+    does not depend on them).  Returns a closure that runs one oracle a->b pass and the bytes it moves.  threads > 1:
+    the oracle's own layer loop runs on that many OpenMP threads for the KV cache, and the weight layers (one oracle
+    call each) are issued from as many host threads - one thread per layer, as far as there are layers."""
+    from concurrent.futures import ThreadPoolExecutor
+
     import oracle
 
     oracle.build()
@@ -151,13 +157,13 @@ def oracle_sample(cfg_name: str, kv_layers=4, n_seqs=None, w_layers=4, threads=1
     m_kv = dict(m, L=kv_layers)
     st = wl.draw_kv_state(cfg, name=cfg_name, seq_lens=lens)
     G = int(st["blocks_per_seq"].sum()) * T
-    KV = wl.draw_kv_logical(dict(cfg, model=m_kv), G, range(kv_layers), dist="words")
+    KV = wl.draw_kv_logical(dict(cfg, model=m_kv), G, range(kv_layers), dist=dist)
     src = oracle.kv_shard(KV, m_kv, T, a, st["NB_src"], lens, st["src_bt"])
     del KV
     free = dict(free_list=st.get("dst_free_list"), free_mask=st.get("dst_free_mask"))
     dst = [np.full(kv_layers * oracle.pool_elems_per_layer(m_kv, T, b, st["NB_dst"]), 0xA5A5, np.uint16)
            for _ in range(b)]
-    W = [oracle.weights_shard(wl.draw_weights_logical(cfg, l, dist="words"), m, a) for l in range(w_layers)]
+    W = [oracle.weights_shard(wl.draw_weights_logical(cfg, l, dist=dist), m, a) for l in range(w_layers)]
     Wd = [oracle.empty_shards(m, b) for _ in range(w_layers)]
     e = 2
     kv_bytes = 2 * st["n_live"] * kv_layers * m["Hkv"] * 2 * T * m["D"] * e
@@ -168,8 +174,12 @@ def oracle_sample(cfg_name: str, kv_layers=4, n_seqs=None, w_layers=4, threads=1
         dst_bt, pairs, n, left, status = oracle.assign_blocks(lens, T, st["src_bt"], st["NB_src"], st["NB_dst"], **free)
         assert status == 0
         oracle.kv_transform(m_kv, T, lens, a, st["NB_src"], st["src_bt"], src, b, st["NB_dst"], dst_bt, dst)
-        for l in range(w_layers):
-            oracle.weights_transform(W[l], m, a, b, dst_shards=Wd[l])
+        if threads > 1:  # the C calls release the interpreter lock: one host thread per weight layer
+            with ThreadPoolExecutor(max_workers=min(threads, w_layers)) as pool:
+                list(pool.map(lambda l: oracle.weights_transform(W[l], m, a, b, dst_shards=Wd[l]), range(w_layers)))
+        else:
+            for l in range(w_layers):
+                oracle.weights_transform(W[l], m, a, b, dst_shards=Wd[l])
 
     desc = (f"{cfg_name}: first {len(lens)} of {cfg['S']} sequences ({st['n_live']} blocks) x {kv_layers} of "
             f"{m['L']} KV layers + {w_layers} of {m['L']} weight layers")
@@ -227,6 +237,37 @@ def run_reference(args, rank, world):
     }))
 
 
+def cpu_baseline(cfg_name: str) -> dict:
+    """The oracle as it stands on the host cores, on bounded samples of the workload: once on one thread, once with
+    one thread per layer over all cores.  The top-level value is the all-cores one; `cores` = threads it used."""
+    run, nbytes, desc = oracle_sample(cfg_name)
+    t0 = time.perf_counter()
+    run()
+    dt1 = time.perf_counter() - t0
+    one = {"value": nbytes / dt1 / 1e9, "unit": "GB/s", "cores": 1, "sample": desc, "seconds": dt1}
+    del run
+    cores = os.cpu_count() or 1
+    cfg = wl.CONFIGS[cfg_name]
+    L_kv = cfg.get("kv_layers") or cfg["model"]["L"]
+    threads = max(1, min(cores, L_kv))
+    w_threads = max(1, min(threads, 8))  # weight layers in the sample (each is hundreds of MB of host memory)
+    # about the same number of bytes as the one-thread sample, spread over `threads` layers: fewer sequences per layer
+    n_seqs = max(1, cfg["S"] * 4 // threads)
+    runN, nbytesN, descN = oracle_sample(cfg_name, kv_layers=threads, n_seqs=n_seqs, w_layers=w_threads,
+                                         threads=threads, dist="counter")
+    t0 = time.perf_counter()
+    runN()
+    dtN = time.perf_counter() - t0
+    import oracle
+
+    oracle.set_threads(1)
+    allc = {"value": nbytesN / dtN / 1e9, "unit": "GB/s", "cores": threads, "host_cores": cores,
+            "threads_kv": threads, "threads_weights": w_threads, "sample": descN, "seconds": dtN}
+    return {"value": allc["value"], "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": descN + f"; {threads} threads (one per KV layer), {w_threads} for the weight layers",
+            "seconds": dtN, "one_thread": one, "all_cores": allc}
+
+
 # ------------------------------------------------------------------------------------------------ GPU leg
 KV_ORDERS = {"head": (0, 0), "token": (1, 1), "token2head": (1, 0), "head2token": (0, 1)}  # (source, destination)
 
@@ -260,6 +301,155 @@ def build_session(cfg_name: str, device, layers=None, kv=True, weights=True, see
             p.fill_(0xA5)
     torch.cuda.synchronize()
     return s, st
+
+
+def measure_config(cfg_name: str, device, steps: int = 5, warmup: int = 3) -> dict:
+    """Device time of the KV and weight calls of one benchmark configuration (default kernel options, all layers the
+    configuration holds), for the per-configuration table of the bench line.  The buffers are left as allocated:
+    the time of a copy does not depend on the values."""
+    import torch
+
+    s, st = build_session(cfg_name, device, fill=False)
+    kv_bytes, w_bytes = s.bytes_rw(st["n_live"])
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        s.status.zero_()
+        s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    marks = []
+    for _ in range(steps):
+        m = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        m[0].record(stream)
+        s.rewrite_block_tables()
+        m[1].record(stream)
+        s.reshard_kv()
+        m[2].record(stream)
+        s.reshard_weights()
+        m[3].record(stream)
+        marks.append(m)
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    bt_ms, kv_ms, w_ms = (statistics.mean(m[i].elapsed_time(m[i + 1]) for m in marks) for i in range(3))
+    peak, _ = peaks()
+    cfg = wl.CONFIGS[cfg_name]
+    out = {"tp": f"{cfg['a']}->{cfg['b']}", "kv_layers": s.kv_layers, "layers": s.L, "live_blocks": st["n_live"],
+           "tables_us": bt_ms * 1e3, "kv_ms": kv_ms, "kv_gbs": kv_bytes / kv_ms / 1e6, "kv_frac": kv_bytes / kv_ms / 1e6 / peak,
+           "w_ms": w_ms, "w_gbs": w_bytes / w_ms / 1e6, "w_frac": w_bytes / w_ms / 1e6 / peak, "steps": steps}
+    del s
+    torch.cuda.empty_cache()
+    return out
+
+
+def build_reshape_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, fill=True, budget_gib=150.0):
+    """One instance reshaped in place between TP=a and TP=b (b = N*a: split; a = N*b: merge back) with the
+    configuration's sequences.  Every worker of the finer side has a pool of the coarser side's capacity, so the
+    layer count is cut to what fits `budget_gib` of device memory (stated in the bench line)."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+    from paper_2509_19729_b200.session import ReshapeSession
+
+    cfg = wl.CONFIGS[cfg_name]
+    m = dict(cfg["model"])
+    a, b = cfg["a"], cfg["b"]
+    direction = "split" if b > a else "merge"
+    N, coarse = max(a, b) // min(a, b), min(a, b)
+    st = wl.draw_kv_state(cfg, seed=seed, name=cfg_name)
+    NB = st["NB_src"]                                   # blocks of the coarser side
+    per_layer = A.amoeba_layout_kv_pool_bytes(A.make_layout(m, coarse, NB)) // m["L"]
+    fit = int(budget_gib * 2**30 // (per_layer * N * coarse))
+    kv_layers = max(1, min(cfg.get("kv_layers") or m["L"], fit, layers or m["L"]))
+    m["L"] = kv_layers
+    src_bt = st["src_bt"] if direction == "split" else np.where(st["src_bt"] >= 0, st["src_bt"] * N, -1)
+    s = ReshapeSession(m, N, coarse, NB, cfg["S"], st["maxb"], st["n_live"], direction=direction, device=device)
+    s.set_tables(st["seq_lens"], src_bt.astype(np.int32))
+    if fill:
+        for i, p in enumerate(s.pools):
+            wl.hash_fill_(p, seed, 600 + i)
+    torch.cuda.synchronize()
+    return s, st
+
+
+def run_reshape(args, rank, world, local):
+    """In-place block reshaping of one instance: one step = the reshaped block table + the KV migration of every
+    header group that leaves its worker.  (Each step re-reads the same source segments: the old workers' memory is
+    never written by a split.)"""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    cfg = wl.CONFIGS[args.config]
+    s, st = build_reshape_session(args.config, device, layers=args.layers)
+    for opt, val in ((A.OPT_COPY_PATH, args.copy_path), (A.OPT_CHUNK_BYTES, args.chunk), (A.OPT_STAGES, args.stages),
+                     (A.OPT_CTAS_PER_SM, args.ctas_per_sm), (A.OPT_MAX_CTAS, args.max_ctas)):
+        if val:
+            s.set_option(opt, val)
+    for item in args.opt:
+        name, val = item.split("=")
+        s.set_option(getattr(A, "OPT_" + name.upper()), int(val))
+    nbytes = s.bytes_rw(st["n_live"])
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(args.warmup):
+        s.status.zero_()
+        s.step()
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0, f"device status {int(s.status.item())}"
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = A.amoeba_launch_count()
+    marks = []
+    t_begin, t_end = ev(), ev()
+    torch.cuda.synchronize()
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        m3 = [ev() for _ in range(3)]
+        m3[0].record(stream)
+        s.reshape_block_tables()
+        m3[1].record(stream)
+        s.reshape_kv()
+        m3[2].record(stream)
+        marks.append(m3)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    barrier(world)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0
+    sec = t_begin.elapsed_time(t_end) / 1e3 / args.steps
+    bt_ms = statistics.mean(m3[0].elapsed_time(m3[1]) for m3 in marks)
+    kv_ms = statistics.mean(m3[1].elapsed_time(m3[2]) for m3 in marks)
+    sec_all, bytes_all = aggregate(world, sec, nbytes, device)
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    kv_gbs = nbytes / (kv_ms / 1e3) / 1e9
+    N = max(cfg["a"], cfg["b"]) // min(cfg["a"], cfg["b"])
+    full = nbytes * N // (N - 1)
+    print(json.dumps({
+        "metric": METRIC, "value": bytes_all / sec_all / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']} in place (one instance)",
+                   "kv_layers": s.kv_layers, "layers_of_model": cfg["model"]["L"], "sequences": cfg["S"],
+                   "live_blocks": st["n_live"], "block_tokens": wl.BLOCK_TOKENS, "kv_bytes_rw": nbytes,
+                   "kv_bytes_rw_out_of_place": full, "weight_bytes_rw": 0,
+                   "pool_bytes": sum(p.numel() for p in s.pools),
+                   "note": "every worker of the finer side holds a pool of the coarser side's capacity; the layer "
+                           "count is what fits one GPU",
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
+        "phases_ms": {"reshape_block_tables": bt_ms, "reshape_kv_inplace": kv_ms},
+        "phases_gbs": {"reshape_kv_inplace": kv_gbs},
+        "roofline": {"kernel": "kv_reshard_pair", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": None,
+    }))
 
 
 def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, fill=True):
@@ -297,7 +487,8 @@ def build_merge_copy_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT
     st = wl.draw_merge_state(cfg, seed=seed, name=cfg_name)
     NB_dst = st["n_live"] + max(st["n_live"] // 64, 1)
     free = wl.rng(seed, "merge_dst_blocks", *cfg_name.encode()).permutation(NB_dst).astype(np.int32)
-    s = MergeCopySession(m, cfg["N"], cfg["a"], st["NB"], NB_dst, st["seq_lens"], st["src_bt"], free, device=device,
+    s = MergeCopySession(m, cfg["N"], cfg["a"], st["NB"], NB_dst, st["seq_lens"], st["src_bt"], free,
+                         st["blocks_per_seq"].sum(axis=1), device=device,
                          src_kv_order=KV_ORDERS[kv_order][0], dst_kv_order=KV_ORDERS[kv_order][1])
     k = 0
     for inst in s.src_pools:
@@ -601,6 +792,11 @@ def main():
                     help="k > 0: transform k layers per call (KV and weights), as when a few layers are transformed "
                          "per inference step; 0 = all layers in one call")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (profiling)")
+    ap.add_argument("--inplace", action="store_true",
+                    help="reshape the one instance in place (block reshaping) instead of copying it into fresh pools; "
+                         "KV cache only, TP degrees must be multiples")
+    ap.add_argument("--no-all-configs", action="store_true",
+                    help="skip the short timing of the other benchmark configurations")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-gib", type=float, default=48.0, help="cap on pinned host memory for the e2e leg")
@@ -614,6 +810,10 @@ def main():
 
     if args.config in wl.MERGE_CONFIGS:
         (run_merge if args.merge_mode == "inplace" else run_merge_copy)(args, rank, world, local)
+        return
+
+    if args.inplace:
+        run_reshape(args, rank, world, local)
         return
 
     import torch
@@ -689,6 +889,14 @@ def main():
     n_seq_layers = (s.L, s.kv_layers, int(s.info.chunk_bytes))
     del s
     torch.cuda.empty_cache()
+    default_run = (args.config == DEFAULT_CONFIG and args.kv_order == "head" and args.layers is None
+                   and not (args.copy_path or args.chunk or args.stages or args.ctas_per_sm or args.max_ctas or args.opt
+                            or args.weight_pad or args.layers_per_call))
+    all_configs = None
+    if default_run and world == 1 and not args.no_all_configs:
+        # the other benchmark configurations, a few steps each, same kernels and options
+        all_configs = {name: measure_config(name, device) for name in wl.CONFIGS
+                       if name not in (args.config, "tiny_2to1")}
     e2e = None if args.no_e2e else run_e2e(args, device, world)
     if rank != 0:
         return
@@ -716,20 +924,22 @@ def main():
                                 "reshard_weights": 100 * w_gbs / NOMINAL_HBM_GBS if w_gbs else None},
         "roofline": {"kernel": "kv_reshard_pair" if not args.copy_path else "kv_reshard", "bound": "hbm", "achieved": kv_gbs, "peak": peak, "unit": "GB/s",
                      "frac": kv_gbs / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": NCU_KV_TRAFFIC_RATIO * kv_bytes if traffic_known else None},
+                     "traffic": NCU_KV_TRAFFIC_RATIO * kv_bytes if traffic_known else None,
+                     "traffic_source": NCU_KV_TRAFFIC_SOURCE if traffic_known else None},
         "roofline_weights": None if not w_gbs else {"kernel": "w_reshard_pair" if not args.copy_path else "w_reshard", "bound": "hbm", "achieved": w_gbs,
                                                     "peak": peak, "unit": "GB/s", "frac": w_gbs / peak},
         "gpu_launches": int(launches), "clocks": clocks, "remeasured_after_slowdown": remeasured,
     }
+    if all_configs is not None:
+        all_configs[args.config] = {"tp": f"{cfg['a']}->{cfg['b']}", "kv_layers": n_seq_layers[1], "layers": n_seq_layers[0],
+                                    "live_blocks": st["n_live"], "tables_us": bt_ms * 1e3, "kv_ms": kv_ms,
+                                    "kv_gbs": kv_gbs, "kv_frac": kv_gbs / peak, "w_ms": w_ms, "w_gbs": w_gbs,
+                                    "w_frac": w_gbs / peak, "steps": args.steps}
+        out["all_configs"] = all_configs
     if e2e is not None:
         out["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        run, nbytes, desc = oracle_sample(args.config)
-        t0 = time.perf_counter()
-        run()
-        dt = time.perf_counter() - t0
-        out["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                               "sample": desc, "seconds": dt}
+        out["cpu_baseline"] = cpu_baseline(args.config)
     print(json.dumps(out))
 
 

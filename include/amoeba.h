@@ -180,9 +180,10 @@ enum {
                                    so a cap below the SM count leaves SMs to kernels running on other streams - the
                                    paper starts its migration on a side stream once enough SMs are free (Sec. 3.1,
                                    Improvement 2) */
-    AMOEBA_OPT_WAIT_TRIES = 9,  /* bulk-copy paths: a kernel's wait on one of its own copies gives up after this many
-                                   non-blocking polls and reports AMOEBA_ERR_TIMEOUT (0 = the default, generous budget).
-                                   For tests of the give-up path; a small value makes healthy copies time out. */
+    AMOEBA_OPT_WAIT_TRIES = 9,  /* bulk-copy paths: value v > 0 makes every wait of a kernel on one of its own copies give
+                                   up after v - 1 non-blocking polls and report AMOEBA_ERR_TIMEOUT (0 = the default,
+                                   generous budget).  For tests of the give-up path: v = 1 gives up at once, so healthy
+                                   copies time out, every time. */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };
@@ -404,13 +405,18 @@ AMOEBA_API amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
  * keep[r] in [0, N) (host array) says which N-th of its shards worker r keeps: it becomes worker r*N + keep[r] of the
  * new partition.  After the call the first bytes of every buffer hold exactly that worker's dense TP = N*a shard
  * (the same bytes amoeba_reshard_weights writes for that worker); the bytes behind it are unspecified leftovers.
- * No second buffer is used; 1/N of the weights is read and written.  The moves are ordered on the stream so that no
- * byte is overwritten before it has been moved (a few launches per call, not one).  Errors: INVALID_ARG (null pointers,
- * keep out of range, layers), UNSUPPORTED (padded layouts, different fused flags, TP not a multiple), ALIGNMENT, CUDA.
+ * No second buffer is used; about 1/N of the weights is read and written (what already sits where it belongs - with
+ * keep[r] = 0 the first section of every buffer and row 0 of o_proj / down_proj - is not touched).  The moves are
+ * ordered on the stream so that no byte is overwritten before it has been moved: one small launch for the first rows
+ * of o_proj / down_proj, then log_N(hidden) - 2 or so launches of the copy kernel (4 for N = 4, 7 for N = 2 at
+ * hidden = 4096).  Errors: INVALID_ARG (null pointers, keep out of range, layers), UNSUPPORTED (padded layouts,
+ * different fused flags, TP not a multiple), ALIGNMENT, CUDA, NO_MEMORY.
+ * amoeba_compact_bytes: the bytes the call reads + writes over all layers for the given keep[] (host arithmetic).
  */
 AMOEBA_API amoeba_status amoeba_compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
                                              const int32_t* keep, int32_t layer_begin, int32_t layer_end,
                                              int32_t* d_status, void* cuda_stream);
+AMOEBA_API amoeba_status amoeba_compact_bytes(const amoeba_plan* plan, const int32_t* keep, int64_t* bytes_rw);
 
 /*
  * amoeba_plan_weight_alias  (Sec. 3.2, Improvement 1: with padded partitions a scale-up needs no weight copy at all)

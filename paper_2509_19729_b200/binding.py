@@ -121,6 +121,7 @@ def _load():
         "amoeba_merge_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
         "amoeba_split_kv_inplace": (I32, [VP, P(VP), VP, I32, I32, VP, VP]),
         "amoeba_compact_weights_inplace": (I32, [VP, P(LayerWeights), P(I32), I32, I32, VP, VP]),
+        "amoeba_compact_bytes": (I32, [VP, P(I32), P(I64)]),
         "amoeba_plan_weight_alias": (I32, [VP, I32, I32, P(I32), P(I64), P(I64)]),
         "amoeba_launch_count": (I64, []),
         "amoeba_status_string": (C.c_char_p, [I32]),
@@ -398,7 +399,15 @@ def amoeba_compact_weights_inplace(plan: Plan, bufs, keep: Sequence[int], layer_
                                                   _stream(stream)), "amoeba_compact_weights_inplace")
 
 
-__all__.append("amoeba_compact_weights_inplace")
+def amoeba_compact_bytes(plan: Plan, keep: Sequence[int]) -> int:
+    """Bytes read + written by ``amoeba_compact_weights_inplace`` over all layers for this ``keep``."""
+    k = (C.c_int32 * len(keep))(*[int(x) for x in keep])
+    out = C.c_int64()
+    _check(_load().amoeba_compact_bytes(plan.handle, k, C.byref(out)), "amoeba_compact_bytes")
+    return out.value
+
+
+__all__ += ["amoeba_compact_weights_inplace", "amoeba_compact_bytes"]
 
 
 def amoeba_plan_weight_alias(plan: Plan, dst_rank: int, tensor: int):

@@ -39,7 +39,7 @@ struct RingShape {
     int32_t lag;          // warp ring: loads lead stores by this many items; pair ring: stores kept in flight
     int32_t stage_bytes;  // bytes per stage
     int32_t hint;         // bit 0: loads evict-first in L2, bit 1: stores evict-first in L2
-    int32_t max_polls;    // 0: default wait budget; > 0: every mbarrier wait gives up after this many non-blocking polls
+    int32_t max_polls;    // 0: default wait budget; v > 0: every mbarrier wait gives up after v - 1 non-blocking polls
 };
 
 // ------------------------------------------------------------------ vector load/store path
@@ -72,39 +72,40 @@ __device__ __forceinline__ void copy_vecs(const uint4* __restrict__ s, uint4* __
 }
 
 // All lanes of a warp call this with the same item: the warp alone moves it, UNROLL 16-byte loads in flight per lane
-// before the first store.  Rows shorter than 512 bytes are dealt to the lanes vector by vector across rows.
+// before the first store.  Rows that are not adjacent in memory are dealt to the lanes vector by vector across rows.
 template <int UNROLL>
-__device__ __forceinline__ void warp_copy_item(const Item& it) {
+__device__ __forceinline__ void warp_copy_rows(const char* __restrict__ src, char* __restrict__ dst, int64_t src_pitch,
+                                               int64_t dst_pitch, int n_rows, int row_bytes) {
     const int lane = threadIdx.x & 31;
-    if (it.n_rows == 1 || (it.src_pitch == it.row_bytes && it.dst_pitch == it.row_bytes)) {
-        copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src), reinterpret_cast<uint4*>(it.dst),
-                          (it.n_rows * it.row_bytes) >> 4, lane, 32);
-    } else if (it.row_bytes >= 512) {
-        for (int r = 0; r < it.n_rows; ++r)
-            copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch),
-                              reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch), it.row_bytes >> 4, lane, 32);
-    } else {
-        const int vpr = it.row_bytes >> 4, n = it.n_rows * vpr;
-        for (int base = 0; base < n; base += 32 * UNROLL) {
-            uint4 v[UNROLL];
+    if (n_rows == 1 || (src_pitch == row_bytes && dst_pitch == row_bytes)) {
+        copy_vecs<UNROLL>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), (n_rows * row_bytes) >> 4,
+                          lane, 32);
+        return;
+    }
+    const int vpr = row_bytes >> 4, n = n_rows * vpr;
+    for (int base = 0; base < n; base += 32 * UNROLL) {
+        uint4 v[UNROLL];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const int i = base + u * 32 + lane;
-                if (i < n) {
-                    const int r = i / vpr, c = i - r * vpr;
-                    v[u] = ld_stream(reinterpret_cast<const uint4*>(it.src + r * it.src_pitch) + c);
-                }
+        for (int u = 0; u < UNROLL; ++u) {
+            const int i = base + u * 32 + lane;
+            if (i < n) {
+                const int r = i / vpr, c = i - r * vpr;
+                v[u] = ld_stream(reinterpret_cast<const uint4*>(src + r * src_pitch) + c);
             }
+        }
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const int i = base + u * 32 + lane;
-                if (i < n) {
-                    const int r = i / vpr, c = i - r * vpr;
-                    st_stream(reinterpret_cast<uint4*>(it.dst + r * it.dst_pitch) + c, v[u]);
-                }
+        for (int u = 0; u < UNROLL; ++u) {
+            const int i = base + u * 32 + lane;
+            if (i < n) {
+                const int r = i / vpr, c = i - r * vpr;
+                st_stream(reinterpret_cast<uint4*>(dst + r * dst_pitch) + c, v[u]);
             }
         }
     }
+}
+template <int UNROLL>
+__device__ __forceinline__ void warp_copy_item(const Item& it) {
+    warp_copy_rows<UNROLL>(it.src, it.dst, it.src_pitch, it.dst_pitch, it.n_rows, it.row_bytes);
 }
 
 // ------------------------------------------------------------------ bulk-copy (TMA) primitives
@@ -146,11 +147,12 @@ constexpr uint32_t kDefaultWaitTries = 1u << 22;
 constexpr uint32_t kDrainWaitTries = 1u << 16;
 // Bounded wait: false if the phase did not complete within the budget, or if *abort became non-zero meanwhile (the
 // other warp of the ring gave up).  max_polls == 0: the default budget of potentially-suspending try_wait calls;
-// max_polls > 0: that many non-blocking polls (a caller-chosen, short limit).
+// max_polls = v > 0: a caller-chosen, short limit of v - 1 non-blocking polls (v = 1: give up at once, which makes
+// the give-up path run on healthy copies, deterministically).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_polls = 0,
                                                   const volatile int32_t* abort = nullptr) {
     if (max_polls) {
-        for (uint32_t i = 0; i < max_polls; ++i)
+        for (uint32_t i = 1; i < max_polls; ++i)
             if (mbar_test_wait(bar, parity)) return true;
         return false;
     }

@@ -190,24 +190,57 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
 //     (the new k section may lie where the kept q rows were);
 //   columns (o_proj, down_proj): row j of the kept column range moves from j*w + keep*w/N to j*w/N; rows are done in
 //     waves [0,1), [1,N), [N,N^2), ...: the destination of wave [m, N*m) ends at byte m*w, where its sources begin.
-// Phases are separate launches on the stream; within a phase all copies are disjoint.
-static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
-                                             const int32_t* keep, int32_t layer_begin, int32_t layer_end,
-                                             int32_t* d_status, void* cuda_stream) {
-    if (!plan || !bufs || !keep || !d_status) return AMOEBA_ERR_INVALID_ARG;
+// The leading waves of a column tensor are tiny (1, N-1, N^2-N ... rows): one CTA per buffer runs them back to back
+// in a single launch of w_compact_lead, a CTA-wide barrier between waves (every wave only depends on earlier waves
+// of the same buffer, and nothing a wave writes is read again).  The remaining waves and the row moves are separate
+// launches of the copy kernel on the stream; within a launch all copies are disjoint.
+namespace amoeba {
+
+constexpr int kMaxLeadBufs = 1024;          // buffers (layer, worker, column tensor) per launch of the lead kernel
+constexpr int64_t kLeadBytes = 1 << 20;     // kept bytes one CTA moves for its buffer before the waves go grid-wide
+
+struct LeadParams {
+    char* bufs[kMaxLeadBufs];
+    uint8_t cls[kMaxLeadBufs];   // 0 = o_proj, 1 = down_proj
+    uint8_t keep[kMaxLeadBufs];  // which N-th of the columns the buffer's worker keeps
+    int64_t w_old[2], w_new[2];  // bytes of a row before / after
+    int32_t rows[2];             // rows [0, rows[c]) are moved here
+    int32_t n;                   // N
+};
+
+__global__ void __launch_bounds__(256) w_compact_lead(const __grid_constant__ LeadParams p) {
+    const int b = blockIdx.x, c = p.cls[b];
+    char* base = p.bufs[b];
+    const int64_t w_old = p.w_old[c], w_new = p.w_new[c], keep_off = p.keep[b] * w_new;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    int64_t lo = 0, hi = 1;
+    while (lo < p.rows[c]) {
+        if (hi > p.rows[c]) hi = p.rows[c];
+        for (int64_t row = lo + warp; row < hi; row += nwarps) {
+            if (row == 0 && keep_off == 0) continue;  // already in place
+            copy_vecs<8>(reinterpret_cast<const uint4*>(base + row * w_old + keep_off),
+                         reinterpret_cast<uint4*>(base + row * w_new), (int)(w_new >> 4), lane, 32);
+        }
+        __syncthreads();  // every load of this wave has returned (its stores were issued after them)
+        lo = hi;
+        hi *= p.n;
+    }
+}
+
+struct CompactSchedule {
+    std::vector<std::vector<amoeba_weight_desc>> phases;  // copy-kernel launches, in order
+    int32_t lead_rows[2] = {0, 0};                        // rows of o_proj / down_proj the lead kernel moves
+    int64_t w_old[2] = {0, 0}, w_new[2] = {0, 0};
+    int64_t bytes_per_layer = 0;                          // bytes read (= written) per layer, all workers
+};
+
+enum { Q, K, V, O, GATE, UP, DOWN };
+
+// What moves where for plan->src (TP = a) -> plan->dst (TP = N*a) with worker r keeping sub-shard keep[r].
+static void compact_schedule(const amoeba_plan* plan, const int32_t* keep, CompactSchedule* out) {
     const amoeba_layout &sl = plan->src, &dl = plan->dst;
     const amoeba_model& m = sl.model;
-    const int L = m.num_layers, a = sl.tp, b = dl.tp;
-    if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
-    if (b % a || sl.weight_pad_parts || dl.weight_pad_parts || sl.fused_qkv != dl.fused_qkv ||
-        sl.fused_gate_up != dl.fused_gate_up)
-        return AMOEBA_ERR_UNSUPPORTED;
-    const int N = b / a;
-    for (int r = 0; r < a; ++r)
-        if (keep[r] < 0 || keep[r] >= N) return AMOEBA_ERR_INVALID_ARG;
-    if (N == 1) return AMOEBA_OK;
-
-    enum { Q, K, V, O, GATE, UP, DOWN };
+    const int a = sl.tp, b = dl.tp, N = b / a;
     const int64_t e = m.elem_bytes, hid = m.hidden, rb = hid * e;
     const int64_t rows_of[kNumTensors] = {(int64_t)m.num_q_heads * m.head_dim, (int64_t)m.num_kv_heads * m.head_dim,
                                           (int64_t)m.num_kv_heads * m.head_dim, 0, m.intermediate, m.intermediate, 0};
@@ -223,16 +256,7 @@ static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoe
         buffer_of[UP] = GATE;
         sec_old[UP] = rows_of[GATE] / a, sec_new[UP] = rows_of[GATE] / b;
     }
-    // every buffer that is touched must be there and aligned
-    for (int l = layer_begin; l < layer_end; ++l)
-        for (int r = 0; r < a; ++r)
-            for (int t = 0; t < kNumTensors; ++t) {
-                const void* ptr = slots(&bufs[(size_t)r * L + l])[buffer_of[t]];
-                if (!ptr) return AMOEBA_ERR_INVALID_ARG;
-                if (reinterpret_cast<uintptr_t>(ptr) % 16) return AMOEBA_ERR_ALIGNMENT;
-            }
-
-    std::vector<std::vector<amoeba_weight_desc>> phases;
+    auto& phases = out->phases;
     auto phase = [&](size_t i) -> std::vector<amoeba_weight_desc>& {
         if (phases.size() <= i) phases.resize(i + 1);
         return phases[i];
@@ -250,17 +274,27 @@ static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoe
                 d.dst_off = sec_new[t] * rb;
                 d.n_rows = 1;
                 d.src_pitch = d.dst_pitch = d.row_bytes;
-                if (d.src_off != d.dst_off) phase(step).push_back(d);
+                if (d.src_off != d.dst_off) {
+                    phase(step).push_back(d);
+                    out->bytes_per_layer += d.row_bytes;
+                }
             }
         }
     const int col_tensors[2] = {O, DOWN};
     const int64_t cols_of[2] = {(int64_t)m.num_q_heads * m.head_dim, m.intermediate};
     for (int c = 0; c < 2; ++c) {
         const int64_t w_old = cols_of[c] / a * e, w_new = cols_of[c] / b * e;
-        int64_t lo = 0, hi = 1;
+        out->w_old[c] = w_old;
+        out->w_new[c] = w_new;
+        // the lead kernel takes rows [0, N^k): the largest such range of at most kLeadBytes kept bytes
+        int64_t lead = 1;
+        while (lead < hid && lead * N * w_new <= kLeadBytes) lead *= N;
+        lead = std::min(lead, hid);
+        out->lead_rows[c] = (int32_t)lead;
+        for (int r = 0; r < a; ++r) out->bytes_per_layer += (lead - (keep[r] == 0 ? 1 : 0)) * w_new;
+        int64_t lo = lead, hi = lead * N;
         for (size_t wave = 0; lo < hid; ++wave) {
             for (int r = 0; r < a; ++r) {
-                if (keep[r] == 0 && lo == 0) continue;  // row 0 of the first column range is already in place
                 amoeba_weight_desc d{};
                 d.src_rank = d.dst_rank = r;
                 d.src_tensor = d.dst_tensor = col_tensors[c];
@@ -271,15 +305,87 @@ static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoe
                 d.src_pitch = w_old;
                 d.dst_pitch = w_new;
                 phase(wave).push_back(d);
+                out->bytes_per_layer += d.row_bytes * d.n_rows;
             }
             lo = hi;
             hi *= N;
         }
     }
+}
 
-    const int64_t cap = plan->opt.w.chunk_bytes > 0 ? plan->opt.w.chunk_bytes : kDefaultWChunk;
+static amoeba_status compact_check(const amoeba_plan* plan, const int32_t* keep) {
+    if (!plan || !keep) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_layout &sl = plan->src, &dl = plan->dst;
+    if (dl.tp % sl.tp || sl.weight_pad_parts || dl.weight_pad_parts || sl.fused_qkv != dl.fused_qkv ||
+        sl.fused_gate_up != dl.fused_gate_up)
+        return AMOEBA_ERR_UNSUPPORTED;
+    for (int r = 0; r < sl.tp; ++r)
+        if (keep[r] < 0 || keep[r] >= dl.tp / sl.tp) return AMOEBA_ERR_INVALID_ARG;
+    return AMOEBA_OK;
+}
+
+}  // namespace amoeba
+
+static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoeba_layer_weights* bufs,
+                                             const int32_t* keep, int32_t layer_begin, int32_t layer_end,
+                                             int32_t* d_status, void* cuda_stream) {
+    if (!bufs || !d_status) return AMOEBA_ERR_INVALID_ARG;
+    amoeba_status st = compact_check(plan, keep);
+    if (st != AMOEBA_OK) return st;
+    const amoeba_layout& sl = plan->src;
+    const int L = sl.model.num_layers, a = sl.tp, N = plan->dst.tp / a;
+    if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
+    if (N == 1 || layer_begin == layer_end) return AMOEBA_OK;
+    // every buffer that is touched must be there and aligned
+    int buffer_of[kNumTensors] = {Q, K, V, O, GATE, UP, DOWN};
+    if (sl.fused_qkv) buffer_of[K] = buffer_of[V] = Q;
+    if (sl.fused_gate_up) buffer_of[UP] = GATE;
+    for (int l = layer_begin; l < layer_end; ++l)
+        for (int r = 0; r < a; ++r)
+            for (int t = 0; t < kNumTensors; ++t) {
+                const void* ptr = slots(&bufs[(size_t)r * L + l])[buffer_of[t]];
+                if (!ptr) return AMOEBA_ERR_INVALID_ARG;
+                if (reinterpret_cast<uintptr_t>(ptr) % 16) return AMOEBA_ERR_ALIGNMENT;
+            }
+    CompactSchedule sch;
+    compact_schedule(plan, keep, &sch);
+    for (int c = 0; c < 2; ++c)
+        if (sch.w_old[c] % 16 || sch.w_new[c] % 16) return AMOEBA_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    for (const auto& ph : phases) {
+
+    // ---- leading waves of the column tensors: one CTA per (layer, worker, tensor) buffer
+    {
+        LeadParams lp;
+        lp.n = N;
+        for (int c = 0; c < 2; ++c) {
+            lp.w_old[c] = sch.w_old[c];
+            lp.w_new[c] = sch.w_new[c];
+            lp.rows[c] = sch.lead_rows[c];
+        }
+        const int col_tensors[2] = {O, DOWN};
+        int n = 0;
+        auto flush = [&]() -> amoeba_status {
+            if (n == 0) return AMOEBA_OK;
+            w_compact_lead<<<n, 256, 0, stream>>>(lp);
+            if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+            count_launch();
+            n = 0;
+            return AMOEBA_OK;
+        };
+        for (int l = layer_begin; l < layer_end; ++l)
+            for (int r = 0; r < a; ++r)
+                for (int c = 0; c < 2; ++c) {
+                    lp.bufs[n] = static_cast<char*>(slots(&bufs[(size_t)r * L + l])[col_tensors[c]]);
+                    lp.cls[n] = (uint8_t)c;
+                    lp.keep[n] = (uint8_t)keep[r];
+                    if (++n == kMaxLeadBufs && (st = flush()) != AMOEBA_OK) return st;
+                }
+        if ((st = flush()) != AMOEBA_OK) return st;
+    }
+
+    // ---- the remaining waves and the row moves
+    const int64_t cap = plan->opt.w.chunk_bytes > 0 ? plan->opt.w.chunk_bytes : kDefaultWChunk;
+    for (const auto& ph : sch.phases) {
         std::vector<WDescDev> descs;
         int64_t items = 0;
         for (const amoeba_weight_desc& d : ph) {
@@ -288,9 +394,22 @@ static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoe
             descs.push_back(chunk_desc(d, cap, &items));
             if (items > INT32_MAX || (int)descs.size() > kMaxWeightDescs) return AMOEBA_ERR_UNSUPPORTED;
         }
-        const amoeba_status st = launch_descs(plan, descs, (int32_t)items, bufs, a, bufs, a, L, layer_begin, layer_end,
-                                              d_status, stream);
+        st = launch_descs(plan, descs, (int32_t)items, bufs, a, bufs, a, L, layer_begin, layer_end, d_status, stream);
         if (st != AMOEBA_OK) return st;
+    }
+    return AMOEBA_OK;
+}
+
+extern "C" amoeba_status amoeba_compact_bytes(const amoeba_plan* plan, const int32_t* keep, int64_t* bytes_rw) {
+    if (!bytes_rw) return AMOEBA_ERR_INVALID_ARG;
+    const amoeba_status st = compact_check(plan, keep);
+    if (st != AMOEBA_OK) return st;
+    try {
+        CompactSchedule sch;
+        if (plan->dst.tp != plan->src.tp) compact_schedule(plan, keep, &sch);
+        *bytes_rw = 2 * sch.bytes_per_layer * plan->src.model.num_layers;
+    } catch (...) {
+        return AMOEBA_ERR_NO_MEMORY;
     }
     return AMOEBA_OK;
 }

@@ -248,11 +248,11 @@ class MergeSession:
             A.amoeba_compact_weights_inplace(self.plan, packed, [i] * self.a, 0, self.L, self.status, stream)
 
     def weight_bytes_rw(self) -> int:
-        """Bytes read + written by compact_weights: 1/N of every instance's weights, both ways."""
+        """Bytes read + written by compact_weights, as the library counts them (what already is in place - e.g. the
+        first section of every buffer of instance 0 - is not moved and not counted)."""
         if not self.inst_w:
             return 0
-        _, w = A.amoeba_plan_bytes(self.plan, 0)
-        return w  # N instances x (1/N of one model copy) x 2
+        return sum(A.amoeba_compact_bytes(self.plan, [i] * self.a) for i in range(self.N))
 
     def merge_block_tables(self, stream=None) -> None:
         A.amoeba_merge_block_tables(self.plan, self.src_bt, self.seq_lens, self.num_seqs, self.maxb, self.dst_bt,
@@ -282,10 +282,10 @@ class MergeCopySession:
     """N instances of TP=a become one instance of TP=N*a in FRESH pools (out of place): one table rewrite and one KV
     call per instance, each given the part of the shared destination free list the earlier instances left.  This is
     what a merge costs without in-place block reshaping (and the only way with token-first pools); it needs a second
-    set of pools.  seq_lens [N][S] and src_bt [N][S][maxb] are host arrays (the block counts that advance the free list
-    are computed from the lengths on the host)."""
+    set of pools.  seq_lens [N][S] and src_bt [N][S][maxb] are host arrays; counts[i] = number of blocks instance i's
+    table names (the caller's bookkeeping: it is what advances the shared free list from one instance to the next)."""
 
-    def __init__(self, model: dict, N: int, a: int, NB_src: int, NB_dst: int, seq_lens, src_bt, free_list,
+    def __init__(self, model: dict, N: int, a: int, NB_src: int, NB_dst: int, seq_lens, src_bt, free_list, counts,
                  kv_layers: Optional[int] = None, block_tokens: int = 16, device="cuda:0",
                  src_kv_order: int = A.KV_HEAD_MAJOR, dst_kv_order: int = A.KV_HEAD_MAJOR):
         self.model, self.N, self.a = model, N, a
@@ -299,7 +299,8 @@ class MergeCopySession:
         bt = torch.as_tensor(src_bt, dtype=torch.int32)
         self.num_seqs, self.maxb = int(bt.shape[1]), int(bt.shape[2])
         i32 = dict(dtype=torch.int32, device=dev)
-        counts = [int(((lens[i].long() + block_tokens - 1) // block_tokens).sum()) for i in range(N)]
+        counts = [int(c) for c in counts]
+        assert len(counts) == N
         self.counts, self.offsets = counts, [sum(counts[:i]) for i in range(N)]
         self.free_list = torch.as_tensor(free_list, dtype=torch.int32).to(dev)
         assert self.free_list.numel() >= sum(counts)

@@ -1,10 +1,10 @@
 """Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times.
 
-The source buffers are filled on the device with a counter hash; the tables are compared whole with the oracle's;
-the KV result is compared on sampled (layer, sequence, block) units - for each, the source worker slices are fetched,
-the oracle re-lays-out that one block on the CPU, and the destination worker slices must equal it; the weights of
-sampled layers are compared whole.  Size-independent properties: word sums are conserved, untouched destination
-blocks keep their fill."""
+The source buffers are filled on the device with a counter hash; the tables are compared whole with the oracle's.
+KV: three whole layers (the first, the last, one drawn at random) of EVERY destination pool are compared element by
+element - live blocks, idle blocks and foreign blocks alike - with the oracle's transformation of the same layer,
+streamed layer by layer through host memory; on the other layers sampled (layer, sequence, block) units are
+re-laid-out by the oracle one by one.  Weights: sampled layers compared whole."""
 import numpy as np
 import pytest
 
@@ -30,14 +30,6 @@ class _BlockView:
     def __getitem__(self, idx):
         l, blk = idx
         return self.v[l, :, blk].reshape(-1) if self.tf else self.v[l, blk]
-
-    def layer_blocks(self, l, NB, ids):
-        """int64 words of the given blocks of layer l, [len(ids), words]."""
-        import torch
-
-        if self.tf:
-            return torch.cat([self.v[l, c].view(torch.int64).view(NB, -1).index_select(0, ids) for c in range(2)], 1)
-        return self.v[l].view(torch.int64).view(NB, -1).index_select(0, ids)
 
 
 @pytest.mark.parametrize("name,kv_order", CASES)
@@ -86,22 +78,19 @@ def test_full_size_config(name, kv_order, oracle):
                 got = dst_v[r][l, did].cpu().numpy().view(np.uint16)
                 assert np.array_equal(got, exp1[r]), (name, l, q, i, r)
 
-        # ---- untouched destination blocks keep the fill (sampled)
-        used = np.zeros(st["NB_dst"], bool)
-        used[exp_pairs[:, 1]] = True
-        idle = np.flatnonzero(~used)
-        if idle.size:
-            for did in g.choice(idle, size=min(16, idle.size), replace=False):
-                for v in dst_v:
-                    assert bool((v[int(g.integers(Lkv)), int(did)] == 0xA5).all())
-
-        # ---- word sums are conserved over the live blocks of every layer (any size, any permutation)
-        live_src = torch.as_tensor(exp_pairs[:, 0].astype(np.int64), device=device)
-        live_dst = torch.as_tensor(exp_pairs[:, 1].astype(np.int64), device=device)
-        for l in sorted(set(int(x) for x in g.integers(Lkv, size=3))):
-            ssum = sum(int(v.layer_blocks(l, st["NB_src"], live_src).sum().item()) for v in src_v)
-            dsum = sum(int(v.layer_blocks(l, st["NB_dst"], live_dst).sum().item()) for v in dst_v)
-            assert (ssum - dsum) % (1 << 64) == 0
+        # ---- KV: whole layers, every word of every destination pool (live, idle and foreign blocks)
+        for l in sorted({0, Lkv - 1, int(g.integers(Lkv))}):
+            src1 = [p.view(Lkv, -1)[l].cpu().numpy().view(np.uint16) for p in s.src_pools]
+            exp1 = [np.full(p.numel() // Lkv // 2, 0xA5A5, np.uint16) for p in s.dst_pools]
+            oracle.kv_transform(one, T, st["seq_lens"], a, st["NB_src"], st["src_bt"], src1, b, st["NB_dst"], exp_bt,
+                                exp1, src_order=so, dst_order=do)
+            del src1
+            for r in range(b):
+                got = s.dst_pools[r].view(Lkv, -1)[l].cpu().numpy().view(np.uint16)
+                if not np.array_equal(got, exp1[r]):
+                    bad = np.flatnonzero(got != exp1[r])
+                    raise AssertionError(f"{name} layer {l} dst pool {r}: {bad.size} words differ, first at {bad[0]}")
+            del exp1
 
         # ---- weights: whole comparison of sampled layers
         for l in sorted(set([0, m["L"] - 1, int(g.integers(m["L"]))])):
@@ -119,8 +108,9 @@ def test_full_size_config(name, kv_order, oracle):
 
 def test_full_size_inplace_merge(oracle):
     """The benchmark's in-place merge workload (4 x TP1 -> TP4) at full size: merged tables and live marks compared
-    whole; sampled old blocks (with whatever mix of live / free they have across the instances) compared with the
-    oracle's merge of just those blocks; word sums of the live blocks conserved per layer."""
+    whole; three whole layers (first, last, one at random) of every pool compared word by word with the oracle's merge
+    of the same layer; on the other layers sampled old blocks (with whatever mix of live / free they have across the
+    instances) compared with the oracle's merge of just those blocks."""
     import torch
 
     import bench
@@ -139,10 +129,8 @@ def test_full_size_inplace_merge(oracle):
         old_v = [p.view(L, NB, -1) for p in s.pools]            # [layer][old block][bytes]
         samples = [(int(g.integers(L)), int(g.integers(NB))) for _ in range(64)]
         before = {(l, p): [v[l, p].cpu().numpy().view(np.uint16).copy() for v in old_v] for l, p in samples}
-        live_old = [torch.as_tensor(np.flatnonzero(exp_live[i]).astype(np.int64), device=device) for i in range(N)]
-        sum_layers = sorted(set(int(x) for x in g.integers(L, size=2)))
-        sums_before = {l: sum(int(old_v[i * a + r][l].view(torch.int64).view(NB, -1).index_select(0, live_old[i]).sum())
-                              for i in range(N) for r in range(a)) for l in sum_layers}
+        whole_layers = sorted({0, L - 1, int(g.integers(L))})
+        layer_before = {l: [v[l].cpu().numpy().view(np.uint16).reshape(-1).copy() for v in old_v] for l in whole_layers}
 
         s.status.zero_()
         s.step()
@@ -161,13 +149,59 @@ def test_full_size_inplace_merge(oracle):
                 got = old_v[w][l, p].cpu().numpy().view(np.uint16)
                 assert np.array_equal(got, mini[w]), (l, p, w)
 
-        new_v = [p.view(L, NB * N, -1) for p in s.pools]        # [layer][new block][bytes]
-        for l in sum_layers:
-            after = 0
-            for i in range(N):
-                ids = live_old[i] * N + i
-                after += sum(int(v[l].view(torch.int64).view(NB * N, -1).index_select(0, ids).sum()) for v in new_v)
-            assert (after - sums_before[l]) % (1 << 64) == 0
+        for l in whole_layers:
+            exp = layer_before.pop(l)
+            _, _, st1 = oracle.kv_merge_inplace(one, T, N, a, NB, st["seq_lens"], st["src_bt"], exp)
+            assert st1 == 0
+            for w in range(N * a):
+                got = old_v[w][l].cpu().numpy().view(np.uint16).reshape(-1)
+                if not np.array_equal(got, exp[w]):
+                    bad = np.flatnonzero(got != exp[w])
+                    raise AssertionError(f"layer {l} pool {w}: {bad.size} words differ, first at {bad[0]}")
+    finally:
+        del s
+        torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["llama3_8b_1to4", "llama3_8b_2to8", "llama3_70b_slice_8to2"])
+def test_full_size_inplace_reshape(name, oracle):
+    """In-place block reshaping of one instance with the benchmark configuration's sequences, in the launch
+    configuration bench.py --inplace times: tables, pair list and free mask compared whole; three whole layers of every
+    pool (old workers' memory and new workers' pools) compared word by word with the oracle."""
+    import torch
+
+    import bench
+
+    cfg = wl.CONFIGS[name]
+    m, T = cfg["model"], wl.BLOCK_TOKENS
+    s, st = bench.build_reshape_session(name, torch.device("cuda:0"))
+    try:
+        N, a, NB, L = s.N, s.a, s.NB, s.kv_layers
+        src_bt = s.src_bt.cpu().numpy()
+        g = np.random.default_rng(13)
+        whole_layers = sorted({0, L - 1, int(g.integers(L))})
+        views = [p.view(L, -1) for p in s.pools]
+        before = {l: [v[l].cpu().numpy().view(np.uint16).copy() for v in views] for l in whole_layers}
+        s.status.zero_()
+        s.step()
+        torch.cuda.synchronize()
+        one = dict(m, L=1)
+        first = True
+        for l in whole_layers:
+            exp = before.pop(l)
+            e_bt, e_pairs, e_n, e_mask, e_left, e_status = oracle.kv_reshape_inplace(
+                s.direction, one, T, N, a, NB, st["seq_lens"], src_bt, exp, pairs_cap=st["n_live"])
+            if first:
+                assert e_status == 0 and int(s.status.item()) == 0
+                assert np.array_equal(s.dst_bt.cpu().numpy(), e_bt)
+                assert int(s.num_pairs.item()) == e_n and np.array_equal(s.pairs.cpu().numpy()[:e_n], e_pairs)
+                assert np.array_equal(s.free_mask.cpu().numpy(), e_mask) and int(s.free_count.item()) == e_left
+                first = False
+            for w in range(N * a):
+                got = views[w][l].cpu().numpy().view(np.uint16)
+                if not np.array_equal(got, exp[w]):
+                    bad = np.flatnonzero(got != exp[w])
+                    raise AssertionError(f"{name} layer {l} pool {w}: {bad.size} words differ, first at {bad[0]}")
     finally:
         del s
         torch.cuda.empty_cache()

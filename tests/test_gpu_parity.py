@@ -670,8 +670,8 @@ def test_out_of_place_calls_refuse_a_buffer_on_both_sides():
 
 @pytest.mark.parametrize("path", [BULK, PAIR])
 def test_wait_budget_running_out_is_reported_and_the_next_call_is_exact(path):
-    """Every wait of a copy kernel on its own bulk copies is bounded.  With a budget of ONE non-blocking poll the
-    first wait of every ring runs out before its (healthy) load can have landed: the kernel must record TIMEOUT, let
+    """Every wait of a copy kernel on its own bulk copies is bounded.  With the smallest budget (give up without
+    polling) the first wait of every ring runs out although its load is healthy: the kernel must record TIMEOUT, let
     the copies it has in flight land, and return - nothing outside the destination buffers is touched, the context
     stays usable, and the same call with the default budget then gives the exact result."""
     import torch

@@ -311,3 +311,22 @@ def test_random_layout_pairs_reproduce_oracle(oracle):
                     assert np.array_equal(dst[r][t], exp[r][n].reshape(-1).view(np.uint8)), (m, a, b, sp, dp, fq, fg, r, n)
                     assert counts[r][t].max() == 1
         done += 1
+
+
+def test_compact_bytes_counts_only_what_moves():
+    """Partial swap, TP 1 -> 4, fused buffers: with keep = 0 the q and gate sections and row 0 of o_proj / down_proj
+    already sit where they belong and are not counted; with keep > 0 everything kept moves."""
+    m = dict(L=3, hidden=64, Hq=16, Hkv=8, D=16, I=192)
+    plan = A.amoeba_plan_create(A.make_layout(m, 1, 4), A.make_layout(m, 4, 16))
+    e, hid, N = 2, m["hidden"], 4
+    rb = hid * e
+    q, kv, ffn = m["Hq"] * m["D"] // N * rb, m["Hkv"] * m["D"] // N * rb, m["I"] // N * rb
+    wo, wd = m["Hq"] * m["D"] // N * e, m["I"] // N * e
+    everything = q + 2 * kv + 2 * ffn + hid * (wo + wd)
+    assert A.amoeba_compact_bytes(plan, [2]) == 2 * m["L"] * everything
+    assert A.amoeba_compact_bytes(plan, [0]) == 2 * m["L"] * (everything - q - ffn - wo - wd)
+    _, w = A.amoeba_plan_bytes(plan, 0)
+    assert A.amoeba_compact_bytes(plan, [3]) * N == w  # one N-th of the weights, read and written
+    with pytest.raises(A.AmoebaError) as err:
+        A.amoeba_compact_bytes(plan, [4])
+    assert err.value.status == A.ERR_INVALID_ARG

@@ -163,15 +163,25 @@ def draw_merge_state(cfg: dict, seed: int = DEFAULT_SEED, name: str = "", T: int
                 blocks_per_seq=nblk, T=T)
 
 
+def counter_words(n: int, salt: int) -> np.ndarray:
+    """n 16-bit words, word i = low 16 bits of (i mod 65521)*40503 + salt: a cheap, reproducible, non-constant fill
+    (one period is computed, the rest is copied)."""
+    period = (np.arange(65521, dtype=np.uint32) * np.uint32(40503) + np.uint32(salt & 0xFFFF)).astype(np.uint16)
+    return np.resize(period, n)
+
+
 def draw_kv_logical(cfg: dict, n_tokens: int, layers, seed: int = DEFAULT_SEED, dist: str = "normal") -> np.ndarray:
     """Logical KV values for the given layers: uint16 [len(layers), n_tokens, Hkv, 2, D].
 
     dist "normal": N(0,1) rounded to the config's 16-bit float type; "words": uniform 16-bit words (several times
-    faster to draw; for timing runs, where the values do not matter)."""
+    faster to draw); "counter": a periodic counter pattern (memory-speed; for timing runs, where the values do not
+    matter)."""
     m = cfg["model"]
     out = np.empty((len(layers), n_tokens, m["Hkv"], 2, m["D"]), dtype=np.uint16)
     for i, l in enumerate(layers):
-        if dist == "words":
+        if dist == "counter":
+            out[i] = counter_words(out[i].size, l).reshape(out.shape[1:])
+        elif dist == "words":
             out[i] = rng(seed, "kv_words", l).integers(0, 65536, size=out.shape[1:], dtype=np.uint16)
         else:
             x = rng(seed, "kv", l).standard_normal(size=out.shape[1:], dtype=np.float32)
@@ -189,6 +199,9 @@ def draw_weights_logical(cfg: dict, layer: int, seed: int = DEFAULT_SEED, std: f
               "down": (hid, I)}
     out = {}
     for j, (n, s) in enumerate(shapes.items()):
+        if dist == "counter":
+            out[n] = counter_words(s[0] * s[1], layer * 7 + j).reshape(s)
+            continue
         if dist == "words":
             out[n] = rng(seed, "w_words", layer, j).integers(0, 65536, size=s, dtype=np.uint16)
             continue
