@@ -574,6 +574,9 @@ def run_merge(args, rank, world, local):
                      (A.OPT_CTAS_PER_SM, args.ctas_per_sm)):
         if val:
             s.set_option(opt, val)
+    for item in args.opt:
+        name, val = item.split("=")
+        s.set_option(getattr(A, "OPT_" + name.upper()), int(val))
     w_bytes = s.weight_bytes_rw()
     nbytes = s.bytes_rw(st["n_live"]) + w_bytes
     stream = torch.cuda.current_stream()

@@ -184,6 +184,8 @@ enum {
                                    up after v - 1 non-blocking polls and report AMOEBA_ERR_TIMEOUT (0 = the default,
                                    generous budget).  For tests of the give-up path: v = 1 gives up at once, so healthy
                                    copies time out, every time. */
+    AMOEBA_OPT_L2_PROMOTION = 10, /* tensor-map copies of token-first pools: L2 promotion of the maps, 1 = none, 2 = 64 B,
+                                   3 = 128 B, 4 = 256 B */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };

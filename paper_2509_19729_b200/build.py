@@ -15,7 +15,7 @@ CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libamoeba.so"
 SOURCES = ["plan.cpp", "block_tables.cu", "kv_reshard.cu", "weights_reshard.cu"]
-HEADERS = ["plan.hpp", "launch.hpp", "copy_engine.cuh"]
+HEADERS = ["plan.hpp", "launch.hpp", "copy_engine.cuh", "kv_items.cuh", "w_items.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",

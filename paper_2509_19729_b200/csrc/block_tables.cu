@@ -3,12 +3,14 @@
 // No CTA ever waits on another.  Two phases:
 //   scan   (1 CTA)  blocks per sequence and their exclusive prefix sum; when the free blocks come as a byte mask,
 //                   their compaction into an ascending id list (16 mask bytes per thread, popc + CTA prefix sum);
-//                   when destination ids can repeat (a free LIST, or ids derived from the source table), the first
-//                   user of every destination id in (sequence, block) order, by atomicMin; the whole-call errors.
+//                   the whole-call errors.
+//   claim  (grid)   only when destination ids can repeat (a free LIST, or ids derived from the source table): the
+//                   first user of every destination id in (sequence, block) order, by atomicMin.
 //   assign (grid)   one warp per 128-entry segment of a block-table row: the k-th block overall takes the k-th free
 //                   id (or the reshaped id of its source block); writes the destination table (with -1 padding) and
 //                   the (source, destination) pair list; an id whose first user is another block is refused.
-// Small tables run both phases in one launch of one CTA; large ones as two launches.
+// Small tables run all phases in one launch of one CTA; larger ones as separate launches, each of which starts when
+// the one before it has completed.
 #include <cuda_runtime.h>
 
 #include <climits>
@@ -162,23 +164,34 @@ __device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) 
     }
     __syncthreads();
 
-    // ---- first user of every destination id (ids from a list or from the source table may repeat)
-    if (!a.free_mask) {
+    // ---- nobody holds a destination id yet (ids from a list or from the source table may repeat)
+    if (!a.free_mask)
         for (int32_t q = tid; q < a.nb_dst; q += kScanThreads) a.area[q] = INT32_MAX;
-        __syncthreads();
-        if (flags[1] == 0) {
-            for (int32_t s = warp; s < a.num_seqs; s += kScanThreads / 32) {
-                const int32_t nb = blocks_needed(a.seq_lens[s], a.block_tokens), off = a.seq_off[s];
-                for (int32_t i = lane; i < nb; i += 32) {
-                    const int32_t d = dst_id_of(a, off + i, a.src_bt[(int64_t)s * a.maxb + i]);
-                    if (d >= 0 && d < a.nb_dst) atomicMin(a.area + d, off + i);
-                }
-            }
+}
+
+// First user of every destination id in (sequence, block) order, by atomicMin over the k of the blocks that are
+// given it.  Any number of threads; thread `t` of `n`.  Runs after scan_phase has completed.
+__device__ void claim_phase(const BtArgs& a, int64_t t, int64_t n) {
+    if (a.free_mask || a.hdr->err) return;
+    if (a.reshape == 0) {  // the k-th block is given the k-th list entry, whatever its source id
+        const int32_t total = a.hdr->total;
+        for (int64_t k = t; k < total; k += n) {
+            const int32_t d = a.free_list[k];
+            if (d >= 0 && d < a.nb_dst) atomicMin(a.area + d, (int32_t)k);
         }
+        return;
+    }
+    const int64_t entries = (int64_t)a.num_seqs * a.maxb;
+    for (int64_t e = t; e < entries; e += n) {
+        const int32_t s = (int32_t)(e / a.maxb), i = (int32_t)(e - (int64_t)s * a.maxb);
+        if (i >= blocks_needed(a.seq_lens[s], a.block_tokens)) continue;
+        const int32_t k = a.seq_off[s] + i;
+        const int32_t d = dst_id_of(a, k, a.src_bt[e]);
+        if (d >= 0 && d < a.nb_dst) atomicMin(a.area + d, k);
     }
 }
 
-// Any number of warps; warp `warp` of `n_warps`.  Runs after scan_phase has completed (next launch, or after a
+// Any number of warps; warp `warp` of `n_warps`.  Runs after claim_phase has completed (next launch, or after a
 // __syncthreads() of the one CTA that ran it).
 __device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
     const int lane = threadIdx.x & 31;
@@ -224,22 +237,29 @@ __global__ void __launch_bounds__(kScanThreads) bt_scan(const __grid_constant__ 
     scan_phase(a, warp_sums, flags);
 }
 
+__global__ void __launch_bounds__(256) bt_claim(const __grid_constant__ BtArgs a) {
+    claim_phase(a, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
+}
+
 __global__ void __launch_bounds__(256) bt_assign(const __grid_constant__ BtArgs a) {
     assign_phase(a, ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, ((int64_t)gridDim.x * blockDim.x) >> 5);
 }
 
-// Both phases in one CTA: what the CTA wrote to global memory in the scan is visible to all its threads after the
-// barrier.
+// All phases in one CTA: what the CTA wrote to global memory in a phase is visible to all its threads after the
+// barrier that ends it.
 __global__ void __launch_bounds__(kScanThreads) bt_fused(const __grid_constant__ BtArgs a) {
     __shared__ int32_t warp_sums[33];
     __shared__ int32_t flags[2];
     scan_phase(a, warp_sums, flags);
     __threadfence_block();
     __syncthreads();
+    claim_phase(a, threadIdx.x, kScanThreads);
+    __threadfence_block();
+    __syncthreads();
     assign_phase(a, threadIdx.x >> 5, kScanThreads / 32);
 }
 
-constexpr int64_t kFusedEntries = 128 * 1024;  // up to this many table entries (and destination ids): one launch
+constexpr int64_t kFusedEntries = 8 * 1024;  // up to this many table entries (and destination ids): one launch
 
 static int64_t align16(int64_t x) { return (x + 15) & ~int64_t(15); }
 
@@ -269,6 +289,13 @@ static amoeba_status launch_tables(const amoeba_plan* plan, BtArgs a, void* d_wo
     if (a.num_seqs == 0 && !a.reshape) return AMOEBA_OK;
     const int sms = cached_device_info().sms;
     if (sms <= 0) return AMOEBA_ERR_CUDA;
+    if (!a.free_mask && a.num_seqs > 0) {  // ids that can repeat: who is first
+        const int64_t work = a.reshape ? entries : std::min<int64_t>(a.pairs_cap, entries);
+        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, (int64_t)sms * 8));
+        bt_claim<<<grid, 256, 0, stream>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+        count_launch();
+    }
     const int64_t units = std::max<int64_t>((int64_t)a.num_seqs * ((a.maxb + kSegment - 1) / kSegment),
                                             a.reshape ? (a.nb_dst + 31) / 32 : 0);
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((units + 7) / 8, (int64_t)sms * 8));

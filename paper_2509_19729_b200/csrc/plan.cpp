@@ -478,6 +478,10 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
                 if (value > 2) return AMOEBA_ERR_INVALID_ARG;
                 k->tensor_maps = (int)value;
                 break;
+            case AMOEBA_OPT_L2_PROMOTION:
+                if (value > 4) return AMOEBA_ERR_INVALID_ARG;
+                k->l2_promotion = (int)value;
+                break;
             case AMOEBA_OPT_WAIT_TRIES:
                 if (value > (int64_t(1) << 30)) return AMOEBA_ERR_INVALID_ARG;
                 k->wait_tries = (int)value;

@@ -54,6 +54,7 @@ struct KernelOpts {
     int hint = 0;         // 1 + bit mask: bit 0 loads evict-first, bit 1 stores evict-first (0 = default)
     int max_ctas = 0;     // cap on the persistent grid (0 = none): leaves SMs free for kernels that run beside the copy
     int tensor_maps = 0;  // KV only: 1 = row copies on token-first sides, 2 = tensor-map boxes (0 = default)
+    int l2_promotion = 0; // KV only: 1 + CUtensorMapL2promotion of the token-first pools' tensor maps (0 = default)
     int wait_tries = 0;   // polls of one bounded mbarrier wait before the kernel gives up (0 = default)
 };
 

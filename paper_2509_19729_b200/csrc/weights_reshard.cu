@@ -8,52 +8,9 @@
 #include "copy_engine.cuh"
 #include "launch.hpp"
 #include "plan.hpp"
+#include "w_items.cuh"
 
 namespace amoeba {
-
-struct WParams {
-    WDescDev descs[kMaxWeightDescs];
-    void* ptrs[kMaxWeightPtrs];  // [layer][src rank][tensor] then, from dst_base, [layer][dst rank][tensor]
-    int32_t n_descs, items_per_layer, n_layers, src_tp, dst_tp, dst_base;
-};
-
-struct WItems {
-    const WParams& p;
-    __device__ __forceinline__ int64_t count() const { return (int64_t)p.items_per_layer * p.n_layers; }
-    __device__ __forceinline__ Item operator()(int64_t w) const {
-        const int32_t layer = (int32_t)(w / p.items_per_layer);
-        const int32_t rem = (int32_t)(w - (int64_t)layer * p.items_per_layer);
-        int lo = 0, hi = p.n_descs - 1;  // last descriptor with item_begin <= rem
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (p.descs[mid].item_begin <= rem) lo = mid;
-            else hi = mid - 1;
-        }
-        const WDescDev& d = p.descs[lo];
-        const int32_t local = rem - d.item_begin;
-        const int32_t rg = local / d.col_chunks, cc = local - rg * d.col_chunks;
-        const int32_t r0 = rg * d.rows_per_item;
-        const int64_t off = (int64_t)cc * d.chunk_bytes;
-        Item it;
-        it.src_map = it.dst_map = nullptr;
-        it.n_rows = min(d.rows_per_item, d.n_rows - r0);
-        it.row_bytes = (int32_t)min((int64_t)d.chunk_bytes, d.row_bytes - off);
-        it.src_pitch = d.src_pitch;
-        it.dst_pitch = d.dst_pitch;
-        const char* s = static_cast<const char*>(p.ptrs[(layer * p.src_tp) * kNumTensors + d.src_slot]);
-        char* t = static_cast<char*>(p.ptrs[p.dst_base + (layer * p.dst_tp) * kNumTensors + d.dst_slot]);
-        if (!t) {  // this destination worker's buffers were not given: its shard is not produced by this call
-            it.n_rows = 0;
-            it.row_bytes = 0;
-            it.src = nullptr;
-            it.dst = nullptr;
-            return it;
-        }
-        it.src = s + d.src_off + r0 * d.src_pitch + off;
-        it.dst = t + d.dst_off + r0 * d.dst_pitch + off;
-        return it;
-    }
-};
 
 template <int UNROLL, int CTAS_PER_SM>
 __global__ void __launch_bounds__(256, CTAS_PER_SM) w_reshard_ldst(const __grid_constant__ WParams p) {
@@ -86,8 +43,6 @@ __global__ void __launch_bounds__(1024) w_reshard_pair(const __grid_constant__ W
     if (!ok && (threadIdx.x & 31) == 0) atomicCAS(status, 0, (int)AMOEBA_ERR_TIMEOUT);
 }
 
-static void* const* slots(const amoeba_layer_weights* w) { return reinterpret_cast<void* const*>(w); }
-
 // Launches the copy kernel over `descs` (per-layer descriptors in kernel form, `items_per_layer` work items) for the
 // layers [layer_begin, layer_end): src is [src_tp][L], dst is [dst_tp][L] (worker-major host arrays of device pointers).
 static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDescDev>& descs, int32_t items_per_layer,
@@ -100,30 +55,14 @@ static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDe
     if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     const KernelOpts& opt = plan->opt.w;
     const int path = opt.copy_path ? opt.copy_path : kWDefaults.copy_path;
-    int stage_bytes = 16;
-    for (const WDescDev& d : descs)
-        stage_bytes = std::max<int64_t>(stage_bytes, (int64_t)d.rows_per_item * d.chunk_bytes);
+    const int stage_bytes = w_stage_bytes(descs);
     const int a = src_tp, b = dst_tp;
-    const int layers_per_launch = std::max(1, kMaxWeightPtrs / ((a + b) * kNumTensors));
+    const int layers_per_launch = weight_layers_per_launch(a, b);
 
     WParams p;  // large: filled per launch
-    p.n_descs = n_descs;
-    p.items_per_layer = items_per_layer;
-    p.src_tp = a;
-    p.dst_tp = b;
-    for (int i = 0; i < n_descs; ++i) p.descs[i] = descs[i];
     for (int l0 = layer_begin; l0 < layer_end; l0 += layers_per_launch) {
         const int nl = std::min(layers_per_launch, layer_end - l0);
-        p.n_layers = nl;
-        p.dst_base = nl * a * kNumTensors;
-        for (int l = 0; l < nl; ++l) {
-            for (int r = 0; r < a; ++r)
-                for (int t = 0; t < kNumTensors; ++t)
-                    p.ptrs[(l * a + r) * kNumTensors + t] = slots(&src[(size_t)r * L + l0 + l])[t];
-            for (int r = 0; r < b; ++r)
-                for (int t = 0; t < kNumTensors; ++t)
-                    p.ptrs[p.dst_base + (l * b + r) * kNumTensors + t] = slots(&dst[(size_t)r * L + l0 + l])[t];
-        }
+        w_fill_params(p, descs, items_per_layer, src, a, dst, b, L, l0, nl);
         const int64_t n_items = (int64_t)p.items_per_layer * nl;
         cudaError_t e;
         if (path == 1) {
@@ -161,23 +100,8 @@ extern "C" amoeba_status amoeba_reshard_weights(const amoeba_plan* plan, const a
     if (!plan || !src || !dst || !d_status) return AMOEBA_ERR_INVALID_ARG;
     const int L = plan->src.model.num_layers, a = plan->src.tp, b = plan->dst.tp;
     if (layer_begin < 0 || layer_end > L || layer_begin > layer_end) return AMOEBA_ERR_INVALID_ARG;
-    // Every buffer a descriptor names must be present and aligned, for every requested layer - except that a
-    // destination worker may be left out of a layer altogether (all seven pointers NULL): its shard is then not produced.
-    auto left_out = [&](int rank, int l) {
-        void* const* sl = slots(&dst[(size_t)rank * L + l]);
-        for (int t = 0; t < kNumTensors; ++t)
-            if (sl[t]) return false;
-        return true;
-    };
-    for (int l = layer_begin; l < layer_end; ++l)
-        for (const WDescDev& d : plan->wdev) {
-            const int dst_rank = d.dst_slot / kNumTensors;
-            const void* t = slots(&dst[(size_t)dst_rank * L + l])[d.dst_slot % kNumTensors];
-            if (!t && left_out(dst_rank, l)) continue;
-            const void* s = slots(&src[(size_t)(d.src_slot / kNumTensors) * L + l])[d.src_slot % kNumTensors];
-            if (!s || !t || s == t) return AMOEBA_ERR_INVALID_ARG;  // out of place: never the same buffer
-            if (reinterpret_cast<uintptr_t>(s) % 16 || reinterpret_cast<uintptr_t>(t) % 16) return AMOEBA_ERR_ALIGNMENT;
-        }
+    const amoeba_status ptrs_ok = w_check_ptrs(plan, src, dst, layer_begin, layer_end);
+    if (ptrs_ok != AMOEBA_OK) return ptrs_ok;
     return launch_descs(plan, plan->wdev, plan->items_per_layer, src, a, dst, b, L, layer_begin, layer_end, d_status,
                         static_cast<cudaStream_t>(cuda_stream));
 }
