@@ -409,7 +409,7 @@ static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void
     if (dev.sms <= 0) return AMOEBA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int path = opt.copy_path == 2 ? 2 : 3;  // a swap needs a staged copy: the rings only
-    const BulkShape bs = bulk_shape(dev, opt, kKvDefaults, path, (int)(2 * p.chunk_bytes));
+    const BulkShape bs = bulk_shape(dev, opt, kMergeDefaults, path, (int)(2 * p.chunk_bytes));
     const int64_t n_items = (int64_t)p.n_layers * p.nb * p.a * p.n_pairs * p.chunks_per_seg;
     const int grid = (int)std::min<int64_t>((n_items + bs.rings - 1) / bs.rings, grid_cap(opt, (int64_t)dev.sms * bs.ctas_per_sm));
     auto kernel = path == 3 ? kv_merge_pair : kv_merge_bulk;
