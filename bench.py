@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 # disjoint memory).  It is a stored counter reading, not something this script measures: the line says so in
 # "traffic_source", and it is only quoted for that workload with default kernel options (None = no reading for the
 # current kernel).
-NCU_KV_TRAFFIC_RATIO = None
+NCU_KV_TRAFFIC_RATIO = 0.9895
 NCU_KV_TRAFFIC_CONFIG = "llama3_8b_1to4"
 NCU_KV_TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1-layer slice, scaled by units processed"
 
@@ -452,6 +452,64 @@ def run_reshape(args, rank, world, local):
     }))
 
 
+def run_compact(args, rank, world, local):
+    """Partial swap of the weights in place (TP a -> b = N*a): every TP=a worker moves the N-th of its shards it keeps
+    (--keep, default the last) to the front of its buffers.  One step = one amoeba_compact_weights_inplace call over
+    all layers.  (Steps after the first move whatever the buffers then hold: the same bytes, the same addresses.)"""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    cfg = wl.CONFIGS[args.config]
+    s, st = build_session(args.config, device, layers=args.layers, kv=False, fill=False)
+    for item in args.opt:
+        name, val = item.split("=")
+        s.set_option(getattr(A, "OPT_" + name.upper()) + A.OPT_WEIGHTS_ONLY, int(val))
+    N = cfg["b"] // cfg["a"]
+    keep = [args.keep if args.keep is not None else N - 1] * cfg["a"]
+    nbytes = A.amoeba_compact_bytes(s.plan, keep) * s.L // cfg["model"]["L"]
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        A.amoeba_compact_weights_inplace(s.plan, s._src_w_packed, keep, 0, s.L, s.status)
+    torch.cuda.synchronize()
+    assert int(s.status.item()) == 0
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = A.amoeba_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(args.steps):
+        A.amoeba_compact_weights_inplace(s.plan, s._src_w_packed, keep, 0, s.L, s.status)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    barrier(world)
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0
+    sec_all, bytes_all = aggregate(world, t0.elapsed_time(t1) / 1e3 / args.steps, nbytes, device)
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    gbs = bytes_all / sec_all / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": sec_all * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']} weights compacted in place", "keep": keep,
+                   "layers": s.L, "kv_bytes_rw": 0, "weight_bytes_rw": nbytes, "extra_weight_memory_bytes": 0,
+                   "launches_per_call": launches / args.steps, "options": args.opt,
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
+        "roofline": {"kernel": "w_reshard_pair", "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                     "frac": gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": None,
+    }))
+
+
 def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, fill=True):
     import torch
 
@@ -798,6 +856,10 @@ def main():
     ap.add_argument("--inplace", action="store_true",
                     help="reshape the one instance in place (block reshaping) instead of copying it into fresh pools; "
                          "KV cache only, TP degrees must be multiples")
+    ap.add_argument("--compact-weights", action="store_true",
+                    help="time the in-place partial swap of the weights (amoeba_compact_weights_inplace) instead of the "
+                         "transformation; TP degrees must be multiples")
+    ap.add_argument("--keep", type=int, default=None, help="--compact-weights: which N-th every worker keeps")
     ap.add_argument("--no-all-configs", action="store_true",
                     help="skip the short timing of the other benchmark configurations")
     ap.add_argument("--no-e2e", action="store_true")
@@ -817,6 +879,9 @@ def main():
 
     if args.inplace:
         run_reshape(args, rank, world, local)
+        return
+    if args.compact_weights:
+        run_compact(args, rank, world, local)
         return
 
     import torch
