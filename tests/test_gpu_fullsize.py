@@ -1,10 +1,14 @@
 """Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times.
 
 The source buffers are filled on the device with a counter hash; the tables are compared whole with the oracle's.
-KV: three whole layers (the first, the last, one drawn at random) of EVERY destination pool are compared element by
-element - live blocks, idle blocks and foreign blocks alike - with the oracle's transformation of the same layer,
-streamed layer by layer through host memory; on the other layers sampled (layer, sequence, block) units are
-re-laid-out by the oracle one by one.  Weights: sampled layers compared whole."""
+KV: whole layers of EVERY destination pool are compared element by element - live blocks, idle blocks and foreign blocks
+alike - with the oracle's transformation of the same layers, streamed through host memory a few layers at a time (the
+oracle's layer loop on as many threads): ALL layers of the headline configuration, three layers (the first, the last,
+one drawn at random) of the others; on the remaining layers sampled (layer, sequence, block) units are re-laid-out by
+the oracle one by one.  Weights: all layers of the headline configuration, three of the others, compared whole."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 
@@ -14,6 +18,9 @@ pytestmark = pytest.mark.gpu
 
 FULL = ["llama3_8b_1to4", "llama3_8b_2to8", "llama2_7b_1to2", "llama2_13b_4to1", "llama3_70b_slice_8to2"]
 
+
+HEADLINE = "llama3_8b_1to4"  # compared completely: every layer of every destination buffer
+GROUP_BYTES = 12 << 30       # source KV bytes streamed through host memory per oracle call
 
 CASES = [(n, "head") for n in FULL] + [("llama3_8b_1to4", "token"), ("llama3_70b_slice_8to2", "token2head"),
                                        ("llama2_7b_1to2", "head2token")]
@@ -78,22 +85,47 @@ def test_full_size_config(name, kv_order, oracle):
                 got = dst_v[r][l, did].cpu().numpy().view(np.uint16)
                 assert np.array_equal(got, exp1[r]), (name, l, q, i, r)
 
-        # ---- KV: whole layers, every word of every destination pool (live, idle and foreign blocks)
-        for l in sorted({0, Lkv - 1, int(g.integers(Lkv))}):
-            src1 = [p.view(Lkv, -1)[l].cpu().numpy().view(np.uint16) for p in s.src_pools]
-            exp1 = [np.full(p.numel() // Lkv // 2, 0xA5A5, np.uint16) for p in s.dst_pools]
-            oracle.kv_transform(one, T, st["seq_lens"], a, st["NB_src"], st["src_bt"], src1, b, st["NB_dst"], exp_bt,
-                                exp1, src_order=so, dst_order=do)
-            del src1
-            for r in range(b):
-                got = s.dst_pools[r].view(Lkv, -1)[l].cpu().numpy().view(np.uint16)
-                if not np.array_equal(got, exp1[r]):
-                    bad = np.flatnonzero(got != exp1[r])
-                    raise AssertionError(f"{name} layer {l} dst pool {r}: {bad.size} words differ, first at {bad[0]}")
-            del exp1
+        # ---- KV: whole layers, every word of every destination pool (live, idle and foreign blocks); consecutive
+        # layers go through the oracle together, its layer loop on one thread per layer
+        everything = name == HEADLINE and kv_order == "head"
+        layers = list(range(Lkv)) if everything else sorted({0, Lkv - 1, int(g.integers(Lkv))})
+        src_layer_bytes = sum(p.numel() for p in s.src_pools) // Lkv
+        per_call = max(1, min(os.cpu_count() or 1, 16, GROUP_BYTES // src_layer_bytes))
+        groups = [[layers[0]]]
+        for l in layers[1:]:
+            if l == groups[-1][-1] + 1 and len(groups[-1]) < per_call:
+                groups[-1].append(l)
+            else:
+                groups.append([l])
+        exp_n_layers, exp_grp = 0, None
+        try:
+            for grp in groups:
+                l0, nl = grp[0], len(grp)
+                oracle.set_threads(nl)
+                src_grp = [p.view(Lkv, -1)[l0:l0 + nl].cpu().numpy().view(np.uint16).reshape(-1) for p in s.src_pools]
+                if exp_n_layers != nl:
+                    exp_grp = [np.empty(p.numel() // Lkv // 2 * nl, np.uint16) for p in s.dst_pools]
+                    exp_n_layers = nl
+                for e in exp_grp:
+                    e.fill(0xA5A5)
+                oracle.kv_transform(dict(m, L=nl), T, st["seq_lens"], a, st["NB_src"], st["src_bt"], src_grp, b,
+                                    st["NB_dst"], exp_bt, exp_grp, src_order=so, dst_order=do)
+                del src_grp
+                for r in range(b):
+                    got = s.dst_pools[r].view(Lkv, -1)[l0:l0 + nl].cpu().numpy().view(np.uint16).reshape(-1)
+                    if not np.array_equal(got, exp_grp[r]):
+                        bad = np.flatnonzero(got != exp_grp[r])
+                        raise AssertionError(f"{name} layers {l0}..{l0 + nl - 1} dst pool {r}: {bad.size} words differ, "
+                                             f"first at {bad[0]}")
+                    del got
+        finally:
+            oracle.set_threads(1)
+            del exp_grp
 
-        # ---- weights: whole comparison of sampled layers
-        for l in sorted(set([0, m["L"] - 1, int(g.integers(m["L"]))])):
+        # ---- weights: whole layers (the C calls release the interpreter lock: a few layers at a time)
+        w_layers = list(range(m["L"])) if everything else sorted({0, m["L"] - 1, int(g.integers(m["L"]))})
+
+        def check_weights(l):
             src_sh = [{n: t.cpu().numpy().view(np.uint16).reshape(oracle.shard_shapes(m, a)[n])
                        for n, t in s.src_w[r][l].items()} for r in range(a)]
             exp = oracle.weights_transform(src_sh, m, a, b)
@@ -101,6 +133,9 @@ def test_full_size_config(name, kv_order, oracle):
                 for n, e in exp[r].items():
                     got = s.dst_w[r][l][n].cpu().numpy().view(np.uint16)
                     assert np.array_equal(got, e.reshape(-1)), (name, "weights", l, r, n)
+
+        with ThreadPoolExecutor(max_workers=min(os.cpu_count() or 1, 8)) as pool:
+            list(pool.map(check_weights, w_layers))
     finally:
         del s
         torch.cuda.empty_cache()
