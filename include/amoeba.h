@@ -31,7 +31,9 @@
  *   - Thread-compatible.  Process-wide state is limited to an atomic launch counter and a few lock-protected
  *     look-up caches (device attributes, the shared-memory opt-in of each kernel, the driver's tensor-map encoder,
  *     the built-in scratch address per device); a plan also caches the tensor maps it encoded for the last set of
- *     pool addresses.  A plan may be used from several threads if its options are not changed concurrently.
+ *     pool addresses.  The per-device caches assume that a device's primary context lives as long as the process: after a
+ *     cudaDeviceReset of a device the library must not be used on that device any more.  A plan may be used from
+ *     several threads if its options are not changed concurrently.
  *     No C++ exception crosses this boundary (a failed host allocation is AMOEBA_ERR_NO_MEMORY).
  *   - AMOEBA_ERR_TIMEOUT: every on-device wait of a kernel on one of its own bulk copies is bounded.  A kernel whose
  *     wait runs out records the code in *d_status, waits (bounded again) for the copies it still has in flight and

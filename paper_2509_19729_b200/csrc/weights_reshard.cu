@@ -132,18 +132,38 @@ struct LeadParams {
     int32_t n;                   // N
 };
 
-__global__ void __launch_bounds__(256) w_compact_lead(const __grid_constant__ LeadParams p) {
+constexpr int kLeadThreads = 1024;
+constexpr int kLeadUnroll = 8;  // 16-byte loads in flight per thread: 128 KiB per CTA
+
+__global__ void __launch_bounds__(kLeadThreads, 1) w_compact_lead(const __grid_constant__ LeadParams p) {
     const int b = blockIdx.x, c = p.cls[b];
     char* base = p.bufs[b];
     const int64_t w_old = p.w_old[c], w_new = p.w_new[c], keep_off = p.keep[b] * w_new;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int vpr = (int)(w_new >> 4);  // 16-byte vectors per row
     int64_t lo = 0, hi = 1;
     while (lo < p.rows[c]) {
         if (hi > p.rows[c]) hi = p.rows[c];
-        for (int64_t row = lo + warp; row < hi; row += nwarps) {
-            if (row == 0 && keep_off == 0) continue;  // already in place
-            copy_vecs<8>(reinterpret_cast<const uint4*>(base + row * w_old + keep_off),
-                         reinterpret_cast<uint4*>(base + row * w_new), (int)(w_new >> 4), lane, 32);
+        // the wave's rows as one flat list of vectors, dealt to all threads; every load of a batch before its stores
+        const int first = (lo == 0 && keep_off == 0) ? vpr : 0;  // row 0 of the first column range is in place
+        const int n = (int)(hi - lo) * vpr;
+        for (int i0 = first + threadIdx.x; i0 < n; i0 += kLeadThreads * kLeadUnroll) {
+            uint4 v[kLeadUnroll];
+#pragma unroll
+            for (int u = 0; u < kLeadUnroll; ++u) {
+                const int i = i0 + u * kLeadThreads;
+                if (i < n) {
+                    const int r = i / vpr, col = i - r * vpr;
+                    v[u] = ld_stream(reinterpret_cast<const uint4*>(base + (lo + r) * w_old + keep_off) + col);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kLeadUnroll; ++u) {
+                const int i = i0 + u * kLeadThreads;
+                if (i < n) {
+                    const int r = i / vpr, col = i - r * vpr;
+                    st_stream(reinterpret_cast<uint4*>(base + (lo + r) * w_new) + col, v[u]);
+                }
+            }
         }
         __syncthreads();  // every load of this wave has returned (its stores were issued after them)
         lo = hi;
@@ -185,10 +205,20 @@ static void compact_schedule(const amoeba_plan* plan, const int32_t* keep, Compa
         if (phases.size() <= i) phases.resize(i + 1);
         return phases[i];
     };
+    // Inside a fused [q;k;v] buffer v may move together with k when its new place ends before the rows k is read
+    // from (for every worker): (Rq + 2 Rk)/b <= Rq/a + keep*Rk/b.  Separate buffers never wait for one another.
+    bool v_with_k = true;
+    if (sl.fused_qkv)
+        for (int r = 0; r < a; ++r)
+            v_with_k = v_with_k && (rows_of[Q] + 2 * rows_of[K]) / b <= rows_of[Q] / a + keep[r] * (rows_of[K] / b);
     const int chains[2][3] = {{Q, K, V}, {GATE, UP, -1}};
     for (const auto& chain : chains)
-        for (int step = 0; step < 3 && chain[step] >= 0; ++step) {
-            const int t = chain[step];
+        for (int pos = 0; pos < 3 && chain[pos] >= 0; ++pos) {
+            const int t = chain[pos];
+            int step = pos;
+            if (!sl.fused_qkv && (t == K || t == V)) step = 0;        // buffers of their own
+            else if (t == V && v_with_k) step = 1;
+            if (!sl.fused_gate_up && t == UP) step = 0;
             for (int r = 0; r < a; ++r) {
                 amoeba_weight_desc d{};
                 d.src_rank = d.dst_rank = r;
@@ -290,7 +320,7 @@ static amoeba_status compact_weights_inplace(const amoeba_plan* plan, const amoe
         int n = 0;
         auto flush = [&]() -> amoeba_status {
             if (n == 0) return AMOEBA_OK;
-            w_compact_lead<<<n, 256, 0, stream>>>(lp);
+            w_compact_lead<<<n, kLeadThreads, 0, stream>>>(lp);
             if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
             count_launch();
             n = 0;

@@ -573,12 +573,27 @@ def test_l2_hints_on_bulk_and_tiled_copies(hint, so, do):
 def test_weights_compacted_in_place(path, fq, fg, a, b, keep):
     """After the call the front of worker r's buffers is the dense TP = b shard of worker r*N + keep[r], byte for byte
     what the oracle's a -> b transformation gives that worker."""
+    m = dict(L=2, hidden=96, Hq=16, Hkv=8, D=16, I=320)   # 96 rows: the waves of the column tensors end raggedly
+    _compact_case(m, path, fq, fg, a, b, keep)
+
+
+@pytest.mark.parametrize("fq", [True, False])
+@pytest.mark.parametrize("hidden", [96, 1200])
+@pytest.mark.parametrize("a,b,keep", [(1, 2, [0]), (1, 2, [1]), (2, 4, [0, 1]), (1, 4, [0]), (1, 4, [3])])
+def test_weights_compacted_in_place_mha(fq, hidden, a, b, keep):
+    """As many K/V heads as query heads: with N = 2 the new v section would land on rows k is still read from, so v
+    moves one launch after k; hidden = 1200 takes the column tensors past the rows one CTA moves alone, with a ragged
+    last wave."""
+    m = dict(L=2, hidden=hidden, Hq=8, Hkv=8, D=16, I=320)
+    _compact_case(m, PAIR, fq, True, a, b, keep)
+
+
+def _compact_case(m, path, fq, fg, a, b, keep):
     import torch
 
     import oracle as O
     import paper_2509_19729_b200 as A
 
-    m = dict(L=2, hidden=96, Hq=16, Hkv=8, D=16, I=320)   # 96 rows: the waves of the column tensors end raggedly
     N = b // a
     dev = torch.device("cuda:0")
     g = np.random.default_rng(a * 31 + b + sum(keep))
