@@ -728,7 +728,7 @@ def run_e2e(args, device, world):
     cfg = wl.CONFIGS[args.config]
     L_full = cfg["model"]["L"]
     # size the layer slice so that the pinned host buffers stay within the cap
-    budget = min(int(args.e2e_gib * 2**30), host_free_bytes() // 3)
+    budget = min(int(args.e2e_gib * 2**30), host_free_bytes() // (3 * max(world, 1)))  # every rank pins its own copy
     s1, st = build_session(args.config, device, layers=1, fill=False, kv_order=args.kv_order,
                            weight_pad=args.weight_pad)
     per_layer = sum(p.numel() for p in s1.src_pools + s1.dst_pools + s1._wbufs)

@@ -330,3 +330,25 @@ def test_compact_bytes_counts_only_what_moves():
     with pytest.raises(A.AmoebaError) as err:
         A.amoeba_compact_bytes(plan, [4])
     assert err.value.status == A.ERR_INVALID_ARG
+
+
+def test_reshape_plans_are_recognised_on_the_host():
+    """In-place reshaping needs TP degrees and block counts that are multiples of each other by the same factor,
+    header-centric pools and one layer stride; the bytes it moves are (N-1)/N of the blocks."""
+    m = GQA
+    unit = 2 * 16 * m["D"] * 2
+    for a, N, NB in ((1, 4, 10), (2, 2, 7), (2, 4, 3)):
+        split = A.amoeba_plan_create(A.make_layout(m, a, NB), A.make_layout(m, a * N, NB * N))
+        back = A.amoeba_plan_create(A.make_layout(m, a * N, NB * N), A.make_layout(m, a, NB))
+        expect = 2 * 5 * m["L"] * (m["Hkv"] // N) * (N - 1) * unit
+        assert A.amoeba_reshape_bytes(split, 5) == expect == A.amoeba_reshape_bytes(back, 5)
+        kv, _ = A.amoeba_plan_bytes(split, 5)
+        assert expect * N == kv * (N - 1)
+    for src, dst in ((A.make_layout(m, 1, 10), A.make_layout(m, 4, 41)),                 # block counts do not match
+                     (A.make_layout(m, 2, 10), A.make_layout(m, 2, 10)),                 # same TP degree
+                     (A.make_layout(m, 1, 10, kv_order=A.KV_TOKEN_MAJOR), A.make_layout(m, 4, 40)),
+                     (A.make_layout(m, 1, 10), A.make_layout(m, 4, 40, kv_layer_stride_bytes=1 << 20))):
+        plan = A.amoeba_plan_create(src, dst)
+        with pytest.raises(A.AmoebaError) as e:
+            A.amoeba_reshape_bytes(plan, 1)
+        assert e.value.status == A.ERR_UNSUPPORTED
