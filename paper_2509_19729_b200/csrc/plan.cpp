@@ -100,10 +100,10 @@ WDescDev chunk_desc(const amoeba_weight_desc& d, int64_t cap, int64_t* item) {
     w.n_rows = d.n_rows;
     w.src_slot = d.src_rank * kNumTensors + d.src_tensor;
     w.dst_slot = d.dst_rank * kNumTensors + d.dst_tensor;
-    if (d.row_bytes > cap) {
+    if (d.row_bytes > cap) {  // cut a long row into the fewest chunks of (nearly) equal size
         w.rows_per_item = 1;
         w.col_chunks = (int32_t)((d.row_bytes + cap - 1) / cap);
-        w.chunk_bytes = (int32_t)cap;
+        w.chunk_bytes = (int32_t)(((d.row_bytes + w.col_chunks - 1) / w.col_chunks + 15) / 16 * 16);
     } else {
         w.rows_per_item = (int32_t)std::min<int64_t>(std::max<int64_t>(1, cap / d.row_bytes), d.n_rows);
         w.col_chunks = 1;
