@@ -98,7 +98,7 @@ __device__ __forceinline__ uint32_t nonzero_bytes(uint32_t w) {
 
 // All kScanThreads threads of ONE CTA.
 __device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     if (tid == 0) flags[0] = flags[1] = 0;  // [0] bad length, [1] whole-call error
     __syncthreads();
 
