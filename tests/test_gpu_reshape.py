@@ -225,3 +225,60 @@ def test_large_tables_take_the_two_launch_path(oracle):
     lens, bt, old = _coarse_instance(oracle, m, T, a, NB, lens_in, seed=8)
     assert bt.size > 128 * 1024
     _check(oracle, "split", m, T, N, a, NB, lens, bt, _with_fresh(old, N))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_reshapes_with_layer_strides(oracle, seed):
+    """Random factor, TP degree, lengths, direction, copy path, item size and a layer stride larger than a dense
+    layer: every byte of every (strided) pool, the words between the layers included."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    g = np.random.default_rng(1000 + seed)
+    m = dict(L=3, hidden=64, Hq=16, Hkv=16, D=16, I=256)
+    T = int(g.choice([4, 8, 16]))
+    N = int(g.choice([2, 4, 8]))
+    a = int(g.choice([x for x in (1, 2, 4, 8) if x * N <= 16]))
+    direction = str(g.choice(["split", "merge"]))
+    lens = g.integers(0 if direction == "split" else 1, 12 * T, size=int(g.integers(1, 9))).astype(np.int32)
+    NB = int(((lens + T - 1) // T).sum()) + int(g.integers(1, 9))
+    dense = oracle.pool_elems_per_layer(m, T, a, NB)
+    stride = dense + 8 * int(g.integers(0, 40))  # elements; a multiple of 16 bytes
+    if direction == "split":
+        lens, bt, old = _coarse_instance(oracle, m, T, a, NB, lens, seed=seed)
+        dense_pools = _with_fresh(old, N)
+    else:
+        lens, bt, dense_pools = _fine_instance(oracle, m, T, N, a, NB, lens, seed=seed)
+    pools = []
+    for w, p in enumerate(dense_pools):
+        q = np.full(m["L"] * stride, 0x7000 + w, np.uint16)
+        q.reshape(m["L"], stride)[:, :dense] = p.reshape(m["L"], dense)
+        pools.append(q)
+    exp = [p.copy() for p in pools]
+    e_bt, e_pairs, e_n, e_mask, e_left, e_status = oracle.kv_reshape_inplace(direction, m, T, N, a, NB, lens, bt, exp,
+                                                                             layer_stride=stride)
+    coarse = A.make_layout(m, a, NB, T, kv_layer_stride_bytes=stride * 2)
+    fine = A.make_layout(m, N * a, NB * N, T, kv_layer_stride_bytes=stride * 2)
+    plan = A.amoeba_plan_create(*((coarse, fine) if direction == "split" else (fine, coarse)))
+    A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, int(g.choice([1, 2, 3])))
+    A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, int(g.choice([64, 512, 8192])))
+    dev = torch.device("cuda:0")
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_pools = [torch.from_numpy(p.view(np.uint8).copy()).to(dev) for p in pools]
+    d_bt, d_lens = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+    d_new = torch.full(bt.shape, -2, **i32)
+    d_pairs = torch.full((bt.size, 2), -3, **i32)
+    d_n, d_left, d_status = torch.zeros(1, **i32), torch.zeros(1, **i32), torch.zeros(1, **i32)
+    d_mask = torch.full((NB * N if direction == "split" else NB,), 7, dtype=torch.uint8, device=dev)
+    ws_bytes = A.amoeba_rewrite_workspace_bytes(plan, len(lens), 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    A.amoeba_reshape_block_tables(plan, d_bt, d_lens, len(lens), bt.shape[1], d_new, d_pairs, bt.size, d_n, d_mask,
+                                  d_left, d_status, ws, ws_bytes)
+    A.amoeba_reshape_kv_inplace(plan, d_pools, d_pairs, d_n, bt.size, 0, m["L"], d_status)
+    torch.cuda.synchronize()
+    assert int(d_status.item()) == e_status == 0
+    assert np.array_equal(d_new.cpu().numpy(), e_bt) and int(d_n.item()) == e_n and int(d_left.item()) == e_left
+    assert np.array_equal(d_pairs.cpu().numpy()[:e_n], e_pairs) and np.array_equal(d_mask.cpu().numpy(), e_mask)
+    for w, (t, e) in enumerate(zip(d_pools, exp)):
+        assert np.array_equal(t.cpu().numpy().view(np.uint16), e), (w, direction, N, a, T)
