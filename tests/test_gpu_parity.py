@@ -706,3 +706,70 @@ def test_wait_budget_running_out_is_reported_and_the_next_call_is_exact(path):
     s.step()
     torch.cuda.synchronize()
     check_case(c, s)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_tables_with_damaged_inputs(seed):
+    """The table kernels alone on random inputs, small enough for one launch or large enough for three: lengths with
+    zeros, free lists with repeated and out-of-range ids, source tables with holes and out-of-range ids, masks, too
+    few free blocks, a pair capacity that is too small - every output word against the oracle."""
+    import torch
+
+    import oracle as O
+    import paper_2509_19729_b200 as A
+
+    g = np.random.default_rng(5000 + seed)
+    T = 16
+    big = seed % 3 == 2
+    S = int(g.integers(1, 400 if big else 40))
+    lens = g.integers(0, (60 if big else 12) * T, size=S).astype(np.int32)
+    lens[g.random(S) < 0.15] = 0
+    nblk = (lens + T - 1) // T
+    maxb = max(int(nblk.max()), 1) + int(g.integers(0, 3))
+    total = int(nblk.sum())
+    NB_src = total + int(g.integers(1, 50))
+    NB_dst = max(1, total + int(g.integers(-3, 60)))
+    bt = np.full((S, maxb), -1, np.int32)
+    ids, k = g.permutation(NB_src), 0
+    for s, n in enumerate(nblk):
+        bt[s, :n] = ids[k:k + n]
+        k += int(n)
+    live = np.argwhere(bt >= 0)
+    for s, i in live[g.random(len(live)) < 0.03]:      # holes and out-of-range source ids
+        bt[s, i] = int(g.choice([-1, NB_src, NB_src + 7]))
+    use_mask = seed % 2 == 1
+    free_list = free_mask = None
+    if use_mask:
+        free_mask = (g.random(NB_dst) < 0.8).astype(np.uint8)
+    else:
+        n_free = max(0, total + int(g.integers(-2, 20)))
+        free_list = g.integers(0, NB_dst, size=n_free).astype(np.int32) if seed % 4 == 0 \
+            else g.permutation(max(NB_dst, n_free))[:n_free].astype(np.int32)   # repeats / ids beyond the pool
+        if n_free:
+            free_list[g.random(n_free) < 0.02] = NB_dst + 3
+    pairs_cap = total if seed % 5 else max(0, total - 1)
+    if seed % 7 == 3 and S > 1:
+        lens[1] = -5
+    m = dict(L=1, hidden=128, Hq=8, Hkv=8, D=64, I=256)
+    plan = A.amoeba_plan_create(A.make_layout(m, 2, NB_src, T), A.make_layout(m, 4, NB_dst, T))
+    e_bt, e_pairs, e_n, e_left, e_st = O.assign_blocks(lens, T, bt, NB_src, NB_dst, free_list=free_list,
+                                                       free_mask=free_mask, pairs_cap=pairs_cap)
+    dev = torch.device("cuda:0")
+    i32 = dict(dtype=torch.int32, device=dev)
+    d_bt, d_lens = torch.from_numpy(bt).to(dev), torch.from_numpy(lens).to(dev)
+    d_new = torch.full(bt.shape, -2, **i32)
+    d_pairs = torch.full((max(pairs_cap, 1), 2), -3, **i32)
+    d_n, d_left, d_status = torch.zeros(1, **i32), torch.zeros(1, **i32), torch.zeros(1, **i32)
+    d_free = torch.from_numpy(free_list).to(dev) if free_list is not None and len(free_list) else \
+        (torch.zeros(1, **i32) if free_list is not None else None)
+    d_mask = torch.from_numpy(free_mask).to(dev) if use_mask else None
+    n_arg = NB_dst if use_mask else len(free_list)
+    ws_bytes = A.amoeba_rewrite_workspace_bytes(plan, S, n_arg)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    A.amoeba_rewrite_block_tables(plan, d_bt, d_lens, S, maxb, d_free, d_mask, n_arg, d_new, d_pairs, pairs_cap, d_n,
+                                  d_left, d_status, ws, ws_bytes)
+    torch.cuda.synchronize()
+    assert int(d_status.item()) == e_st
+    assert int(d_n.item()) == e_n and int(d_left.item()) == e_left
+    assert np.array_equal(d_new.cpu().numpy(), e_bt)
+    assert np.array_equal(d_pairs.cpu().numpy()[:e_n], e_pairs)
