@@ -510,6 +510,98 @@ def run_compact(args, rank, world, local):
     }))
 
 
+def run_beside(args, rank, world, local):
+    """The copy beside a compute kernel (Sec. 3.1, Improvement 2: the migration runs on a side stream while the SMs it
+    does not use keep computing).  The KV and weight calls of --layers layers (default 8) run with their grid capped at
+    --max-ctas CTAs on one stream while a dense bf16 GEMM (torch.matmul, a library kernel: the neighbour, not the
+    product) runs on another.  Reported: each alone, and each while the other one covers its whole timed region."""
+    import torch
+
+    import paper_2509_19729_b200 as A
+
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    s, st = build_session(args.config, device, layers=args.layers or 8, fill=False)
+    if args.max_ctas:
+        s.set_option(A.OPT_MAX_CTAS, args.max_ctas)
+    kv_bytes, w_bytes = s.bytes_rw(st["n_live"])
+    n = 8192
+    x = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    y = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    z = torch.empty(n, n, device=device, dtype=torch.bfloat16)
+    copy_stream, gemm_stream = torch.cuda.Stream(), torch.cuda.Stream()
+    s.rewrite_block_tables()
+    torch.cuda.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def copies(k):
+        a, b = ev(), ev()
+        with torch.cuda.stream(copy_stream):
+            a.record(copy_stream)
+            for _ in range(k):
+                s.reshard_kv(copy_stream)
+                s.reshard_weights(copy_stream)
+            b.record(copy_stream)
+        return a, b, k
+
+    def gemms(k):
+        a, b = ev(), ev()
+        with torch.cuda.stream(gemm_stream):
+            a.record(gemm_stream)
+            for _ in range(k):
+                torch.matmul(x, y, out=z)
+            b.record(gemm_stream)
+        return a, b, k
+
+    gbs = lambda t: (kv_bytes + w_bytes) * t[2] / (t[0].elapsed_time(t[1]) / 1e3) / 1e9
+    tfs = lambda t: 2.0 * n ** 3 * t[2] / (t[0].elapsed_time(t[1]) / 1e3) / 1e12
+    for _ in range(2):  # warm-up of both
+        copies(2), gemms(10)
+        torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = A.amoeba_launch_count()
+    c_alone = copies(4)
+    torch.cuda.synchronize()
+    g_alone = gemms(40)
+    torch.cuda.synchronize()
+    one_copy_ms = c_alone[0].elapsed_time(c_alone[1]) / 4
+    one_gemm_ms = g_alone[0].elapsed_time(g_alone[1]) / 40
+    # the copy inside a longer batch of GEMMs
+    k_g = int(6 * one_copy_ms / one_gemm_ms) + 20
+    g_long = gemms(k_g)
+    c_in = copies(3)
+    torch.cuda.synchronize()
+    # the GEMMs inside a longer batch of copies
+    k_c = int(30 * one_gemm_ms / one_copy_ms) + 4
+    c_long = copies(k_c)
+    g_in = gemms(20)
+    torch.cuda.synchronize()
+    launches = A.amoeba_launch_count() - launches0
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    assert int(s.status.item()) == 0
+    if rank != 0:
+        return
+    peak, peak_kind = peaks()
+    cfg = wl.CONFIGS[args.config]
+    print(json.dumps({
+        "metric": METRIC, "value": gbs(c_in), "unit": "GB/s", "n_gpus": world, "steps": 3, "warmup": 4,
+        "ms_per_step": c_in[0].elapsed_time(c_in[1]) / 3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.config, "tp": f"{cfg['a']}->{cfg['b']}", "layers": s.L,
+                   "max_ctas": args.max_ctas or "all SMs", "neighbour": f"torch.matmul bf16 {n}^3 on a second stream",
+                   "kv_bytes_rw": kv_bytes, "weight_bytes_rw": w_bytes,
+                   "l2_policy": "no flush: every step streams far more than the 126 MB L2"},
+        "copy_gbs": {"alone": gbs(c_alone), "beside_gemm": gbs(c_in)},
+        "gemm_tflops": {"alone": tfs(g_alone), "beside_copy": tfs(g_in)},
+        "roofline": {"kernel": "kv_reshard_pair + w_reshard_pair", "bound": "hbm", "achieved": gbs(c_in), "peak": peak,
+                     "unit": "GB/s", "frac": gbs(c_in) / peak, "peak_kind": f"of {peak_kind}", "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks, "e2e": None,
+    }))
+
+
 def build_merge_session(cfg_name: str, device, layers=None, seed=wl.DEFAULT_SEED, fill=True):
     import torch
 
@@ -856,6 +948,9 @@ def main():
     ap.add_argument("--inplace", action="store_true",
                     help="reshape the one instance in place (block reshaping) instead of copying it into fresh pools; "
                          "KV cache only, TP degrees must be multiples")
+    ap.add_argument("--beside-gemm", action="store_true",
+                    help="run the copy (grid capped by --max-ctas) while a dense GEMM runs on a second stream and "
+                         "report both throughputs, alone and together")
     ap.add_argument("--compact-weights", action="store_true",
                     help="time the in-place partial swap of the weights (amoeba_compact_weights_inplace) instead of the "
                          "transformation; TP degrees must be multiples")
@@ -882,6 +977,9 @@ def main():
         return
     if args.compact_weights:
         run_compact(args, rank, world, local)
+        return
+    if args.beside_gemm:
+        run_beside(args, rank, world, local)
         return
 
     import torch
