@@ -74,7 +74,8 @@ enum {
 enum { AMOEBA_MAX_TP = 32 }; /* and at most 36 intersecting (source worker, destination worker) pairs: 256 weight
                                 descriptors per layer; nested degrees up to 32 -> 1 and 1 -> 32 fit */
 
-/* Transformer shape.  elem_bytes is the size of one weight / KV element (2: fp16 or bf16). */
+/* Transformer shape.  elem_bytes is the size of one weight / KV element: 2 (fp16, bf16 - the paper's types), 1 (8-bit
+ * formats) or 4; the elements are moved, never interpreted.  Every contiguous run must still be a multiple of 16 bytes. */
 typedef struct {
     int32_t num_layers, hidden, num_q_heads, num_kv_heads, head_dim, intermediate, elem_bytes;
 } amoeba_model;

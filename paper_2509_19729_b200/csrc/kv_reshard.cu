@@ -182,7 +182,7 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Tensor map of one worker's token-first pool [layer][K/V][block][token][header][dim] (16-bit elements), with the
+// Tensor map of one worker's token-first pool [layer][K/V][block][token][header][dim] (1-, 2- or 4-byte elements), with the
 // dimensions ordered {dim, token, K/V, header, layer} so that a box lands in shared memory as
 // [header][K/V][token][dim]: the header-centric order of the same data.
 constexpr int kDefaultL2Promotion = 1;  // 1 + CU_TENSOR_MAP_L2_PROMOTION_NONE
@@ -200,7 +200,10 @@ static bool encode_pool_map(CUtensorMap* out, const void* pool, const amoeba_lay
                                    (cuuint64_t)layer_stride};
     const cuuint32_t box[5] = {(cuuint32_t)lay.model.head_dim, (cuuint32_t)bx.tokens, 2, (cuuint32_t)bx.heads, 1};
     const cuuint32_t elem_strides[5] = {1, 1, 1, 1, 1};
-    return encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 5, const_cast<void*>(pool), dims, strides, box, elem_strides,
+    const int e = lay.model.elem_bytes;  // the elements are opaque: any unsigned type of their size will do
+    const CUtensorMapDataType type = e == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                            : e == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;
+    return encode(out, type, 5, const_cast<void*>(pool), dims, strides, box, elem_strides,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, (CUtensorMapL2promotion)promo,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -24,7 +24,7 @@ static amoeba_status check_layout(const amoeba_layout& l) {
     if (m.num_layers <= 0 || m.hidden <= 0 || m.num_q_heads <= 0 || m.num_kv_heads <= 0 || m.head_dim <= 0 ||
         m.intermediate <= 0 || l.tp <= 0 || l.block_tokens <= 0 || l.num_blocks <= 0 || l.kv_layer_stride_bytes < 0)
         return AMOEBA_ERR_INVALID_ARG;
-    if (m.elem_bytes != 2) return AMOEBA_ERR_UNSUPPORTED;
+    if (m.elem_bytes != 1 && m.elem_bytes != 2 && m.elem_bytes != 4) return AMOEBA_ERR_UNSUPPORTED;
     if (l.kv_order != AMOEBA_KV_HEAD_MAJOR && l.kv_order != AMOEBA_KV_TOKEN_MAJOR) return AMOEBA_ERR_UNSUPPORTED;
     if (l.tp > AMOEBA_MAX_TP) return AMOEBA_ERR_UNSUPPORTED;
     // Even partition of the headers and of the FFN width over the workers; K/V header replication for

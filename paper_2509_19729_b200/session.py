@@ -37,13 +37,13 @@ class Session:
                  pairs_cap: int, kv_layers: Optional[int] = None, kv: bool = True, weights: bool = True,
                  fused_qkv: bool = True, fused_gate_up: bool = True, block_tokens: int = 16, device="cuda:0",
                  dst_fill: Optional[int] = 0xA5, src_kv_order: int = A.KV_HEAD_MAJOR,
-                 dst_kv_order: int = A.KV_HEAD_MAJOR, src_weight_pad=None, dst_weight_pad=None):
+                 dst_kv_order: int = A.KV_HEAD_MAJOR, src_weight_pad=None, dst_weight_pad=None, elem_bytes: int = 2):
         self.model, self.a, self.b = model, a, b
         self.device = torch.device(device)
         pad = lambda p: dict(weight_pad_parts=p[0], weight_page_bytes=p[1]) if p else {}  # (P, page bytes) or None
-        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up,
+        self.src_layout = A.make_layout(model, a, NB_src, block_tokens, fused_qkv, fused_gate_up, elem_bytes,
                                         kv_order=src_kv_order, **pad(src_weight_pad))
-        self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up,
+        self.dst_layout = A.make_layout(model, b, NB_dst, block_tokens, fused_qkv, fused_gate_up, elem_bytes,
                                         kv_order=dst_kv_order, **pad(dst_weight_pad))
         self.plan = A.amoeba_plan_create(self.src_layout, self.dst_layout)
         self.info = A.amoeba_plan_kv_info(self.plan)

@@ -773,3 +773,55 @@ def test_random_tables_with_damaged_inputs(seed):
     assert int(d_n.item()) == e_n and int(d_left.item()) == e_left
     assert np.array_equal(d_new.cpu().numpy(), e_bt)
     assert np.array_equal(d_pairs.cpu().numpy()[:e_n], e_pairs)
+
+
+@pytest.mark.parametrize("so,do", [(HC, HC), (TF, HC), (HC, TF)])
+@pytest.mark.parametrize("e,a,b", [(1, 2, 4), (1, 4, 1), (4, 1, 2), (4, 8, 2)])
+def test_element_sizes_one_and_four_bytes(e, a, b, so, do):
+    """Elements are opaque, so a state of e-byte elements is byte for byte a 16-bit state with the innermost extent
+    scaled by e/2: head_dim for the KV cache, the input width for the row-split weights, the column count for the
+    column-split ones.  The 16-bit oracle gives the expected bytes; the library runs with elem_bytes = e."""
+    import torch
+
+    import oracle as O
+    from paper_2509_19729_b200.session import Session
+
+    m = dict(L=2, hidden=256, Hq=16, Hkv=8, D=64, I=512)           # the model as the library sees it
+    scale = lambda x: x * e // 2
+    lens = [1, 16, 17, 200, 0, 77]
+    # ---- KV: the same bytes as 16-bit words with head_dim * e / 2
+    ckv = make_case(dict(m, D=scale(m["D"])), a, b, lens, weights=False, seed=e * 10 + a, src_order=so, dst_order=do)
+    s = Session(m, a, b, ckv.NB_src, ckv.NB_dst, len(lens), ckv.maxb, ckv.pairs_cap, weights=False, elem_bytes=e,
+                src_kv_order=so, dst_kv_order=do)
+    s.set_tables(ckv.seq_lens, ckv.src_bt, ckv.free_list, ckv.free_mask)
+    for t, p in zip(s.src_pools, ckv.src_pools):
+        assert t.numel() == p.nbytes
+        t.copy_(torch.from_numpy(p.view(np.uint8)))
+    s.step()
+    torch.cuda.synchronize()
+    check_case(ckv, s)
+    # ---- weights: row-split tensors as 16-bit rows of hidden * e / 2, column-split ones with head_dim and I scaled
+    rows_m = dict(m, hidden=scale(m["hidden"]))
+    cols_m = dict(m, D=scale(m["D"]), I=scale(m["I"]))
+    g = np.random.default_rng(e)
+    w = Session(m, a, b, 4, 4, 1, 1, 1, kv=False, elem_bytes=e)
+    expected = []
+    for l in range(m["L"]):
+        Wr = {n: g.integers(0, 65536, size=sh, dtype=np.uint16) for n, sh in O.logical_shapes(rows_m).items()}
+        Wc = {n: g.integers(0, 65536, size=sh, dtype=np.uint16) for n, sh in O.logical_shapes(cols_m).items()}
+        src_r, src_c = O.weights_shard(Wr, rows_m, a), O.weights_shard(Wc, cols_m, a)
+        exp_r, exp_c = O.weights_transform(src_r, rows_m, a, b), O.weights_transform(src_c, cols_m, a, b)
+        pick = lambda rs, cs: {"q": rs["q"], "gate": rs["gate"], "o": cs["o"], "down": cs["down"]}
+        for r in range(a):
+            for n, arr in pick(src_r[r], src_c[r]).items():
+                assert w.src_w[r][l][n].numel() == arr.nbytes, (n, w.src_w[r][l][n].numel(), arr.nbytes)
+                w.src_w[r][l][n].copy_(torch.from_numpy(arr.reshape(-1).view(np.uint8)))
+        expected.append([pick(exp_r[r], exp_c[r]) for r in range(b)])
+    w.reshard_weights()
+    torch.cuda.synchronize()
+    assert int(w.status.item()) == 0
+    for l in range(m["L"]):
+        for r in range(b):
+            for n, arr in expected[l][r].items():
+                got = w.dst_w[r][l][n].cpu().numpy().view(np.uint16)
+                assert np.array_equal(got, arr.reshape(-1)), (l, r, n)

@@ -94,7 +94,7 @@ def test_layout_validation():
         (A.make_layout(m, 2, 0), A.ERR_INVALID_ARG),                     # empty pool
         (A.make_layout(dict(m, D=12), 2, 8), A.ERR_INVALID_ARG),         # different model on the two sides
         (A.make_layout(m, 2, 8, block_tokens=8), A.ERR_INVALID_ARG),     # different block size
-        (A.make_layout(m, 2, 8, elem_bytes=3), A.ERR_UNSUPPORTED),
+        (A.make_layout(m, 2, 8, elem_bytes=3), A.ERR_UNSUPPORTED),                 # 1, 2 and 4 are the sizes taken
         (A.make_layout(m, 2, 8, kv_layer_stride_bytes=1024), A.ERR_INVALID_ARG),  # stride smaller than a layer
     ]:
         with pytest.raises(A.AmoebaError) as e:
