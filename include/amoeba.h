@@ -61,7 +61,8 @@ typedef enum {
     AMOEBA_ERR_CUDA = 6,           /* a CUDA runtime call failed (launch error, no device) */
     AMOEBA_ERR_TIMEOUT = 7,        /* a bounded on-device wait on the kernel's own bulk copy ran out */
     AMOEBA_ERR_TOO_LARGE = 8,      /* the problem needs more scratch than the library's built-in scratch array holds */
-    AMOEBA_ERR_NO_MEMORY = 9       /* a host allocation inside the library failed */
+    AMOEBA_ERR_NO_MEMORY = 9,      /* a host allocation inside the library failed */
+    AMOEBA_ERR_INTERNAL = 10       /* checked build only: a work item would have reached outside its buffer (skipped) */
 } amoeba_status;
 
 /* Storage order of one layer of a worker's KV pool (Sec. 3.1).  HEAD_MAJOR is the paper's header-centric layout

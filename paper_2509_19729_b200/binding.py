@@ -6,6 +6,7 @@ current stream.  Every function raises :class:`AmoebaError` when the C call retu
 from __future__ import annotations
 
 import ctypes as C
+import os
 from typing import Optional, Sequence
 
 from . import build as _build
@@ -21,12 +22,12 @@ __all__ = [
 ]
 
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_NO_FREE_BLOCKS, ERR_BAD_BLOCK_ID, ERR_CUDA, ERR_TIMEOUT,
- ERR_TOO_LARGE, ERR_NO_MEMORY) = range(10)
+ ERR_TOO_LARGE, ERR_NO_MEMORY, ERR_INTERNAL) = range(11)
 STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS", "BAD_BLOCK_ID", "CUDA", "TIMEOUT",
-                "TOO_LARGE", "NO_MEMORY"]
+                "TOO_LARGE", "NO_MEMORY", "INTERNAL"]
 BUILTIN_SCRATCH_BYTES = 1 << 20
 __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
-            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "ERR_NO_MEMORY", "BUILTIN_SCRATCH_BYTES", "OPT_WAIT_TRIES", "OPT_L2_PROMOTION",
+            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "ERR_NO_MEMORY", "ERR_INTERNAL", "BUILTIN_SCRATCH_BYTES", "OPT_WAIT_TRIES", "OPT_L2_PROMOTION",
             "amoeba_rewrite_block_tables_builtin_scratch", "amoeba_reshape_block_tables", "amoeba_reshape_kv_inplace",
             "amoeba_reshape_bytes"]
 (OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS,
@@ -80,20 +81,26 @@ class WeightDesc(C.Structure):
 _lib = None
 
 
+# AMOEBA_BINDING_BUILD=checked makes this binding load the checked build of the library (every work item tested against
+# the extent of its buffers, see build.py) instead of the normal one: a switch of the Python binding for test runs,
+# the C library itself reads no environment variable.
+_CHECKED = os.environ.get("AMOEBA_BINDING_BUILD", "") == "checked"
+
+
 def library_path():
-    return _build.LIB
+    return _build.LIB_CHECKED if _CHECKED else _build.LIB
 
 
 def _load():
     global _lib
     if _lib is not None:
         return _lib
-    if _build.needs_build():
+    if _build.needs_build(_CHECKED):
         try:
-            _build.build()
+            _build.build(checked=_CHECKED)
         except Exception as e:  # no silent fallback: the product is the CUDA library
-            raise ImportError(f"libamoeba.so is missing or stale and could not be built: {e}") from e
-    lib = C.CDLL(str(_build.LIB))
+            raise ImportError(f"{library_path().name} is missing or stale and could not be built: {e}") from e
+    lib = C.CDLL(str(library_path()))
     P, I32, I64, VP = C.POINTER, C.c_int32, C.c_int64, C.c_void_p
     sig = {
         "amoeba_plan_create": (I32, [P(Layout), P(Layout), P(VP)]),

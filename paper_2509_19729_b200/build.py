@@ -14,6 +14,8 @@ HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libamoeba.so"
+LIB_CHECKED = HERE / "libamoeba_checked.so"  # the same sources with -DAMOEBA_CHECK_ITEMS: every work item is tested
+#                                              against the extent of its buffers before it is moved
 SOURCES = ["plan.cpp", "block_tables.cu", "kv_reshard.cu", "weights_reshard.cu"]
 HEADERS = ["plan.hpp", "launch.hpp", "copy_engine.cuh", "kv_items.cuh", "w_items.cuh"]
 
@@ -30,26 +32,30 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def needs_build() -> bool:
-    if not LIB.exists():
+def needs_build(checked: bool = False) -> bool:
+    lib = LIB_CHECKED if checked else LIB
+    if not lib.exists():
         return True
-    t = LIB.stat().st_mtime
+    t = lib.stat().st_mtime
     deps = [CSRC / s for s in SOURCES + HEADERS] + [INCLUDE / "amoeba.h"]
     return any(d.stat().st_mtime > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    if not force and not needs_build():
-        return LIB
-    tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> Path:
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not needs_build(checked):
+        return lib
+    tmp = lib.with_suffix(f".tmp{os.getpid()}.so")
     cmd = [_nvcc(), *NVCC_FLAGS, f"-I{INCLUDE}", f"-I{CSRC}"]
+    if checked:
+        cmd += ["-DAMOEBA_CHECK_ITEMS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [str(CSRC / s) for s in SOURCES] + ["-o", str(tmp)]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

@@ -42,6 +42,17 @@ struct RingShape {
     int32_t max_polls;    // 0: default wait budget; v > 0: every mbarrier wait gives up after v - 1 non-blocking polls
 };
 
+// Checked build (-DAMOEBA_CHECK_ITEMS): every work item is tested against the extent of the buffers it addresses
+// before it is moved; an item that would reach outside sets AMOEBA_ERR_INTERNAL in the status word and is skipped.
+// True if n_rows rows of row_bytes, the first at byte `off` of a buffer and consecutive ones `pitch` apart, lie inside
+// [0, size).
+__device__ __forceinline__ bool rows_inside(int64_t off, int64_t pitch, int32_t n_rows, int32_t row_bytes, int64_t size) {
+    if (n_rows <= 0) return true;
+    const int64_t last = off + (int64_t)(n_rows - 1) * pitch;
+    const int64_t lo = pitch >= 0 ? off : last, hi = (pitch >= 0 ? last : off) + row_bytes;
+    return lo >= 0 && hi <= size;
+}
+
 // ------------------------------------------------------------------ vector load/store path
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;

@@ -28,6 +28,7 @@ struct KvParams {
     // destination worker r*N IS source worker r; -N, the other way round.  The header unit a worker retains
     // (every N-th) is not a work item at all: `moving_units` counts the others.
     int32_t reshape, moving_units;
+    int64_t src_span, dst_span;  // bytes of a source / destination pool the layers of this call reach into
 };
 
 // Tensor maps of the token-first pools, one per worker: dimensions {dim, token of the layer's K or V region,
@@ -108,6 +109,13 @@ struct KvItems {
         it.dst = p.dst[rb] + layer * p.dst_layer_stride +
                  pool_offset(p.dst_token_major, p.nb_dst, p.heads_dst, p.block_tokens, p.vec_bytes, ids.y, hb, c) +
                  r0 * p.dst_row_pitch + in_row;
+#ifdef AMOEBA_CHECK_ITEMS
+        if (!rows_inside(it.src - p.src[ra], it.src_pitch, it.n_rows, it.row_bytes, p.src_span) ||
+            !rows_inside(it.dst - p.dst[rb], it.dst_pitch, it.n_rows, it.row_bytes, p.dst_span)) {
+            atomicCAS(p.status, 0, (int)AMOEBA_ERR_INTERNAL);
+            it.n_rows = 0;
+        }
+#endif
         return it;
     }
 };
@@ -168,6 +176,13 @@ struct KvBoxItems {
                      pool_offset(false, p.nb_dst, p.heads_dst, p.block_tokens, p.vec_bytes, ids.y, hb, 0) +
                      t0 * p.vec_bytes;
         }
+#ifdef AMOEBA_CHECK_ITEMS  // the header-centric sides; a tensor map checks its own coordinates against its extents
+        if ((it.src && !rows_inside(it.src - p.src[ra], it.src_pitch, it.n_rows, it.row_bytes, p.src_span)) ||
+            (it.dst && !rows_inside(it.dst - p.dst[rb], it.dst_pitch, it.n_rows, it.row_bytes, p.dst_span))) {
+            atomicCAS(p.status, 0, (int)AMOEBA_ERR_INTERNAL);
+            it.n_rows = 0;
+        }
+#endif
         return it;
     }
 };
@@ -209,6 +224,8 @@ inline void kv_fill_geometry(const amoeba_plan* plan, KvParams& p) {
     p.nb_dst = plan->dst.num_blocks;
     p.heads_src = plan->heads_src;
     p.heads_dst = plan->heads_dst;
+    p.src_span = (int64_t)(p.layer_begin + p.n_layers) * plan->src_layer_stride;
+    p.dst_span = (int64_t)(p.layer_begin + p.n_layers) * plan->dst_layer_stride;
     p.moving_units = g.head_units;
     if (p.reshape) {  // one unit = the headers of one worker of the finer side; every N-th stays
         const int n = p.reshape > 0 ? p.reshape : -p.reshape;

@@ -92,6 +92,8 @@ struct MergeParams {
     int64_t layer_stride, block_bytes, seg_bytes, chunk_bytes;
     int32_t n_inst, a, nb, layer_begin, n_layers, chunks_per_seg, n_pairs;
     int32_t split;  // 0: merge (a live block sends its segments away), 1: the way back (a live block gathers them)
+    int32_t* status;
+    int64_t span;   // bytes of a pool the layers of this call reach into
 };
 
 struct MergeItems {
@@ -126,6 +128,13 @@ struct MergeItems {
         const int64_t base = layer * p.layer_stride + (int64_t)blk * p.block_bytes + (int64_t)chunk * p.chunk_bytes;
         char* A = p.pools[i * p.a + r] + base + k * p.seg_bytes;  // leaves instance i's worker for merged worker r*N+k
         char* B = p.pools[k * p.a + r] + base + i * p.seg_bytes;  // leaves instance k's worker for merged worker r*N+i
+#ifdef AMOEBA_CHECK_ITEMS
+        if (!rows_inside(A - p.pools[i * p.a + r], 0, 1, (int32_t)p.chunk_bytes, p.span) ||
+            !rows_inside(B - p.pools[k * p.a + r], 0, 1, (int32_t)p.chunk_bytes, p.span)) {
+            atomicCAS(p.status, 0, (int)AMOEBA_ERR_INTERNAL);
+            return it;
+        }
+#endif
         if (live_i && live_k) {
             it.n_rows = 2;
             it.src = A;
@@ -407,6 +416,8 @@ static amoeba_status merge_or_split_kv(bool split, const amoeba_plan* plan, void
     p.n_layers = layer_end - layer_begin;
     p.n_pairs = n * (n - 1) / 2;
     p.split = split ? 1 : 0;
+    p.status = d_status;
+    p.span = (int64_t)layer_end * p.layer_stride;
 
     const DeviceInfo dev = cached_device_info();
     if (dev.sms <= 0) return AMOEBA_ERR_CUDA;

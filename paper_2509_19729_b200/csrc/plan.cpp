@@ -566,6 +566,7 @@ const char* amoeba_status_string(amoeba_status s) {
         case AMOEBA_ERR_TIMEOUT: return "on-device wait for a bulk copy ran out";
         case AMOEBA_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch array";
         case AMOEBA_ERR_NO_MEMORY: return "host memory allocation failed";
+        case AMOEBA_ERR_INTERNAL: return "a work item outside its buffer was skipped (checked build)";
     }
     return "unknown status";
 }

@@ -14,6 +14,8 @@ struct WParams {
     WDescDev descs[kMaxWeightDescs];
     void* ptrs[kMaxWeightPtrs];  // [layer][src rank][tensor] then, from dst_base, [layer][dst rank][tensor]
     int32_t n_descs, items_per_layer, n_layers, src_tp, dst_tp, dst_base;
+    int32_t* status;                                         // where an item outside its buffer is reported (checked build)
+    int64_t src_bytes[kNumTensors], dst_bytes[kNumTensors];  // size of a worker's buffer of each kind (checked build)
 };
 
 struct WItems {
@@ -50,6 +52,13 @@ struct WItems {
         }
         it.src = s + d.src_off + r0 * d.src_pitch + off;
         it.dst = t + d.dst_off + r0 * d.dst_pitch + off;
+#ifdef AMOEBA_CHECK_ITEMS
+        if (!rows_inside(it.src - s, it.src_pitch, it.n_rows, it.row_bytes, p.src_bytes[d.src_slot % kNumTensors]) ||
+            !rows_inside(it.dst - t, it.dst_pitch, it.n_rows, it.row_bytes, p.dst_bytes[d.dst_slot % kNumTensors])) {
+            atomicCAS(p.status, 0, (int)AMOEBA_ERR_INTERNAL);
+            it.n_rows = 0;
+        }
+#endif
         return it;
     }
 };

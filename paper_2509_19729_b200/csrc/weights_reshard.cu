@@ -60,6 +60,12 @@ static amoeba_status launch_descs(const amoeba_plan* plan, const std::vector<WDe
     const int layers_per_launch = weight_layers_per_launch(a, b);
 
     WParams p;  // large: filled per launch
+    p.status = d_status;
+    const amoeba_layout& dst_layout = src == dst ? plan->src : plan->dst;  // in place: one set of buffers, one layout
+    for (int t = 0; t < kNumTensors; ++t) {
+        amoeba_layout_weight_bytes(&plan->src, t, &p.src_bytes[t]);
+        amoeba_layout_weight_bytes(&dst_layout, t, &p.dst_bytes[t]);
+    }
     for (int l0 = layer_begin; l0 < layer_end; l0 += layers_per_launch) {
         const int nl = std::min(layers_per_launch, layer_end - l0);
         w_fill_params(p, descs, items_per_layer, src, a, dst, b, L, l0, nl);
