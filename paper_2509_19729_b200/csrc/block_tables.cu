@@ -1,6 +1,6 @@
 // Destination block bookkeeping for the KV migration (Sec. 3.1: each worker prepares reserved pages for the KV it
 // receives), and the block tables of the in-place block reshaping of one instance (Sec. 3.1, Improvement 1).
-// No CTA ever waits on another.  Two phases:
+// No CTA ever waits on another.  Three phases:
 //   scan   (1 CTA)  blocks per sequence and their exclusive prefix sum; when the free blocks come as a byte mask,
 //                   their compaction into an ascending id list (16 mask bytes per thread, popc + CTA prefix sum);
 //                   the whole-call errors.
@@ -99,7 +99,7 @@ __device__ __forceinline__ uint32_t nonzero_bytes(uint32_t w) {
 // All kScanThreads threads of ONE CTA.
 __device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) {
     const int tid = threadIdx.x;
-    if (tid == 0) flags[0] = flags[1] = 0;  // [0] bad length, [1] whole-call error
+    if (tid == 0) flags[0] = 0;  // a negative or too long sequence was seen
     __syncthreads();
 
     // ---- blocks per sequence and their exclusive prefix sum
@@ -160,7 +160,6 @@ __device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) 
         *a.num_pairs = assigned;
         *a.free_count_out = (int32_t)n_free - assigned;
         if (err) atomicCAS(a.status, 0, err);
-        flags[1] = err;
     }
     __syncthreads();
 
@@ -233,7 +232,7 @@ __device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
 
 __global__ void __launch_bounds__(kScanThreads) bt_scan(const __grid_constant__ BtArgs a) {
     __shared__ int32_t warp_sums[33];
-    __shared__ int32_t flags[2];
+    __shared__ int32_t flags[1];
     scan_phase(a, warp_sums, flags);
 }
 
@@ -249,7 +248,7 @@ __global__ void __launch_bounds__(256) bt_assign(const __grid_constant__ BtArgs 
 // barrier that ends it.
 __global__ void __launch_bounds__(kScanThreads) bt_fused(const __grid_constant__ BtArgs a) {
     __shared__ int32_t warp_sums[33];
-    __shared__ int32_t flags[2];
+    __shared__ int32_t flags[1];
     scan_phase(a, warp_sums, flags);
     __threadfence_block();
     __syncthreads();
