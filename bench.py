@@ -1084,7 +1084,9 @@ def main():
                    "max_ctas": args.max_ctas or "all SMs", "options": args.opt, "copy_path": {0: "pair (default)", 1: "ldst", 2: "bulk", 3: "pair"}[args.copy_path],
                    "chunk_bytes": n_seq_layers[2]},
         "phases_ms": {"rewrite_block_tables": bt_ms, "reshard_kv": kv_ms, "reshard_weights": w_ms,
-                      "reshard_kv_min": min(phase[1]), "reshard_weights_min": min(phase[2])},
+                      "reshard_kv_min": min(phase[1]), "reshard_weights_min": min(phase[2]),
+                      "reshard_kv_median": statistics.median(phase[1]),
+                      "reshard_weights_median": statistics.median(phase[2])},
         "phases_gbs": {"reshard_kv": kv_gbs, "reshard_weights": w_gbs},
         "pct_of_nominal_8TBs": {"reshard_kv": 100 * kv_gbs / NOMINAL_HBM_GBS,
                                 "reshard_weights": 100 * w_gbs / NOMINAL_HBM_GBS if w_gbs else None},
