@@ -20,7 +20,31 @@ FULL = ["llama3_8b_1to4", "llama3_8b_2to8", "llama2_7b_1to2", "llama2_13b_4to1",
 
 
 HEADLINE = "llama3_8b_1to4"  # compared completely: every layer of every destination buffer
-GROUP_BYTES = 12 << 30       # source KV bytes streamed through host memory per oracle call
+GROUP_BYTES = 12 << 30       # source KV bytes streamed through host memory per oracle call (less on a small host)
+
+
+def _host_available() -> int:
+    """Bytes of host memory that can still be taken (MemAvailable), or a large number if it cannot be read."""
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 1 << 40
+
+
+def _group_bytes() -> int:
+    # an oracle call holds the sources, the expected destinations and its own logical copy: about 3.5 x the sources
+    return max(1 << 30, min(GROUP_BYTES, _host_available() // 8))
+
+
+def _whole_layers(g, L, bytes_per_layer):
+    """First, last and one random layer - or fewer when three layers (held twice) do not fit the host comfortably."""
+    layers = sorted({0, L - 1, int(g.integers(L))})
+    while len(layers) > 1 and 4 * len(layers) * bytes_per_layer > _host_available() // 2:
+        layers.pop()
+    return layers
 
 CASES = [(n, "head") for n in FULL] + [("llama3_8b_1to4", "token"), ("llama3_70b_slice_8to2", "token2head"),
                                        ("llama2_7b_1to2", "head2token")]
@@ -90,7 +114,7 @@ def test_full_size_config(name, kv_order, oracle):
         everything = name == HEADLINE and kv_order == "head"
         layers = list(range(Lkv)) if everything else sorted({0, Lkv - 1, int(g.integers(Lkv))})
         src_layer_bytes = sum(p.numel() for p in s.src_pools) // Lkv
-        per_call = max(1, min(os.cpu_count() or 1, 16, GROUP_BYTES // src_layer_bytes))
+        per_call = max(1, min(os.cpu_count() or 1, 16, _group_bytes() // src_layer_bytes))
         groups = [[layers[0]]]
         for l in layers[1:]:
             if l == groups[-1][-1] + 1 and len(groups[-1]) < per_call:
@@ -164,7 +188,7 @@ def test_full_size_inplace_merge(oracle):
         old_v = [p.view(L, NB, -1) for p in s.pools]            # [layer][old block][bytes]
         samples = [(int(g.integers(L)), int(g.integers(NB))) for _ in range(64)]
         before = {(l, p): [v[l, p].cpu().numpy().view(np.uint16).copy() for v in old_v] for l, p in samples}
-        whole_layers = sorted({0, L - 1, int(g.integers(L))})
+        whole_layers = _whole_layers(g, L, sum(p.numel() for p in s.pools) // L)
         layer_before = {l: [v[l].cpu().numpy().view(np.uint16).reshape(-1).copy() for v in old_v] for l in whole_layers}
 
         s.status.zero_()
@@ -214,7 +238,7 @@ def test_full_size_inplace_reshape(name, oracle):
         N, a, NB, L = s.N, s.a, s.NB, s.kv_layers
         src_bt = s.src_bt.cpu().numpy()
         g = np.random.default_rng(13)
-        whole_layers = sorted({0, L - 1, int(g.integers(L))})
+        whole_layers = _whole_layers(g, L, sum(p.numel() for p in s.pools) // L)
         views = [p.view(L, -1) for p in s.pools]
         before = {l: [v[l].cpu().numpy().view(np.uint16).copy() for v in views] for l in whole_layers}
         s.status.zero_()
