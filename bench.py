@@ -240,19 +240,24 @@ def run_reference(args, rank, world):
 def cpu_baseline(cfg_name: str) -> dict:
     """The oracle as it stands on the host cores, on bounded samples of the workload: once on one thread, once with
     one thread per layer over all cores.  The top-level value is the all-cores one; `cores` = threads it used."""
-    run, nbytes, desc = oracle_sample(cfg_name)
+    cfg = wl.CONFIGS[cfg_name]
+    m = cfg["model"]
+    st = wl.draw_kv_state(cfg, name=cfg_name)
+    layer_bytes = st["n_live"] * m["Hkv"] * 2 * wl.BLOCK_TOKENS * m["D"] * 2  # live KV of one layer
+    # a sample of k layers holds about 4 k copies of that on the host (sources, destinations, logical state twice)
+    k1 = int(max(1, min(4, host_free_bytes() // 2 // (4 * layer_bytes)))) if host_free_bytes() else 4
+    run, nbytes, desc = oracle_sample(cfg_name, kv_layers=k1, w_layers=k1)
     t0 = time.perf_counter()
     run()
     dt1 = time.perf_counter() - t0
     one = {"value": nbytes / dt1 / 1e9, "unit": "GB/s", "cores": 1, "sample": desc, "seconds": dt1}
     del run
     cores = os.cpu_count() or 1
-    cfg = wl.CONFIGS[cfg_name]
     L_kv = cfg.get("kv_layers") or cfg["model"]["L"]
     threads = max(1, min(cores, L_kv))
     w_threads = max(1, min(threads, 8))  # weight layers in the sample (each is hundreds of MB of host memory)
     # about the same number of bytes as the one-thread sample, spread over `threads` layers: fewer sequences per layer
-    n_seqs = max(1, cfg["S"] * 4 // threads)
+    n_seqs = max(1, cfg["S"] * k1 // threads)
     runN, nbytesN, descN = oracle_sample(cfg_name, kv_layers=threads, n_seqs=n_seqs, w_layers=w_threads,
                                          threads=threads, dist="counter")
     t0 = time.perf_counter()
