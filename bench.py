@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 # disjoint memory).  It is a stored counter reading, not something this script measures: the line says so in
 # "traffic_source", and it is only quoted for that workload with default kernel options (None = no reading for the
 # current kernel).
-NCU_KV_TRAFFIC_RATIO = 0.9895
+NCU_KV_TRAFFIC_RATIO = 0.9893
 NCU_KV_TRAFFIC_CONFIG = "llama3_8b_1to4"
 NCU_KV_TRAFFIC_SOURCE = "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 1-layer slice, scaled by units processed"
 

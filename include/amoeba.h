@@ -190,6 +190,11 @@ enum {
                                    copies time out, every time. */
     AMOEBA_OPT_L2_PROMOTION = 10, /* tensor-map copies of token-first pools: L2 promotion of the maps, 1 = none, 2 = 64 B,
                                    3 = 128 B, 4 = 256 B */
+    AMOEBA_OPT_PAIR_ORDER = 11, /* order of the pair list the table calls write: 1 = table order (entry k = the k-th
+                                   block), 2 = ascending by destination id (the out-of-place KV copy then writes every
+                                   destination pool front to back, which DRAM rewards with 1 - 2 %; the in-place reshape
+                                   measured 2 % slower with it), 0 = default: 2 for amoeba_rewrite_block_tables, 1 for
+                                   amoeba_reshape_block_tables */
     AMOEBA_OPT_WEIGHTS_ONLY = 16,
     AMOEBA_OPT_KV_ONLY = 32
 };
@@ -208,7 +213,11 @@ AMOEBA_API amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t optio
  * in  d_src_bt   int32 [num_seqs][max_blocks_per_seq], entries past a sequence's blocks are -1
  *     d_seq_lens int32 [num_seqs]
  * out d_dst_bt   int32 [num_seqs][max_blocks_per_seq], fully written, -1 past each sequence's blocks
- *     d_pairs    int32 [pairs_cap][2]: entry k = (source block, destination block) of the k-th block
+ *     d_pairs    int32 [pairs_cap][2]: one (source block, destination block) entry per block, a work list for
+ *                amoeba_reshard_kv.  By default the entries are ascending by destination id, and the entries of
+ *                blocks that were given no destination id - (-1,-1) - close the list; with AMOEBA_OPT_PAIR_ORDER = 1
+ *                entry k belongs to the k-th block in (sequence, block) order.  A block with a destination but a
+ *                bad source id has (-1,-1) in its place in either order.
  *     d_num_pairs, d_dst_free_count_out  int32 scalars: number of pairs, free blocks left
  *     d_status   int32 scalar, sticky (see conventions)
  * d_workspace: scratch of at least amoeba_rewrite_workspace_bytes(...) bytes, 16-byte aligned, contents irrelevant
@@ -244,8 +253,8 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables(const amoeba_plan* plan, co
  * performs no cudaMalloc / cudaFree and calls no allocating routine of any library.
  *
  * Limit: the scratch array is AMOEBA_BUILTIN_SCRATCH_BYTES (1 MiB) per GPU, held by every GPU that loads the library
- * until the process exits.  It must cover amoeba_rewrite_workspace_bytes(...), i.e. roughly num_seqs + the larger of
- * the plan's two block counts <= 262 000 entries, in either free-block form; larger problems are refused with
+ * until the process exits.  It must cover amoeba_rewrite_workspace_bytes(...), i.e. roughly num_seqs + twice the larger
+ * of the plan's two block counts <= 262 000 entries, in either free-block form; larger problems are refused with
  * AMOEBA_ERR_TOO_LARGE and nothing is launched - use amoeba_rewrite_block_tables with your own workspace for those.
  *
  * First use on a device: the first call made while a given device is current looks up that device's address of the
@@ -301,7 +310,8 @@ AMOEBA_API amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* 
  * amoeba_reshard_kv inside the TP = N*a pools, using free ids q = 0 mod N whose followers q+1 .. q+N-1 are free too).
  *
  * amoeba_reshape_block_tables: same inputs as amoeba_rewrite_block_tables without a free list.  Writes d_dst_bt
- * (p -> p*N, or q -> q/N; -1 past each sequence's blocks), the pair list (old id, new id) in (sequence, block) order,
+ * (p -> p*N, or q -> q/N; -1 past each sequence's blocks), the pair list (old id, new id) - entry k = the k-th block in
+ * (sequence, block) order unless AMOEBA_OPT_PAIR_ORDER = 2 asks for destination order as described above -,
  * d_dst_free_mask_out: uint8 [destination num_blocks], 1 = free afterwards, and the free count.  Workspace as for
  * amoeba_rewrite_block_tables.  Device-detected errors: whole call as there (no NO_FREE_BLOCKS); per block ->
  * BAD_BLOCK_ID, table entry -1, pair (-1,-1), block not moved: an id outside the source pool, -1 inside a sequence,

@@ -27,11 +27,12 @@ STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "ALIGNMENT", "NO_FREE_BLOCKS
                 "TOO_LARGE", "NO_MEMORY", "INTERNAL"]
 BUILTIN_SCRATCH_BYTES = 1 << 20
 __all__ += ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_ALIGNMENT", "ERR_NO_FREE_BLOCKS", "ERR_BAD_BLOCK_ID",
-            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "ERR_NO_MEMORY", "ERR_INTERNAL", "BUILTIN_SCRATCH_BYTES", "OPT_WAIT_TRIES", "OPT_L2_PROMOTION",
+            "ERR_CUDA", "ERR_TIMEOUT", "ERR_TOO_LARGE", "ERR_NO_MEMORY", "ERR_INTERNAL", "BUILTIN_SCRATCH_BYTES", "OPT_WAIT_TRIES", "OPT_L2_PROMOTION", "OPT_PAIR_ORDER", "PAIR_ORDER_TABLE", "PAIR_ORDER_DESTINATION",
             "amoeba_rewrite_block_tables_builtin_scratch", "amoeba_reshape_block_tables", "amoeba_reshape_kv_inplace",
             "amoeba_reshape_bytes"]
 (OPT_COPY_PATH, OPT_CTAS_PER_SM, OPT_CHUNK_BYTES, OPT_STAGES, OPT_LAG, OPT_WARPS, OPT_L2_HINT, OPT_TENSOR_MAPS,
- OPT_MAX_CTAS, OPT_WAIT_TRIES, OPT_L2_PROMOTION) = range(11)
+ OPT_MAX_CTAS, OPT_WAIT_TRIES, OPT_L2_PROMOTION, OPT_PAIR_ORDER) = range(12)
+PAIR_ORDER_TABLE, PAIR_ORDER_DESTINATION = 1, 2
 OPT_WEIGHTS_ONLY, OPT_KV_ONLY = 16, 32  # add to an option id to set one kernel only
 COPY_PATH_LDST, COPY_PATH_BULK, COPY_PATH_PAIR = 1, 2, 3
 KV_HEAD_MAJOR, KV_TOKEN_MAJOR = 0, 1  # [block][header][K/V][token][dim] / [K/V][block][token][header][dim]

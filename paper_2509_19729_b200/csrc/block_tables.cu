@@ -1,11 +1,13 @@
 // Destination block bookkeeping for the KV migration (Sec. 3.1: each worker prepares reserved pages for the KV it
 // receives), and the block tables of the in-place block reshaping of one instance (Sec. 3.1, Improvement 1).
-// No CTA ever waits on another.  Three phases:
+// No CTA ever waits on another.  Phases:
 //   scan   (1 CTA)  blocks per sequence and their exclusive prefix sum; when the free blocks come as a byte mask,
 //                   their compaction into an ascending id list (16 mask bytes per thread, popc + CTA prefix sum);
 //                   the whole-call errors.
 //   claim  (grid)   only when destination ids can repeat (a free LIST, or ids derived from the source table): the
 //                   first user of every destination id in (sequence, block) order, by atomicMin.
+//   rank   (1 CTA)  only for the pair list in destination order: the number of given destination ids below every id
+//                   (prefix sum over the ids), i.e. where the pair of the block that was given the id goes.
 //   assign (grid)   one warp per 128-entry segment of a block-table row: the k-th block overall takes the k-th free
 //                   id (or the reshaped id of its source block); writes the destination table (with -1 padding) and
 //                   the (source, destination) pair list; an id whose first user is another block is refused.
@@ -25,7 +27,8 @@ struct BtHeader {  // first 64 bytes of the workspace
     int32_t total;   // blocks assigned by this call (0 on a whole-call error)
     int32_t n_free;  // free destination blocks before the call
     int32_t err;     // whole-call error code or 0
-    int32_t pad[13];
+    int32_t n_given; // destination order: blocks that were given a destination id (the others' pairs go to the tail)
+    int32_t pad[12];
 };
 
 struct BtArgs {
@@ -36,6 +39,7 @@ struct BtArgs {
     BtHeader* hdr;
     int32_t* seq_off;     // [num_seqs] exclusive prefix sum of the blocks per sequence
     int32_t* area;        // mask form: compacted ascending free ids; otherwise: first user of every destination id
+    int32_t* rank;        // destination order (not mask form): number of given destination ids below every id
     int32_t* dst_bt;
     int2* pairs;
     int32_t* num_pairs;
@@ -44,6 +48,7 @@ struct BtArgs {
     uint8_t* free_mask_out;  // reshaping only: 1 = free id of the destination side
     int32_t num_seqs, block_tokens, maxb, n_free_or_nb, pairs_cap, nb_src, nb_dst;
     int32_t reshape;  // 0: ids from the free list / mask; +N: destination id = source id * N; -N: source id / N
+    int32_t dst_order;  // 1: pair list ascending by destination id (a mask hands ids out in that order anyway)
 };
 
 constexpr int kScanThreads = 1024;
@@ -157,6 +162,7 @@ __device__ void scan_phase(const BtArgs& a, int32_t* warp_sums, int32_t* flags) 
         a.hdr->total = assigned;
         a.hdr->n_free = (int32_t)n_free;
         a.hdr->err = err;
+        a.hdr->n_given = 0;
         *a.num_pairs = assigned;
         *a.free_count_out = (int32_t)n_free - assigned;
         if (err) atomicCAS(a.status, 0, err);
@@ -190,13 +196,51 @@ __device__ void claim_phase(const BtArgs& a, int64_t t, int64_t n) {
     }
 }
 
-// Any number of warps; warp `warp` of `n_warps`.  Runs after claim_phase has completed (next launch, or after a
-// __syncthreads() of the one CTA that ran it).
+// Pair list in destination order: rank[d] = number of destination ids below d that some block was given.  All
+// kScanThreads threads of ONE CTA; runs after claim_phase has completed.  Each warp owns one contiguous run of ids
+// (a whole number of 32-id rows): it counts the given ids of its run, the CTA scans the 32 counts, and the warp
+// walks its run again (the flags are in L1/L2 by then) handing out ranks row by row.
+__device__ void rank_phase(const BtArgs& a, int32_t* warp_sums) {
+    if (!a.dst_order || a.free_mask) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kWarps = kScanThreads / 32;
+    const bool ok = a.hdr->err == 0;
+    const int32_t rows = ok ? ((a.nb_dst + 31) / 32 + kWarps - 1) / kWarps : 0;  // 32-id rows per warp
+    const int64_t first = (int64_t)warp * rows * 32;
+    int32_t mine = 0;
+#pragma unroll 8
+    for (int32_t j = 0; j < rows; ++j) {
+        const int64_t d = first + (int64_t)j * 32 + lane;
+        mine += (d < a.nb_dst && a.area[d] != INT32_MAX) ? 1 : 0;
+    }
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    __syncthreads();  // warp_sums may still be read by the phase before
+    if (lane == 0) warp_sums[warp] = mine;
+    __syncthreads();
+    int32_t before = 0, given = 0;
+    for (int w = 0; w < kWarps; ++w) {
+        const int32_t c = warp_sums[w];
+        before += w < warp ? c : 0;
+        given += c;
+    }
+    for (int32_t j = 0; j < rows; ++j) {
+        const int64_t d = first + (int64_t)j * 32 + lane;
+        const bool flag = d < a.nb_dst && a.area[d] != INT32_MAX;
+        const unsigned row = __ballot_sync(0xffffffffu, flag);
+        if (d < a.nb_dst) a.rank[d] = before + __popc(row & ((1u << lane) - 1u));
+        before += __popc(row);
+    }
+    if (threadIdx.x == 0) a.hdr->n_given = given;
+}
+
+// Any number of warps; warp `warp` of `n_warps`.  Runs after claim_phase (and rank_phase) has completed (next launch,
+// or after a __syncthreads() of the one CTA that ran it).
 __device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
     const int lane = threadIdx.x & 31;
     const int32_t segs_per_row = (a.maxb + kSegment - 1) / kSegment;
     const bool call_failed = a.hdr->err != 0;
     const bool check_first = a.free_mask == nullptr;
+    const bool by_rank = a.dst_order && check_first;  // where the pairs go: by destination id, refused blocks last
     bool bad = false;
     int32_t refused = 0;  // reshaping: blocks that keep no destination id
     for (int64_t unit = warp; unit < (int64_t)a.num_seqs * segs_per_row; unit += n_warps) {
@@ -214,7 +258,9 @@ __device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
                 if (dst_ok && check_first && a.area[dst] != k) dst_ok = false;  // an earlier block holds this id
                 const bool src_ok = src >= 0 && src < a.nb_src;
                 out = dst_ok ? dst : -1;
-                a.pairs[k] = (dst_ok && src_ok) ? make_int2(src, dst) : make_int2(-1, -1);
+                const int2 pair = (dst_ok && src_ok) ? make_int2(src, dst) : make_int2(-1, -1);
+                if (!by_rank) a.pairs[k] = pair;
+                else if (dst_ok) a.pairs[a.rank[dst]] = pair;
                 bad |= !(dst_ok && src_ok);
                 refused += !dst_ok;
             }
@@ -222,6 +268,9 @@ __device__ void assign_phase(const BtArgs& a, int64_t warp, int64_t n_warps) {
         }
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(a.status, 0, (int)AMOEBA_ERR_BAD_BLOCK_ID);
+    if (by_rank)  // the blocks that were given no destination id: their (-1,-1) pairs close the list
+        for (int64_t k = a.hdr->n_given + warp * 32 + lane; k < a.hdr->total; k += n_warps * 32)
+            a.pairs[k] = make_int2(-1, -1);
     if (a.reshape) {
         refused = __reduce_add_sync(0xffffffffu, refused);
         if (refused && lane == 0) atomicAdd(a.free_count_out, refused);
@@ -240,6 +289,11 @@ __global__ void __launch_bounds__(256) bt_claim(const __grid_constant__ BtArgs a
     claim_phase(a, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
 }
 
+__global__ void __launch_bounds__(kScanThreads) bt_rank(const __grid_constant__ BtArgs a) {
+    __shared__ int32_t warp_sums[33];
+    rank_phase(a, warp_sums);
+}
+
 __global__ void __launch_bounds__(256) bt_assign(const __grid_constant__ BtArgs a) {
     assign_phase(a, ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, ((int64_t)gridDim.x * blockDim.x) >> 5);
 }
@@ -255,6 +309,9 @@ __global__ void __launch_bounds__(kScanThreads) bt_fused(const __grid_constant__
     claim_phase(a, threadIdx.x, kScanThreads);
     __threadfence_block();
     __syncthreads();
+    rank_phase(a, warp_sums);
+    __threadfence_block();
+    __syncthreads();
     assign_phase(a, threadIdx.x >> 5, kScanThreads / 32);
 }
 
@@ -262,9 +319,12 @@ constexpr int64_t kFusedEntries = 8 * 1024;  // up to this many table entries (a
 
 static int64_t align16(int64_t x) { return (x + 15) & ~int64_t(15); }
 
+static int64_t ids_bytes(const amoeba_plan* plan) {
+    return align16(4 * (int64_t)std::max(plan->src.num_blocks, plan->dst.num_blocks));
+}
+
 static int64_t tables_workspace_bytes(const amoeba_plan* plan, int32_t num_seqs) {
-    return (int64_t)sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)) +
-           align16(4 * (int64_t)std::max(plan->src.num_blocks, plan->dst.num_blocks));
+    return (int64_t)sizeof(BtHeader) + align16(4 * ((int64_t)num_seqs + 1)) + 2 * ids_bytes(plan);
 }
 
 static amoeba_status launch_tables(const amoeba_plan* plan, BtArgs a, void* d_workspace, cudaStream_t stream) {
@@ -272,6 +332,9 @@ static amoeba_status launch_tables(const amoeba_plan* plan, BtArgs a, void* d_wo
     a.hdr = reinterpret_cast<BtHeader*>(ws);
     a.seq_off = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader));
     a.area = reinterpret_cast<int32_t*>(ws + sizeof(BtHeader) + align16(4 * ((int64_t)a.num_seqs + 1)));
+    a.rank = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(a.area) + ids_bytes(plan));
+    // 0 = default: destination order, but table order when reshaping in place (measured faster there)
+    a.dst_order = plan->opt.pair_order == 2 || (plan->opt.pair_order == 0 && !a.reshape);
     a.block_tokens = plan->src.block_tokens;
     a.nb_src = plan->src.num_blocks;
     a.nb_dst = plan->dst.num_blocks;
@@ -294,6 +357,11 @@ static amoeba_status launch_tables(const amoeba_plan* plan, BtArgs a, void* d_wo
         bt_claim<<<grid, 256, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
         count_launch();
+        if (a.dst_order) {
+            bt_rank<<<1, kScanThreads, 0, stream>>>(a);
+            if (cudaGetLastError() != cudaSuccess) return AMOEBA_ERR_CUDA;
+            count_launch();
+        }
     }
     const int64_t units = std::max<int64_t>((int64_t)a.num_seqs * ((a.maxb + kSegment - 1) / kSegment),
                                             a.reshape ? (a.nb_dst + 31) / 32 : 0);

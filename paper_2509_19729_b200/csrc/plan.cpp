@@ -438,6 +438,11 @@ amoeba_status amoeba_plan_set_option(amoeba_plan* plan, int32_t option, int64_t 
     const int which = option / AMOEBA_OPT_WEIGHTS_ONLY;  // 0 both kernels, 1 weights only, 2 KV only
     const int id = option % AMOEBA_OPT_WEIGHTS_ONLY;
     if (which > 2) return AMOEBA_ERR_INVALID_ARG;
+    if (option == AMOEBA_OPT_PAIR_ORDER) {  // a property of the table calls, not of a copy kernel
+        if (value > 2) return AMOEBA_ERR_INVALID_ARG;
+        plan->opt.pair_order = (int)value;
+        return AMOEBA_OK;
+    }
     KernelOpts* targets[2] = {which != 1 ? &plan->opt.kv : nullptr, which != 2 ? &plan->opt.w : nullptr};
     for (KernelOpts* k : targets) {
         if (!k) continue;

@@ -60,6 +60,7 @@ struct KernelOpts {
 
 struct Options {
     KernelOpts kv, w;
+    int pair_order = 0;  // pair list of the table calls: 0 / 2 ascending by destination id, 1 in table order
 };
 
 // How the KV copy of one (block pair, layer) is cut into 2-D work items.  A "unit" is the largest piece that is a

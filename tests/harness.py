@@ -14,6 +14,21 @@ class Case:
     pass
 
 
+def pairs_in_destination_order(pairs, dst_bt, seq_lens, T):
+    """The oracle's pair list (entry k = k-th block in (sequence, block) order) in the order the library writes it by
+    default: ascending by the destination id each block was given, the pairs of blocks that were given none - they are
+    (-1,-1) - at the end.  `dst_bt` is the oracle's destination table (-1 where a block got no id)."""
+    pairs = np.asarray(pairs, np.int32).reshape(-1, 2)
+    if len(pairs) == 0:
+        return pairs
+    nblk = (np.maximum(np.asarray(seq_lens, np.int64), 0) + T - 1) // T
+    given = np.concatenate([np.asarray(dst_bt)[s, :n] for s, n in enumerate(nblk)])
+    assert len(given) == len(pairs)
+    has = given >= 0
+    order = np.flatnonzero(has)[np.argsort(given[has], kind="stable")]
+    return np.concatenate([pairs[order], np.full((int((~has).sum()), 2), -1, np.int32)])
+
+
 def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_slack=0.25, dst_occupied=0.3, seed=0,
               fused_qkv=True, fused_gate_up=True, weights=True, kv=True, dtype="bf16", free_override=None,
               src_bt_override=None, pairs_cap=None, src_order=0, dst_order=0, src_pad=None, dst_pad=None):
@@ -116,7 +131,8 @@ def check_case(c, s):
     assert int(s.num_pairs.item()) == c.exp_n
     assert int(s.free_count.item()) == c.exp_left
     assert np.array_equal(s.dst_bt.cpu().numpy(), c.exp_dst_bt)
-    assert np.array_equal(s.pairs.cpu().numpy()[:c.exp_n], c.exp_pairs)
+    assert np.array_equal(s.pairs.cpu().numpy()[:c.exp_n],
+                          pairs_in_destination_order(c.exp_pairs, c.exp_dst_bt, c.seq_lens, c.T))
     assert np.all(s.pairs.cpu().numpy()[c.exp_n:] == -3)  # pair slots past N untouched
     if c.kv:
         for r, (t, e) in enumerate(zip(s.dst_pools, c.exp_dst_pools)):

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 import workloads as wl
-from harness import check_case, make_case, run_case
+from harness import check_case, make_case, pairs_in_destination_order, run_case
 
 pytestmark = pytest.mark.gpu
 
@@ -651,6 +651,37 @@ def test_weights_compaction_host_errors():
         == A.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("form", ["list", "mask"])
+def test_pair_list_order_option(form):
+    """The pair list comes ascending by destination id (the default; the tail holds the (-1,-1) pairs of blocks that
+    were given no id) or, with the option set, in (sequence, block) order.  Tables, counts, status and the copied
+    pools are the same either way."""
+    import paper_2509_19729_b200 as A
+
+    lens = [160, 48, 0, 300, 7]
+    base = make_case(GQA, 2, 4, lens, weights=False, seed=8, dst_form=form)
+    if form == "list":
+        free = base.free_list.copy()
+        free[5] = free[1]          # one block is refused: its pair goes to the tail in destination order
+        c = make_case(GQA, 2, 4, lens, weights=False, seed=8, free_override=(free, None))
+        assert c.exp_status == 5
+    else:
+        c = base
+    for order in (A.PAIR_ORDER_DESTINATION, A.PAIR_ORDER_TABLE):
+        s = run_case(c, PAIR, options=[(A.OPT_PAIR_ORDER, order)])
+        got = s.pairs.cpu().numpy()[:c.exp_n]
+        if order == A.PAIR_ORDER_TABLE:
+            assert np.array_equal(got, c.exp_pairs)
+        else:
+            live = got[got[:, 1] >= 0, 1]
+            assert np.all(np.diff(live) > 0) and np.all(got[len(live):] == -1)
+            assert sorted(map(tuple, got)) == sorted(map(tuple, c.exp_pairs))
+        assert int(s.num_pairs.item()) == c.exp_n and int(s.status.item()) == c.exp_status
+        assert np.array_equal(s.dst_bt.cpu().numpy(), c.exp_dst_bt)
+        for t, e in zip(s.dst_pools, c.exp_dst_pools):
+            assert np.array_equal(t.cpu().numpy().view(np.uint16), e)
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_free_list_that_names_an_id_twice(path):
     """Two blocks must never share a destination: the first block (in sequence, block order) given an id keeps it,
@@ -752,6 +783,8 @@ def test_random_tables_with_damaged_inputs(seed):
         lens[1] = -5
     m = dict(L=1, hidden=128, Hq=8, Hkv=8, D=64, I=256)
     plan = A.amoeba_plan_create(A.make_layout(m, 2, NB_src, T), A.make_layout(m, 4, NB_dst, T))
+    if seed % 2 == 0 and seed % 3 != 0:
+        A.amoeba_plan_set_option(plan, A.OPT_PAIR_ORDER, A.PAIR_ORDER_TABLE)
     e_bt, e_pairs, e_n, e_left, e_st = O.assign_blocks(lens, T, bt, NB_src, NB_dst, free_list=free_list,
                                                        free_mask=free_mask, pairs_cap=pairs_cap)
     dev = torch.device("cuda:0")
@@ -772,7 +805,9 @@ def test_random_tables_with_damaged_inputs(seed):
     assert int(d_status.item()) == e_st
     assert int(d_n.item()) == e_n and int(d_left.item()) == e_left
     assert np.array_equal(d_new.cpu().numpy(), e_bt)
-    assert np.array_equal(d_pairs.cpu().numpy()[:e_n], e_pairs)
+    table_order = seed % 2 == 0 and seed % 3 != 0   # both pair orders get their share of the seeds
+    assert np.array_equal(d_pairs.cpu().numpy()[:e_n],
+                          e_pairs if table_order else pairs_in_destination_order(e_pairs, e_bt, lens, T))
 
 
 @pytest.mark.parametrize("so,do", [(HC, HC), (TF, HC), (HC, TF)])

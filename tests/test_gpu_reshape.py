@@ -4,6 +4,8 @@ the pair list, the free mask and count, the status word - split (TP a -> N*a) an
 import numpy as np
 import pytest
 
+from harness import pairs_in_destination_order
+
 pytestmark = pytest.mark.gpu
 
 MHA8 = dict(L=2, hidden=64, Hq=8, Hkv=8, D=16, I=64)
@@ -263,6 +265,9 @@ def test_random_reshapes_with_layer_strides(oracle, seed):
     plan = A.amoeba_plan_create(*((coarse, fine) if direction == "split" else (fine, coarse)))
     A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, int(g.choice([1, 2, 3])))
     A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, int(g.choice([64, 512, 8192])))
+    by_destination = seed % 2 == 1  # half the seeds ask for the pair list in destination order
+    if by_destination:
+        A.amoeba_plan_set_option(plan, A.OPT_PAIR_ORDER, A.PAIR_ORDER_DESTINATION)
     dev = torch.device("cuda:0")
     i32 = dict(dtype=torch.int32, device=dev)
     d_pools = [torch.from_numpy(p.view(np.uint8).copy()).to(dev) for p in pools]
@@ -279,6 +284,8 @@ def test_random_reshapes_with_layer_strides(oracle, seed):
     torch.cuda.synchronize()
     assert int(d_status.item()) == e_status == 0
     assert np.array_equal(d_new.cpu().numpy(), e_bt) and int(d_n.item()) == e_n and int(d_left.item()) == e_left
-    assert np.array_equal(d_pairs.cpu().numpy()[:e_n], e_pairs) and np.array_equal(d_mask.cpu().numpy(), e_mask)
+    assert np.array_equal(d_pairs.cpu().numpy()[:e_n],
+                          pairs_in_destination_order(e_pairs, e_bt, lens, T) if by_destination else e_pairs)
+    assert np.array_equal(d_mask.cpu().numpy(), e_mask)
     for w, (t, e) in enumerate(zip(d_pools, exp)):
         assert np.array_equal(t.cpu().numpy().view(np.uint16), e), (w, direction, N, a, T)

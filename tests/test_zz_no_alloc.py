@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 
 import workloads as wl
+from harness import pairs_in_destination_order
 
 pytestmark = pytest.mark.gpu
 
@@ -90,7 +91,8 @@ def test_builtin_scratch_matches_workspace_entry_point_twice_in_a_row(oracle):
         e_bt, e_pairs, e_n, e_left, e_status = _oracle_outputs(oracle, s)
         assert e_status == 0 and int(o[4][0]) == 0
         assert np.array_equal(o[0], e_bt) and int(o[2][0]) == e_n and int(o[3][0]) == e_left
-        assert np.array_equal(o[1][:e_n], e_pairs) and np.all(o[1][e_n:] == -3)
+        assert np.array_equal(o[1][:e_n], pairs_in_destination_order(e_pairs, e_bt, s.state["seq_lens"], 16))
+        assert np.all(o[1][e_n:] == -3)
     # and once more in the opposite order
     for (s, _), e in reversed(list(zip(cases, expected))):
         _reset(s)
