@@ -461,6 +461,66 @@ def test_random_shapes_orders_and_options():
                                  f"lens {lens}: {e}") from e
 
 
+@pytest.mark.parametrize("seed", range(64))
+def test_random_cases_with_ring_shapes_and_injected_errors(seed):
+    """One seeded random case per seed: model shape, TP pair, block size, lengths up to hundreds of blocks, free list or
+    mask, storage orders, weights, copy path, item size, ring shape, grid cap - and in a third of the cases one damaged
+    input (an id twice or out of range in the free list, a bad source id, a pair list or a free list that is too short,
+    a negative length).  Everything is compared with the oracle, the untouched bytes included."""
+    import paper_2509_19729_b200 as A
+
+    g = np.random.default_rng(77000 + seed)
+    Hkv = int(g.choice([1, 2, 4, 6, 8, 12, 20, 40]))
+    tps = [d for d in range(1, 33) if Hkv % d == 0]
+    a, b = int(g.choice(tps)), int(g.choice(tps))
+    m = dict(L=int(g.integers(1, 4)), hidden=64 * int(g.integers(1, 9)), Hq=Hkv * int(g.choice([1, 2, 4])), Hkv=Hkv,
+             D=int(g.choice([16, 32, 64, 128])), I=int(np.lcm(a, b)) * 8 * int(g.integers(1, 12)))
+    T = int(g.choice([8, 16, 32]))
+    S = int(g.integers(1, 10))
+    lens = [int(x) for x in g.integers(0, int(g.choice([3, 40, 300])) * T, size=S)]
+    form = "mask" if g.random() < 0.35 else "list"
+    kw = dict(T=T, dst_form=form, seed=seed, fused_qkv=bool(g.integers(2)), fused_gate_up=bool(g.integers(2)),
+              weights=bool(g.integers(2)) and m["hidden"] * max(m["I"], m["Hq"] * m["D"]) < 3e6,
+              src_order=int(g.random() < 0.3), dst_order=int(g.random() < 0.3), src_free=float(g.choice([0.0, 0.2, 0.5])))
+    path = int(g.choice([LDST, BULK, PAIR, PAIR]))
+    opts = [(A.OPT_CHUNK_BYTES, int(g.choice([256, 1024, 2048, 4096, 8192, 16384, 32768])))]
+    for opt, lo, hi, p in ((A.OPT_STAGES, 2, 9, 0.5), (A.OPT_WARPS, 1, 9, 0.5), (A.OPT_LAG, 1, 4, 0.5),
+                           (A.OPT_TENSOR_MAPS, 1, 2, 0.3), (A.OPT_L2_HINT, 1, 5, 0.3)):
+        if g.random() < p:
+            opts.append((opt, int(g.integers(lo, hi))))
+    if g.random() < 0.3:
+        opts.append((A.OPT_MAX_CTAS, int(g.choice([1, 3, 17, 100]))))
+    c = make_case(m, a, b, lens, **kw)
+    kind = int(g.integers(0, 6)) if g.random() < 0.35 and c.n_live > 2 else -1
+    free, bt, cap = None, None, None
+    if kind == 0 and form == "list":
+        fl = c.free_list.copy()
+        i, j = g.choice(c.n_live, 2, replace=False)
+        fl[i] = fl[j]
+        free = (fl, None)
+    elif kind == 1 and form == "list":
+        fl = c.free_list.copy()
+        fl[int(g.integers(0, c.n_live))] = int(g.choice([-1, -7, c.NB_dst, c.NB_dst + 5, 2**31 - 1]))
+        free = (fl, None)
+    elif kind == 2:
+        bt = c.src_bt.copy()
+        rows, cols = np.nonzero(bt >= 0)
+        k = int(g.integers(0, len(rows)))
+        bt[rows[k], cols[k]] = int(g.choice([-1, -5, c.NB_src, c.NB_src + 3, 2**31 - 1]))
+    elif kind == 3:
+        cap = int(g.integers(0, c.n_live))
+    elif kind == 4 and form == "list":
+        free = (c.free_list[:int(g.integers(1, c.n_live))].copy(), None)
+    elif kind == 5:
+        lens[int(g.integers(0, S))] = -int(g.integers(1, 50))
+    if kind >= 0:
+        c = make_case(m, a, b, lens, free_override=free, src_bt_override=bt, pairs_cap=cap, **kw)
+    try:
+        check_case(c, run_case(c, path, options=opts))
+    except Exception as e:
+        raise AssertionError(f"m={m} T={T} {a}->{b} lens {lens} {kw} path {path} opts {opts} damaged {kind}: {e}") from e
+
+
 @pytest.mark.parametrize("a,b", [(32, 1), (1, 32), (32, 32), (16, 32)])
 def test_largest_tp_degrees(a, b):
     """The largest worker counts the library accepts: 32 pools on a side, one header per worker."""
