@@ -201,6 +201,45 @@ def test_side_stream():
     check_case(c, s)
 
 
+def test_host_threads_with_their_own_plans_and_streams():
+    """The library is thread-compatible: host threads that use different plans may call it at the same time (the
+    binding releases the interpreter lock inside every call).  Four threads, each with its own plan, buffers and
+    stream - two of them with token-first pools, whose tensor maps are cached per plan - run their transformation
+    twenty times while the others do; every result is compared with the oracle."""
+    import threading
+
+    import torch
+
+    cases = [make_case(GQA, 1, 4, [300, 77, 45], seed=31), make_case(GQA, 4, 2, [100, 37, 200], seed=32),
+             make_case(GQA, 2, 4, [64, 500], seed=33, weights=False, src_order=TF, dst_order=HC),
+             make_case(GQA, 2, 1, [250, 9, 9], seed=34, weights=False, src_order=TF, dst_order=TF)]
+    paths = [PAIR, LDST, PAIR, BULK]
+    sessions = [run_case(c, p, steps=0) for c, p in zip(cases, paths)]
+    streams = [torch.cuda.Stream() for _ in cases]
+    errors = []
+    go = threading.Barrier(len(cases))
+
+    def work(s, st):
+        try:
+            torch.cuda.set_device(0)
+            go.wait()
+            for _ in range(20):
+                s.step(st)
+            st.synchronize()
+        except Exception as e:  # surfaced below: an exception in a thread would otherwise be lost
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(s, st)) for s, st in zip(sessions, streams)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    for c, s in zip(cases, sessions):
+        check_case(c, s)
+
+
 # ---- token-first storage order (Sec. 3.1: the layout of mainstream engines) on either or both sides
 HC, TF = 0, 1
 ORDERS = [(TF, TF), (TF, HC), (HC, TF)]
