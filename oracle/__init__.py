@@ -247,6 +247,26 @@ def assign_blocks(seq_lens, T, src_bt, NB_src, NB_dst, free_list=None, free_mask
     return dst_bt, pairs[:npairs.value].copy(), npairs.value, nfree.value, st.value
 
 
+def pairs_by_destination(pairs, dst_bt, seq_lens, T):
+    """The work list of ``assign_blocks`` / ``kv_reshape_inplace`` (entry k = the k-th block in (sequence, block) order)
+    listed the other way the table calls offer: ascending by the destination id each block was given, and the blocks
+    that were given none - their entries are (-1,-1) - at the end.  The paper fixes no order of the migration work
+    (Sec. 3.1); the set of pairs is the same in both orders.  ``dst_bt`` is the destination table of the same call
+    (-1 where a block got no id).  Plain loops."""
+    pairs = np.asarray(pairs, dtype=np.int32).reshape(-1, 2)
+    if len(pairs) == 0:  # a call that failed as a whole lists nothing
+        return pairs
+    given, k = [], 0
+    for s, length in enumerate(seq_lens):
+        for i in range((max(int(length), 0) + T - 1) // T):
+            given.append((int(dst_bt[s][i]), k))
+            k += 1
+    assert k == len(pairs)
+    with_id = sorted(e for e in given if e[0] >= 0)  # destination ids are distinct: no ties
+    out = [pairs[k] for _, k in with_id] + [(-1, -1)] * (len(given) - len(with_id))
+    return np.asarray(out, dtype=np.int32).reshape(-1, 2)
+
+
 
 def kv_split_inplace(m, T, N, a, NB, seq_lens, bt, pools, status=0, layer_stride=None):
     """The way back from ``kv_merge_inplace``: one instance of TP=N*a becomes N instances of TP=a in place.

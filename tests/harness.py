@@ -15,18 +15,8 @@ class Case:
 
 
 def pairs_in_destination_order(pairs, dst_bt, seq_lens, T):
-    """The oracle's pair list (entry k = k-th block in (sequence, block) order) in the order the library writes it by
-    default: ascending by the destination id each block was given, the pairs of blocks that were given none - they are
-    (-1,-1) - at the end.  `dst_bt` is the oracle's destination table (-1 where a block got no id)."""
-    pairs = np.asarray(pairs, np.int32).reshape(-1, 2)
-    if len(pairs) == 0:
-        return pairs
-    nblk = (np.maximum(np.asarray(seq_lens, np.int64), 0) + T - 1) // T
-    given = np.concatenate([np.asarray(dst_bt)[s, :n] for s, n in enumerate(nblk)])
-    assert len(given) == len(pairs)
-    has = given >= 0
-    order = np.flatnonzero(has)[np.argsort(given[has], kind="stable")]
-    return np.concatenate([pairs[order], np.full((int((~has).sum()), 2), -1, np.int32)])
+    """The oracle's pair list in the order the library writes it by default (ascending by destination id)."""
+    return oracle.pairs_by_destination(pairs, dst_bt, seq_lens, T)
 
 
 def make_case(model, a, b, seq_lens, T=16, src_free=0.2, dst_form="list", dst_slack=0.25, dst_occupied=0.3, seed=0,

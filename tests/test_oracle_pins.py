@@ -596,3 +596,22 @@ def test_assign_blocks_refuses_an_id_handed_out_twice(oracle):
     assert tuple(pairs[3]) == (-1, -1) and tuple(pairs[1]) == (int(bt[0, 1]), 7)
     given = [x for x in flat if x >= 0]
     assert len(set(given)) == len(given)
+
+
+def test_pairs_by_destination_worked_by_hand(oracle):
+    """The other order of the work list, on an input small enough to sort by hand: five blocks, one of which is refused
+    its destination (id 7 is named twice) and one of which has a bad source id but a good destination."""
+    T, NB = 4, 12
+    seq_lens = [12, 7]                                   # 3 + 2 blocks
+    bt = np.array([[5, 1, 9], [2, 30, -1]], np.int32)    # block 4 names source id 30 of a pool with 12 blocks
+    free = np.array([7, 3, 7, 0, 4, 6], np.int32)
+    dst_bt, pairs, n, left, st = oracle.assign_blocks(seq_lens, T, bt, NB, NB, free_list=free)
+    assert st == oracle.BAD_BLOCK_ID and n == 5
+    assert dst_bt.tolist() == [[7, 3, -1], [0, 4, -1]]
+    assert pairs.tolist() == [[5, 7], [1, 3], [-1, -1], [2, 0], [-1, -1]]          # (sequence, block) order
+    by_dst = oracle.pairs_by_destination(pairs, dst_bt, seq_lens, T)
+    #          dst 0    dst 3   dst 4: bad source   dst 7   the refused block
+    assert by_dst.tolist() == [[2, 0], [1, 3], [-1, -1], [5, 7], [-1, -1]]
+    # a call that failed as a whole lists nothing in either order
+    dst_bt, pairs, n, _, st = oracle.assign_blocks(seq_lens, T, bt, NB, NB, free_list=free[:2])
+    assert st == oracle.NO_FREE_BLOCKS and n == 0 and len(oracle.pairs_by_destination(pairs, dst_bt, seq_lens, T)) == 0
