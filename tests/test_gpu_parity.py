@@ -687,7 +687,23 @@ def test_weights_compacted_in_place_mha(fq, hidden, a, b, keep):
     _compact_case(m, PAIR, fq, True, a, b, keep)
 
 
-def _compact_case(m, path, fq, fg, a, b, keep):
+@pytest.mark.parametrize("seed", range(40))
+def test_random_compactions(seed):
+    """Seeded random shapes for the partial swap: factor, worker count, kept parts, head counts, row counts from 16 to
+    2500 (a quarter of the seeds pass the rows one CTA moves alone), fused or separate buffers, copy path, item size."""
+    g = np.random.default_rng(4400 + seed)
+    N, a = int(g.choice([2, 4, 8])), int(g.choice([1, 2, 4]))
+    b = a * N
+    Hkv = b * int(g.choice([1, 2]))
+    big = seed % 4 == 0
+    m = dict(L=int(g.integers(1, 3)), hidden=16 * int(g.integers(1, 160 if big else 24)), Hq=Hkv * int(g.choice([1, 2, 4])),
+             Hkv=Hkv, D=int(g.choice([16, 32, 64])), I=b * 8 * int(g.integers(1, 64 if big else 12)))
+    keep = [int(g.integers(0, N)) for _ in range(a)]
+    _compact_case(m, int(g.choice([LDST, BULK, PAIR, PAIR])), bool(g.integers(2)), bool(g.integers(2)), a, b, keep,
+                  chunk=int(g.choice([256, 1024, 4096, 8192, 16384])))
+
+
+def _compact_case(m, path, fq, fg, a, b, keep, chunk=1024):
     import torch
 
     import oracle as O
@@ -699,7 +715,7 @@ def _compact_case(m, path, fq, fg, a, b, keep):
     plan = A.amoeba_plan_create(A.make_layout(m, a, 4, fused_qkv=fq, fused_gate_up=fg),
                                 A.make_layout(m, b, 4, fused_qkv=fq, fused_gate_up=fg))
     A.amoeba_plan_set_option(plan, A.OPT_COPY_PATH, path)
-    A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, 1024)
+    A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, chunk)
     bufs, exp = [[None] * m["L"] for _ in range(a)], []
     for l in range(m["L"]):
         W = {n: g.integers(0, 65536, size=s, dtype=np.uint16) for n, s in O.logical_shapes(m).items()}
@@ -716,7 +732,7 @@ def _compact_case(m, path, fq, fg, a, b, keep):
         for l in range(m["L"]):
             for n, e in exp[l][w].items():
                 got = bufs[r][l][n].cpu().numpy().view(np.uint16)[:e.size]
-                assert np.array_equal(got, e.reshape(-1)), (r, l, n)
+                assert np.array_equal(got, e.reshape(-1)), (r, l, n, m, a, b, keep, path, fq, fg, chunk)
 
 
 def test_weights_compaction_host_errors():
