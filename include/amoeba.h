@@ -286,7 +286,9 @@ AMOEBA_API amoeba_status amoeba_rewrite_block_tables_builtin_scratch(
  * src_pools[h / (Hkv/a)] to dst_pools[h / (Hkv/b)], read at the addresses of the source layout's kv_order and
  * written at those of the destination layout's kv_order.
  * src_pools / dst_pools are HOST arrays of a / b device pointers (read during the call only).
- * A pair with an id outside its pool is skipped and sets BAD_BLOCK_ID in *d_status.
+ * A pair with an id outside its pool is skipped and sets BAD_BLOCK_ID in *d_status.  The list may be in any order -
+ * the result is the same - provided no destination id appears twice (amoeba_rewrite_block_tables never lists one
+ * twice); the order only decides in which order DRAM is visited (see AMOEBA_OPT_PAIR_ORDER).
  */
 AMOEBA_API amoeba_status amoeba_reshard_kv(const amoeba_plan* plan, const void* const* src_pools, void* const* dst_pools,
                                 const int32_t* d_pairs, const int32_t* d_num_pairs, int32_t pairs_cap,
