@@ -110,6 +110,11 @@ def test_layout_validation():
     A.amoeba_plan_set_option(plan, A.OPT_CHUNK_BYTES, 1024)
     assert A.amoeba_plan_kv_info(plan).chunk_bytes == 1024
     assert A.amoeba_rewrite_workspace_bytes(plan, 10, 100) >= 64 + 44 + 4 * 8  # header, offsets, one word per block id
+    for order in (0, A.PAIR_ORDER_TABLE, A.PAIR_ORDER_DESTINATION):
+        A.amoeba_plan_set_option(plan, A.OPT_PAIR_ORDER, order)
+    with pytest.raises(A.AmoebaError) as e:
+        A.amoeba_plan_set_option(plan, A.OPT_PAIR_ORDER, 3)  # no such order
+    assert e.value.status == A.ERR_INVALID_ARG
 
 
 def test_no_device_means_cuda_error_not_a_fallback():
