@@ -257,6 +257,41 @@ def test_split_matches_oracle(oracle, N, a):
         assert np.array_equal(g, e), w
 
 
+def _random_instances(oracle, seed):
+    g = np.random.default_rng(9100 + seed)
+    Hkv = int(g.choice([2, 4, 8, 16]))
+    N = int(g.choice([x for x in (2, 4, 8) if Hkv % x == 0]))
+    a = int(g.choice([x for x in (1, 2, 4) if Hkv % (x * N) == 0]))
+    m = dict(L=int(g.integers(1, 4)), hidden=64, Hq=Hkv, Hkv=Hkv, D=int(g.choice([16, 32, 64])), I=64 * N * a)
+    T = int(g.choice([4, 8, 16]))
+    lens_pi = [[int(x) for x in g.integers(0, 12 * T, size=int(g.integers(1, 6)))] for _ in range(N)]
+    NB = max(sum((l + T - 1) // T for l in li) for li in lens_pi) + int(g.integers(1, 9))
+    lens, bt, pools = _instances(oracle, m, T, N, a, NB, lens_pi, seed=seed)
+    return g, m, T, N, a, NB, lens, bt, pools
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_merges_and_splits(oracle, seed):
+    """Seeded random shapes, instance counts, worker counts, block sizes, lengths and ring shapes: the merge against the
+    oracle, then - from the oracle's merged state with every unnamed block overwritten - the split back."""
+    import paper_2509_19729_b200 as A
+
+    g, m, T, N, a, NB, lens, bt, pools = _random_instances(oracle, seed)
+    opts = [(A.OPT_COPY_PATH, int(g.choice([2, 3]))), (A.OPT_CHUNK_BYTES, int(g.choice([32, 256, 2048, 8192, 65536]))),
+            (A.OPT_WARPS, int(g.integers(1, 8))), (A.OPT_STAGES, int(g.integers(2, 8)))]
+    _check(oracle, m, T, N, a, NB, lens, bt, [p.copy() for p in pools], options=opts)
+    merged_bt, _, st = oracle.kv_merge_inplace(m, T, N, a, NB, lens, bt, pools)
+    assert st == 0
+    _scribble_free_blocks(m, T, N, a, NB, merged_bt, pools, seed=seed)
+    exp_pools = [p.copy() for p in pools]
+    exp_bt, exp_live, exp_status = oracle.kv_split_inplace(m, T, N, a, NB, lens, merged_bt, exp_pools)
+    got_pools, got_bt, got_live, got_status = _run_split(m, T, N, a, NB, lens, merged_bt, pools)
+    assert got_status == exp_status == 0
+    assert np.array_equal(got_bt, exp_bt) and np.array_equal(got_live, exp_live)
+    for w, (x, e) in enumerate(zip(got_pools, exp_pools)):
+        assert np.array_equal(x, e), (w, m, T, N, a, NB)
+
+
 def test_split_device_detected_errors(oracle):
     m, T, N, a, NB = MHA8, 4, 2, 1, 9
     lens, bt, pools = _instances(oracle, m, T, N, a, NB, [[8, 4, 20], [5, 9]], seed=2)
